@@ -1,0 +1,155 @@
+/*
+ * stief.h -- C boundary of the B200 (sm_100a) library for decode attention over a KV cache that is
+ * stored, per KV head, as projections onto column-orthonormal bases:
+ *
+ *     K_down = K U_k  in R^{n x r_k},   V_down = V U_v  in R^{n x r_v}          (paper Eq. 1, Sec. 3.2)
+ *
+ * and attended through the reconstructions K_tilde = K_down U_k^T, V_tilde = V_down U_v^T
+ * (Eq. 2 / Eq. 7) with ordinary per-head attention softmax(q K_tilde^T / sqrt(d_h)) V_tilde (Eq. 18).
+ * Because q K_tilde^T = (q U_k) K_down^T and p V_tilde = (p V_down) U_v^T, everything is evaluated
+ * in the compressed space and the reconstructions are never formed.
+ *
+ * General rules
+ *  - Every pointer below is a DEVICE pointer unless its name ends in _host.  The caller owns all
+ *    memory.  No entry point allocates, frees or synchronises; all work is enqueued on `stream`
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *  - bf16 tensors are passed as uint16_t* (raw bit patterns).  d_h must be 128.  Ranks must be one of
+ *    32, 48, 64, 96, 128 (STIEF_ERR_UNSUPPORTED otherwise).  Ranks are per layer, equal across heads.
+ *  - Return value: a stief_status for problems the host can see (bad arguments, launch failure).
+ *    Problems only the device can see (a page id outside the pool, a position beyond the block
+ *    table, a wait that ran out) are reported through the optional `status` word: a device int32
+ *    the caller zeroes; the first error code wins; read it after synchronising.  A kernel that
+ *    detects such a problem skips or redirects the offending access; it never traps.
+ *  - Cache layout (bit-exact contract): pools are [num_pages][Hkv][64][r] bf16, r fastest.  Token t
+ *    of sequence b, KV head h, lives at element ((block_table[b][t/64]*Hkv + h)*64 + t%64)*r.
+ *    Rows of a page at or beyond the sequence length are unspecified and never influence a result.
+ *  - Query head g reads KV head g / (Hq/Hkv) (contiguous GQA groups).
+ *  - The softmax scale is always 1/sqrt(d_h) = 1/sqrt(128), never 1/sqrt(r_k): attention is defined
+ *    on tensors of the original dimension (Eq. 7, Eq. 18).
+ *  - RoPE (or any other positional map) is the caller's business: k, q arrive as the attention block
+ *    sees them.
+ */
+#ifndef STIEF_H_
+#define STIEF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum stief_status {
+  STIEF_OK = 0,
+  STIEF_ERR_INVALID_ARG = 1,  /* NULL/misaligned pointer, bad shape                                    */
+  STIEF_ERR_UNSUPPORTED = 2,  /* rank or head dimension not compiled in                                */
+  STIEF_ERR_WORKSPACE = 3,    /* workspace too small for the requested number of splits                */
+  STIEF_ERR_CUDA = 4,         /* a CUDA runtime/driver call failed (cudaGetLastError is left readable) */
+  STIEF_ERR_BOUNDS = 5,       /* device-side: page id or position out of range (status word only)      */
+  STIEF_ERR_TIMEOUT = 6       /* device-side: a bounded wait on an async copy ran out (status word)    */
+};
+
+#define STIEF_PAGE 64
+#define STIEF_D_HEAD 128
+
+/* One decoder layer's compressed cache and bases.
+ * U_k: [Hkv][128][r_k] bf16 row-major (r fastest) with head stride uk_head_stride elements; stride 0
+ * means one key basis shared by all heads of the layer (the paper's head-sharing scheme, Sec. 3.3).
+ * U_v: [Hkv][128][r_v], per-head value bases (stride 128*r_v) or shared (stride 0).
+ * A NULL basis keeps that side full rank (Algorithm 2 lets a layer keep keys or values
+ * uncompressed): the rank must then be 128 and rows are stored / used unprojected.
+ * The same U buffers serve compression, query projection and back-projection.
+ * Alignment: pools and bases 128 bytes. */
+typedef struct stief_layer {
+  int32_t Hq, Hkv, d;
+  int32_t r_k, r_v;
+  int32_t num_pages;
+  const uint16_t* U_k;
+  int64_t uk_head_stride;
+  const uint16_t* U_v;
+  int64_t uv_head_stride;
+  uint16_t* k_pool; /* [num_pages][Hkv][64][r_k] */
+  uint16_t* v_pool; /* [num_pages][Hkv][64][r_v] */
+} stief_layer;
+
+/* Paging state of the batch, shared by all layers.  block_table is [B][max_pages_per_seq] int32
+ * page ids; seq_lens is [B] int32.  The library never writes either. */
+typedef struct stief_batch {
+  int32_t B, max_pages_per_seq;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+} stief_batch;
+
+/* Eq. 1 for a whole prompt: for every b, t < seq_lens[b], h: K_down[t,h,:] = rnd_bf16(K[b,t,h,:] U_k[h])
+ * and the same for V, accumulated in fp32, stored to the paged pools.  K, V are bf16 with element
+ * strides stride_b (between sequences) and stride_t (between tokens); heads are contiguous blocks of
+ * 128 elements; rows must be 16-byte aligned.  T_max bounds seq_lens (it sizes the launch; tokens
+ * beyond seq_lens[b] are not read). */
+int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K,
+                           const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
+                           int32_t* status, void* stream);
+
+/* Eq. 1 for one new token per sequence: projects k_new, v_new [B][Hkv][128] and stores the rows at
+ * position seq_lens[b] (the page block_table[b][seq_lens[b]/64] must already be assigned).  The
+ * caller advances its seq_lens afterwards (stief_advance_seq_lens does it on the device). */
+int stief_append(const stief_layer* layer, const stief_batch* batch, const uint16_t* k_new,
+                 const uint16_t* v_new, int32_t* status, void* stream);
+
+/* Split-T planning.  The context of every sequence is cut into at most S chunks of
+ * chunk_pages = ceil(max_pages_per_seq / S) pages; chunk s covers pages [s*chunk_pages, (s+1)*chunk_pages)
+ * clipped to the sequence.  stief_decode_num_splits proposes S for the current device;
+ * stief_decode_workspace_bytes sizes the scratch buffer for a given S.  Workspace layout (fp32):
+ *   q_proj      [B][Hq][r_k]        scaled projected queries (q U_k) * log2(e)/sqrt(128)
+ *   partial_o   [B][Hq][S][r_v]     chunk-normalised mixes p V_down (compressed space)
+ *   partial_lse [B][Hq][S]          natural-log sum-exp of each chunk's scores
+ * The buffer must be 128-byte aligned. */
+int32_t stief_decode_num_splits(int32_t B, int32_t Hkv, int32_t max_pages_per_seq);
+size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t r_k, int32_t r_v, int32_t num_splits);
+
+/* Decode attention (Eq. 18 on the reconstructions of Eq. 7, one query row per head): q [B][Hq][128]
+ * bf16 attends to tokens [0, seq_lens[b] + len_add) of every sequence; len_add is 0, or 1 when the
+ * token of this step was appended on the same stream and seq_lens not yet advanced.  Runs the query
+ * projection, the split-T kernel (scores, online softmax, mix, all in the compressed space) and, when
+ * `out` is not NULL, stief_split_combine.  out [B][Hq][128] bf16; out_lse [B][Hq] fp32 natural-log
+ * sum-exp, optional.  A sequence of length 0 yields a zero row and lse = -inf.
+ * num_splits 0 lets the library choose (the workspace must then hold stief_decode_num_splits splits). */
+int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
+                           int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_splits,
+                           uint16_t* out, float* out_lse, int32_t* status, void* stream);
+
+/* Merge of the per-chunk results by log-sum-exp (an exact re-association of Eq. 18) followed by the
+ * back-projection o = o_down U_v^T (Eq. 7 applied to the mixed values; linear, so done once after the
+ * merge).  Reads the workspace written by stief_decode_attention with the same batch, len_add and
+ * num_splits.  Chunks beyond a sequence's length weigh nothing and are never read. */
+int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int32_t len_add,
+                        const void* workspace, int32_t num_splits, uint16_t* out, float* out_lse,
+                        int32_t* status, void* stream);
+
+/* One decode step of one layer: append (k_new, v_new) at seq_lens[b], then attend over
+ * seq_lens[b] + 1 tokens.  Same result as stief_append followed by stief_decode_attention with
+ * len_add = 1, in fewer launches. */
+int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
+                      const uint16_t* k_new, const uint16_t* v_new, void* workspace,
+                      size_t workspace_bytes, int32_t num_splits, uint16_t* out, float* out_lse,
+                      int32_t* status, void* stream);
+
+/* The same step for callers whose activations live in host memory: q_host, k_new_host, v_new_host
+ * are copied to `staging` (device, stief_host_staging_bytes) with cudaMemcpyAsync on `stream`, the
+ * step runs, and out is copied back to out_host.  Nothing is synchronised: the caller waits on the
+ * stream before reading out_host.  Host buffers should be pinned for the copies to be asynchronous. */
+size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
+int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
+                           const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging,
+                           void* workspace, size_t workspace_bytes, int32_t num_splits,
+                           uint16_t* out_host, int32_t* status, void* stream);
+
+/* seq_lens[b] += delta on the device (so a captured step can be replayed). */
+int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream);
+
+const char* stief_status_string(int status);
+int stief_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STIEF_H_ */

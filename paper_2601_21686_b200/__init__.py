@@ -1,0 +1,199 @@
+"""Python binding of libstief.so: decode attention over a rank-compressed KV cache on B200.
+
+Argument marshalling only.  Every function has the name and the meaning of the C entry point
+declared in ``include/stief.h``; tensors are torch CUDA tensors used as device memory, and the work is
+enqueued on torch's current stream.  There is no fallback: if the CUDA library has not been built the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libstief.so")
+
+STIEF_OK, STIEF_ERR_INVALID_ARG, STIEF_ERR_UNSUPPORTED, STIEF_ERR_WORKSPACE = 0, 1, 2, 3
+STIEF_ERR_CUDA, STIEF_ERR_BOUNDS, STIEF_ERR_TIMEOUT = 4, 5, 6
+PAGE = 64
+D_HEAD = 128
+
+
+class StiefError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class _CLayer(ctypes.Structure):
+    _fields_ = [("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("r_k", ctypes.c_int32), ("r_v", ctypes.c_int32), ("num_pages", ctypes.c_int32),
+                ("U_k", ctypes.c_void_p), ("uk_head_stride", ctypes.c_int64),
+                ("U_v", ctypes.c_void_p), ("uv_head_stride", ctypes.c_int64),
+                ("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p)]
+
+
+class _CBatch(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+                ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p)]
+
+
+_lib_handle = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library (loads it on first use; raises if it was never built)."""
+    global _lib_handle
+    if _lib_handle is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_21686_b200.build` "
+                               "(there is no non-CUDA path)")
+        L = ctypes.CDLL(LIB_PATH)
+        P, I32, I64, SZ = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        LP, BP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch)
+        sig = {
+            "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, P, P]),
+            "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
+            "stief_decode_num_splits": (I32, [I32, I32, I32]),
+            "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
+            "stief_decode_attention": (ctypes.c_int, [LP, BP, P, I32, P, SZ, I32, P, P, P, P]),
+            "stief_split_combine": (ctypes.c_int, [LP, BP, I32, P, I32, P, P, P, P]),
+            "stief_decode_step": (ctypes.c_int, [LP, BP, P, P, P, P, SZ, I32, P, P, P, P]),
+            "stief_host_staging_bytes": (SZ, [I32, I32, I32]),
+            "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, P, P]),
+            "stief_advance_seq_lens": (ctypes.c_int, [P, I32, I32, P]),
+            "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+            "stief_version": (ctypes.c_int, []),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib_handle = L
+    return _lib_handle
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+@dataclass
+class Layer:
+    """One decoder layer's compressed cache and bases (device tensors).  U_k [Hkv or 1, 128, r_k],
+    U_v [Hkv or 1, 128, r_v] bf16 (None = that side kept full rank); pools [num_pages, Hkv, 64, r] bf16."""
+    Hq: int
+    Hkv: int
+    r_k: int
+    r_v: int
+    U_k: Optional[torch.Tensor]
+    U_v: Optional[torch.Tensor]
+    k_pool: torch.Tensor
+    v_pool: torch.Tensor
+
+    @property
+    def num_pages(self) -> int:
+        return self.k_pool.shape[0]
+
+    def c(self) -> _CLayer:
+        uk_stride = 0 if self.U_k is None or self.U_k.shape[0] == 1 else self.U_k.stride(0)
+        uv_stride = 0 if self.U_v is None or self.U_v.shape[0] == 1 else self.U_v.stride(0)
+        return _CLayer(self.Hq, self.Hkv, D_HEAD, self.r_k, self.r_v, self.num_pages, _ptr(self.U_k), uk_stride,
+                       _ptr(self.U_v), uv_stride, _ptr(self.k_pool), _ptr(self.v_pool))
+
+
+@dataclass
+class Batch:
+    """Paging state: block_table [B, max_pages_per_seq] int32, seq_lens [B] int32 (device tensors)."""
+    block_table: torch.Tensor
+    seq_lens: torch.Tensor
+
+    def c(self) -> _CBatch:
+        return _CBatch(self.block_table.shape[0], self.block_table.shape[1], _ptr(self.block_table), _ptr(self.seq_lens))
+
+
+def _check(rc: int, where: str):
+    if rc != STIEF_OK:
+        raise StiefError(rc, where)
+
+
+def status_string(code: int) -> str:
+    return lib().stief_status_string(code).decode()
+
+
+def stief_version() -> int:
+    return lib().stief_version()
+
+
+def stief_prefill_compress(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
+                           status: Optional[torch.Tensor] = None):
+    """K, V [B, T, Hkv, 128] bf16 (strides over b and t free, heads and d contiguous) -> paged compressed cache."""
+    assert K.stride(3) == 1 and K.stride(2) == D_HEAD and V.stride() == K.stride()
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_prefill_compress(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
+                                        K.shape[1] if T_max is None else T_max, _ptr(status), _stream()),
+           "stief_prefill_compress")
+
+
+def stief_append(layer: Layer, batch: Batch, k_new: torch.Tensor, v_new: torch.Tensor, status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_append(ctypes.byref(cl), ctypes.byref(cb), _ptr(k_new), _ptr(v_new), _ptr(status), _stream()),
+           "stief_append")
+
+
+def stief_decode_num_splits(B: int, Hkv: int, max_pages_per_seq: int) -> int:
+    return lib().stief_decode_num_splits(B, Hkv, max_pages_per_seq)
+
+
+def stief_decode_workspace_bytes(B: int, Hq: int, r_k: int, r_v: int, num_splits: int) -> int:
+    return lib().stief_decode_workspace_bytes(B, Hq, r_k, r_v, num_splits)
+
+
+def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, num_splits: int = 0,
+                           out: Optional[torch.Tensor] = None, out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
+                           status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), num_splits, _ptr(out), _ptr(out_lse),
+                                        _ptr(status), _stream()), "stief_decode_attention")
+
+
+def stief_split_combine(layer: Layer, batch: Batch, workspace: torch.Tensor, num_splits: int, out: torch.Tensor,
+                        out_lse: Optional[torch.Tensor] = None, len_add: int = 0, status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_split_combine(ctypes.byref(cl), ctypes.byref(cb), len_add, _ptr(workspace), num_splits, _ptr(out),
+                                     _ptr(out_lse), _ptr(status), _stream()), "stief_split_combine")
+
+
+def stief_decode_step(layer: Layer, batch: Batch, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                      workspace: torch.Tensor, out: torch.Tensor, num_splits: int = 0, out_lse: Optional[torch.Tensor] = None,
+                      status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_decode_step(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), num_splits, _ptr(out), _ptr(out_lse),
+                                   _ptr(status), _stream()), "stief_decode_step")
+
+
+def stief_host_staging_bytes(B: int, Hq: int, Hkv: int) -> int:
+    return lib().stief_host_staging_bytes(B, Hq, Hkv)
+
+
+def stief_decode_step_host(layer: Layer, batch: Batch, q_host: torch.Tensor, k_new_host: torch.Tensor, v_new_host: torch.Tensor,
+                           staging: torch.Tensor, workspace: torch.Tensor, out_host: torch.Tensor, num_splits: int = 0,
+                           status: Optional[torch.Tensor] = None):
+    """Host (pinned) q/k/v/out buffers; copies and kernels are enqueued, nothing is synchronised."""
+    assert not q_host.is_cuda and not out_host.is_cuda
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_decode_step_host(ctypes.byref(cl), ctypes.byref(cb), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
+                                        _ptr(staging), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                        num_splits, _ptr(out_host), _ptr(status), _stream()), "stief_decode_step_host")
+
+
+def stief_advance_seq_lens(seq_lens: torch.Tensor, delta: int = 1):
+    _check(lib().stief_advance_seq_lens(_ptr(seq_lens), seq_lens.numel(), delta, _stream()), "stief_advance_seq_lens")

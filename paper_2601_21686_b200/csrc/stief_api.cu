@@ -1,0 +1,340 @@
+// C-ABI entry points: argument checks, split planning, workspace carving, tensor-map encoding and
+// kernel launches.  No allocation, no synchronisation; everything is enqueued on the caller's stream.
+#include <cstring>
+
+#include "stief_kernels.h"
+
+namespace stief {
+
+cudaError_t launch_decode_rk32(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
+cudaError_t launch_decode_rk48(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
+cudaError_t launch_decode_rk64(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
+cudaError_t launch_decode_rk96(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
+cudaError_t launch_decode_rk128(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
+
+cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st) {
+  switch (a.L.r_k) {
+    case 32: return launch_decode_rk32(a, tmK, tmV, st);
+    case 48: return launch_decode_rk48(a, tmK, tmV, st);
+    case 64: return launch_decode_rk64(a, tmK, tmV, st);
+    case 96: return launch_decode_rk96(a, tmK, tmV, st);
+    case 128: return launch_decode_rk128(a, tmK, tmV, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+int decode_box_width(int r) { return (r % 64 == 0) ? 64 : (r % 32 == 0) ? 32 : 16; }
+
+namespace {
+
+bool rank_ok(int r) { return r == 32 || r == 48 || r == 64 || r == 96 || r == 128; }
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_layer(const stief_layer* l) {
+  if (!l) return STIEF_ERR_INVALID_ARG;
+  if (l->Hq <= 0 || l->Hkv <= 0 || l->Hq % l->Hkv != 0 || l->num_pages <= 0) return STIEF_ERR_INVALID_ARG;
+  if (l->d != kD) return STIEF_ERR_UNSUPPORTED;
+  if (!rank_ok(l->r_k) || !rank_ok(l->r_v)) return STIEF_ERR_UNSUPPORTED;
+  if (!l->k_pool || !l->v_pool || !aligned(l->k_pool, 128) || !aligned(l->v_pool, 128)) return STIEF_ERR_INVALID_ARG;
+  if ((l->U_k && !aligned(l->U_k, 128)) || (l->U_v && !aligned(l->U_v, 128))) return STIEF_ERR_INVALID_ARG;
+  if ((!l->U_k && l->r_k != kD) || (!l->U_v && l->r_v != kD)) return STIEF_ERR_INVALID_ARG;
+  if (l->uk_head_stride < 0 || l->uv_head_stride < 0) return STIEF_ERR_INVALID_ARG;
+  if ((l->uk_head_stride % 64) != 0 || (l->uv_head_stride % 64) != 0) return STIEF_ERR_INVALID_ARG;   // keeps every head's basis 128-byte aligned
+  if ((long long)l->num_pages * l->Hkv * kPage >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
+  return STIEF_OK;
+}
+int check_batch(const stief_batch* b) {
+  if (!b || b->B <= 0 || b->max_pages_per_seq <= 0 || !b->block_table || !b->seq_lens) return STIEF_ERR_INVALID_ARG;
+  if (b->B > 65535) return STIEF_ERR_INVALID_ARG;
+  return STIEF_OK;
+}
+
+LayerDev to_dev(const stief_layer* l) {
+  LayerDev d;
+  d.Hq = l->Hq; d.Hkv = l->Hkv; d.G = l->Hq / l->Hkv; d.r_k = l->r_k; d.r_v = l->r_v; d.num_pages = l->num_pages;
+  d.U_k = reinterpret_cast<const __nv_bfloat16*>(l->U_k); d.uk_stride = l->uk_head_stride;
+  d.U_v = reinterpret_cast<const __nv_bfloat16*>(l->U_v); d.uv_stride = l->uv_head_stride;
+  d.k_pool = reinterpret_cast<__nv_bfloat16*>(l->k_pool); d.v_pool = reinterpret_cast<__nv_bfloat16*>(l->v_pool);
+  return d;
+}
+BatchDev to_dev(const stief_batch* b) {
+  BatchDev d;
+  d.B = b->B; d.max_pages = b->max_pages_per_seq; d.block_table = b->block_table; d.seq_lens = b->seq_lens;
+  return d;
+}
+
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return 148;
+  }
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = 148;
+    }
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+// The one place that turns (max_pages, requested splits) into (chunk_pages, S): decode and combine
+// must agree on it because it fixes the workspace layout.
+void plan_splits(int max_pages, int requested, int* chunk_pages, int* S) {
+  int s = requested < 1 ? 1 : requested;
+  if (s > max_pages) s = max_pages;
+  const int cp = (max_pages + s - 1) / s;
+  *chunk_pages = cp;
+  *S = (max_pages + cp - 1) / cp;
+}
+
+struct Workspace {
+  float* q_proj;
+  float* partial_o;
+  float* partial_lse;
+  size_t bytes;
+};
+Workspace carve(void* base, int B, int Hq, int r_k, int r_v, int S) {
+  Workspace w;
+  size_t off = 0;
+  uint8_t* p = static_cast<uint8_t*>(base);
+  w.q_proj = reinterpret_cast<float*>(p + off);
+  off += align_up((size_t)B * Hq * r_k * 4, 128);
+  w.partial_o = reinterpret_cast<float*>(p + off);
+  off += align_up((size_t)B * Hq * S * r_v * 4, 128);
+  w.partial_lse = reinterpret_cast<float*>(p + off);
+  off += align_up((size_t)B * Hq * S * 4, 128);
+  w.bytes = off;
+  return w;
+}
+
+// ---- tensor maps ----------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// pool viewed as a 2-D bf16 tensor [rows = num_pages*Hkv*64][r]; box = 64 rows x box-width, swizzle span = box row
+bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  const int bw = decode_box_width(r);
+  const cuuint64_t gdim[2] = {(cuuint64_t)r, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)r * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)bw, (cuuint32_t)kPage};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle sw = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  const CUresult rc = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS;
+}
+
+int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+               const uint16_t* v_new, int len_add, void* workspace, size_t workspace_bytes, int num_splits, uint16_t* out,
+               float* out_lse, int32_t* status, cudaStream_t st) {
+  int rc = check_layer(layer);
+  if (rc) return rc;
+  rc = check_batch(batch);
+  if (rc) return rc;
+  if (!q || !aligned(q, 16) || !workspace || !aligned(workspace, 128)) return STIEF_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return STIEF_ERR_INVALID_ARG;
+  if (k_new && (!aligned(k_new, 16) || !aligned(v_new, 16))) return STIEF_ERR_INVALID_ARG;
+  if (out && !aligned(out, 16)) return STIEF_ERR_INVALID_ARG;
+  if (len_add < 0 || len_add > 1) return STIEF_ERR_INVALID_ARG;
+  if (num_splits < 0) return STIEF_ERR_INVALID_ARG;
+  if (num_splits == 0) num_splits = stief_decode_num_splits(batch->B, layer->Hkv, batch->max_pages_per_seq);
+  int chunk_pages, S;
+  plan_splits(batch->max_pages_per_seq, num_splits, &chunk_pages, &S);
+  if (S > 65535 || (long long)layer->Hkv * ((layer->Hq / layer->Hkv + 7) / 8) > 65535) return STIEF_ERR_INVALID_ARG;
+  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->r_k, layer->r_v, S);
+  if (w.bytes > workspace_bytes) return STIEF_ERR_WORKSPACE;
+
+  const LayerDev L = to_dev(layer);
+  const BatchDev Bt = to_dev(batch);
+  const long long rows = (long long)layer->num_pages * layer->Hkv * kPage;
+  CUtensorMap tmK, tmV;
+  if (!make_pool_map(&tmK, layer->k_pool, layer->r_k, rows) || !make_pool_map(&tmV, layer->v_pool, layer->r_v, rows))
+    return STIEF_ERR_CUDA;
+
+  PreArgs pa;
+  pa.L = L; pa.Bt = Bt;
+  pa.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  pa.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
+  pa.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
+  pa.q_proj = w.q_proj; pa.status = status;
+  if (launch_pre(pa, st) != cudaSuccess) return STIEF_ERR_CUDA;
+
+  DecodeLaunch da;
+  da.L = L; da.Bt = Bt; da.q_proj = w.q_proj; da.partial_o = w.partial_o; da.partial_lse = w.partial_lse;
+  da.S = S; da.chunk_pages = chunk_pages; da.len_add = len_add; da.status = status;
+  if (launch_decode(da, tmK, tmV, st) != cudaSuccess) return STIEF_ERR_CUDA;
+
+  if (out) {
+    CombineArgs ca;
+    ca.L = L; ca.Bt = Bt; ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
+    ca.S = S; ca.chunk_pages = chunk_pages; ca.len_add = len_add;
+    ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;
+    if (launch_combine(ca, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  }
+  return STIEF_OK;
+}
+
+}  // namespace
+}  // namespace stief
+
+using namespace stief;
+
+extern "C" {
+
+int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K, const uint16_t* V,
+                           int64_t stride_b, int64_t stride_t, int32_t T_max, int32_t* status, void* stream) {
+  int rc = check_layer(layer);
+  if (rc) return rc;
+  rc = check_batch(batch);
+  if (rc) return rc;
+  if (!K || !V || !aligned(K, 16) || !aligned(V, 16)) return STIEF_ERR_INVALID_ARG;
+  if (T_max <= 0 || stride_t < (int64_t)layer->Hkv * kD || stride_b < 0 || (stride_t % 8) != 0 || (stride_b % 8) != 0)
+    return STIEF_ERR_INVALID_ARG;
+  if (2 * batch->B > 65535) return STIEF_ERR_INVALID_ARG;
+  PrefillArgs a;
+  a.L = to_dev(layer); a.Bt = to_dev(batch);
+  a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);
+  a.stride_b = stride_b; a.stride_t = stride_t; a.T_max = T_max; a.status = status;
+  return launch_prefill(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+int stief_append(const stief_layer* layer, const stief_batch* batch, const uint16_t* k_new, const uint16_t* v_new,
+                 int32_t* status, void* stream) {
+  int rc = check_layer(layer);
+  if (rc) return rc;
+  rc = check_batch(batch);
+  if (rc) return rc;
+  if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return STIEF_ERR_INVALID_ARG;
+  PreArgs pa;
+  pa.L = to_dev(layer); pa.Bt = to_dev(batch);
+  pa.q = nullptr;
+  pa.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
+  pa.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
+  pa.q_proj = nullptr; pa.status = status;
+  return launch_pre(pa, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+int32_t stief_decode_num_splits(int32_t B, int32_t Hkv, int32_t max_pages_per_seq) {
+  if (B <= 0 || Hkv <= 0 || max_pages_per_seq <= 0) return 1;
+  // aim at ~8 work items per SM (two resident CTAs, four rounds), at least 4 pages per item
+  const long long units = (long long)B * Hkv;
+  const long long target = (long long)sm_count() * 8;
+  long long s = (target + units - 1) / units;
+  const long long smax = (max_pages_per_seq + 3) / 4;
+  if (s > smax) s = smax;
+  if (s < 1) s = 1;
+  int chunk_pages, S;
+  plan_splits(max_pages_per_seq, (int)s, &chunk_pages, &S);
+  return S;
+}
+
+size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t r_k, int32_t r_v, int32_t num_splits) {
+  if (B <= 0 || Hq <= 0 || r_k <= 0 || r_v <= 0 || num_splits <= 0) return 0;
+  return carve(nullptr, B, Hq, r_k, r_v, num_splits).bytes;
+}
+
+int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int32_t len_add,
+                           void* workspace, size_t workspace_bytes, int32_t num_splits, uint16_t* out, float* out_lse,
+                           int32_t* status, void* stream) {
+  return run_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_splits, out, out_lse, status,
+                    static_cast<cudaStream_t>(stream));
+}
+
+int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int32_t len_add, const void* workspace,
+                        int32_t num_splits, uint16_t* out, float* out_lse, int32_t* status, void* stream) {
+  (void)status;
+  int rc = check_layer(layer);
+  if (rc) return rc;
+  rc = check_batch(batch);
+  if (rc) return rc;
+  if (!workspace || !aligned(workspace, 128) || !out || !aligned(out, 16) || num_splits < 0 || len_add < 0 || len_add > 1)
+    return STIEF_ERR_INVALID_ARG;
+  if (num_splits == 0) num_splits = stief_decode_num_splits(batch->B, layer->Hkv, batch->max_pages_per_seq);
+  int chunk_pages, S;
+  plan_splits(batch->max_pages_per_seq, num_splits, &chunk_pages, &S);
+  const Workspace w = carve(const_cast<void*>(workspace), batch->B, layer->Hq, layer->r_k, layer->r_v, S);
+  CombineArgs ca;
+  ca.L = to_dev(layer); ca.Bt = to_dev(batch);
+  ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
+  ca.S = S; ca.chunk_pages = chunk_pages; ca.len_add = len_add;
+  ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;
+  return launch_combine(ca, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+                      const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_splits, uint16_t* out,
+                      float* out_lse, int32_t* status, void* stream) {
+  if (!k_new || !v_new || !out) return STIEF_ERR_INVALID_ARG;
+  return run_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_splits, out, out_lse, status,
+                    static_cast<cudaStream_t>(stream));
+}
+
+size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv) {
+  if (B <= 0 || Hq <= 0 || Hkv <= 0) return 0;
+  // q, k_new, v_new, out -- each section 128-byte aligned
+  return align_up((size_t)B * Hq * kD * 2, 128) * 2 + align_up((size_t)B * Hkv * kD * 2, 128) * 2;
+}
+
+int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
+                           const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging, void* workspace,
+                           size_t workspace_bytes, int32_t num_splits, uint16_t* out_host, int32_t* status, void* stream) {
+  if (!layer || !batch || !q_host || !k_new_host || !v_new_host || !staging || !out_host || !aligned(staging, 128))
+    return STIEF_ERR_INVALID_ARG;
+  if (batch->B <= 0 || layer->Hq <= 0 || layer->Hkv <= 0) return STIEF_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t qb = (size_t)batch->B * layer->Hq * kD * 2, kb = (size_t)batch->B * layer->Hkv * kD * 2;
+  uint8_t* p = static_cast<uint8_t*>(staging);
+  uint16_t* dq = reinterpret_cast<uint16_t*>(p);
+  uint16_t* dk = reinterpret_cast<uint16_t*>(p + align_up(qb, 128));
+  uint16_t* dv = reinterpret_cast<uint16_t*>(p + align_up(qb, 128) + align_up(kb, 128));
+  uint16_t* dout = reinterpret_cast<uint16_t*>(p + align_up(qb, 128) + 2 * align_up(kb, 128));
+  if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  const int rc = stief_decode_step(layer, batch, dq, dk, dv, workspace, workspace_bytes, num_splits, dout, nullptr, status, stream);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  return STIEF_OK;
+}
+
+int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream) {
+  if (!seq_lens || B <= 0) return STIEF_ERR_INVALID_ARG;
+  return launch_advance(seq_lens, B, delta, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+const char* stief_status_string(int status) {
+  switch (status) {
+    case STIEF_OK: return "ok";
+    case STIEF_ERR_INVALID_ARG: return "invalid argument";
+    case STIEF_ERR_UNSUPPORTED: return "unsupported rank or head dimension";
+    case STIEF_ERR_WORKSPACE: return "workspace too small";
+    case STIEF_ERR_CUDA: return "CUDA call failed";
+    case STIEF_ERR_BOUNDS: return "page id or position out of range (device)";
+    case STIEF_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int stief_version(void) { return 100; }
+
+}  // extern "C"

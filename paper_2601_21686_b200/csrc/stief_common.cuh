@@ -1,0 +1,181 @@
+// Shared device-side helpers for the sm_100a kernels: PTX wrappers (mbarrier, TMA, ldmatrix, mma),
+// bf16 packing, the status word, and launch descriptors passed from the host API to the kernels.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "stief.h"
+
+namespace stief {
+
+constexpr int kPage = STIEF_PAGE;       // tokens per cache page
+constexpr int kD = STIEF_D_HEAD;        // head dimension
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ---------------------------------------------------------------------------------------------
+// status word: first error wins
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void report(int32_t* status, int code) {
+  if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+// ---------------------------------------------------------------------------------------------
+// shared-memory addresses, mbarriers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  `abort_flag` (shared memory) short-circuits every later wait of the CTA once one
+// wait has run out, so a lost copy can never hang the kernel: results are then garbage, the status
+// word says STIEF_ERR_TIMEOUT, and control flow continues to the normal exit.
+constexpr uint32_t kWaitSpins = 1u << 24;
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  for (uint32_t i = 0; i < kWaitSpins; ++i) {
+    if (mbar_try_wait(bar, parity)) return;
+    if ((i & 1023u) == 1023u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  report(status, STIEF_ERR_TIMEOUT);
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// TMA (tensor maps live in kernel parameter space as __grid_constant__)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+}
+// 2-D tiled load global -> shared, completion counted in bytes on an mbarrier.  x is the inner
+// (element) coordinate: x * element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// warp-level matrix ops
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D += A(16x16, row) * B(16x8, col), bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {   // 2^x, ex2.approx: exp2(-inf) = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------------------------------------
+// bf16 helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {   // lo -> bits [0,16)
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): two bf16 words carrying ~16 significant bits
+__device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16(x0, x1);
+  lo = pack_bf16(x0 - bf16_lo(hi), x1 - bf16_hi(hi));
+}
+
+// ---------------------------------------------------------------------------------------------
+// swizzled page tiles in shared memory
+// ---------------------------------------------------------------------------------------------
+// A page tile holds 64 cache rows of R bf16.  It is fetched as R/BW boxes of 64 rows x BW elements,
+// BW the largest of 64/32/16 dividing R, each box stored with the TMA swizzle whose span equals the
+// box row (128/64/32 bytes), so that the eight 16-byte row pieces of an 8x8 ldmatrix tile fall in
+// distinct banks.
+template <int R>
+struct Tile {
+  static constexpr int BW = (R % 64 == 0) ? 64 : (R % 32 == 0) ? 32 : 16;   // box width, elements
+  static constexpr int NB = R / BW;                                         // boxes per tile
+  static constexpr int RB = BW * 2;                                         // box row bytes
+  static constexpr int CPB = BW / 8;                                        // 16-byte chunks per box row
+  static constexpr int BOX_BYTES = kPage * RB;
+  static constexpr int BYTES = kPage * R * 2;
+  // byte offset inside the tile of 16-byte chunk c (0 .. R/8-1) of row t
+  __device__ static __forceinline__ uint32_t chunk(int t, int c) {
+    const int sub = c / CPB, cc = c % CPB;
+    uint32_t off = static_cast<uint32_t>(t * RB + cc * 16);
+    off ^= ((off >> 7) & (CPB - 1)) << 4;
+    return static_cast<uint32_t>(sub * BOX_BYTES) + off;
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// plain-old-data launch descriptors (host API -> kernels)
+// ---------------------------------------------------------------------------------------------
+struct LayerDev {
+  int Hq, Hkv, G, r_k, r_v, num_pages;
+  const __nv_bfloat16* U_k;
+  long long uk_stride;
+  const __nv_bfloat16* U_v;
+  long long uv_stride;
+  __nv_bfloat16* k_pool;
+  __nv_bfloat16* v_pool;
+};
+struct BatchDev {
+  int B, max_pages;
+  const int* block_table;
+  const int* seq_lens;
+};
+
+}  // namespace stief

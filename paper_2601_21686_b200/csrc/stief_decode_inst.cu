@@ -1,0 +1,54 @@
+// Instantiations of the split-T decode kernel for one key rank (STIEF_RK, given on the command line)
+// and every supported value rank.  Compiled once per key rank so the build parallelises.
+#include "stief_decode.cuh"
+#include "stief_kernels.h"
+
+#ifndef STIEF_RK
+#error "compile with -DSTIEF_RK=<key rank>"
+#endif
+
+namespace stief {
+
+template <int RK, int RV>
+static cudaError_t launch_one(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st) {
+  using C = DecodeCfg<RK, RV>;
+  auto kern = decode_split_kernel<RK, RV>;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  DecodeArgs k;
+  k.L = a.L;
+  k.Bt = a.Bt;
+  k.q_proj = a.q_proj;
+  k.partial_o = a.partial_o;
+  k.partial_lse = a.partial_lse;
+  k.S = a.S;
+  k.chunk_pages = a.chunk_pages;
+  k.len_add = a.len_add;
+  k.status = a.status;
+  dim3 grid(a.S, a.L.Hkv * ((a.L.G + 7) / 8), a.Bt.B);
+  kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tmK, tmV, k);
+  return cudaGetLastError();
+}
+
+#define STIEF_CAT_(a, b) a##b
+#define STIEF_CAT(a, b) STIEF_CAT_(a, b)
+
+cudaError_t STIEF_CAT(launch_decode_rk, STIEF_RK)(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                                                  cudaStream_t st) {
+  switch (a.L.r_v) {
+    case 32: return launch_one<STIEF_RK, 32>(a, tmK, tmV, st);
+    case 48: return launch_one<STIEF_RK, 48>(a, tmK, tmV, st);
+    case 64: return launch_one<STIEF_RK, 64>(a, tmK, tmV, st);
+    case 96: return launch_one<STIEF_RK, 96>(a, tmK, tmV, st);
+    case 128: return launch_one<STIEF_RK, 128>(a, tmK, tmV, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace stief

@@ -1,0 +1,293 @@
+"""GPU parity: the CUDA path (through the C-ABI library) against the fp64 CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: cache layout/indexing bit-exact; cache values within 1 bf16 ulp of
+the oracle's rounded projection (or a correct rounding inside the fp32 accumulation bound); attention outputs
+max-abs <= 1e-2 and relative-L2 <= 5e-3."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2601_21686_b200 as S
+from oracle import stief_oracle as O
+from paper_2601_21686_b200 import inputs as I
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+
+RANKS = (32, 48, 64, 96, 128)
+
+
+def _sync_status(c):
+    torch.cuda.synchronize()
+    return int(c.status.item())
+
+
+def _prefill_and_check(c: U.Case):
+    S.stief_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    assert _sync_status(c) == 0
+    Kd, Vd = U.oracle_cache(c)
+    Kf, Vf = U.f64(c.K), U.f64(c.V)
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    second = 0
+    for b in range(c.B):
+        n = int(c.seq_lens[b])
+        if n == 0:
+            continue
+        gk = U.gpu_cache_rows(c, c.layer.k_pool, b, n)
+        gv = U.gpu_cache_rows(c, c.layer.v_pool, b, n)
+        for h in range(c.Hkv):
+            s1, _ = U.check_cache(gk[:, h], Kf[b, :n, h], O.basis_of(Uk, h), Kd[b][:, h])
+            s2, _ = U.check_cache(gv[:, h], Vf[b, :n, h], O.basis_of(Uv, h), Vd[b][:, h])
+            second += s1 + s2
+    total = sum(int(n) for n in c.seq_lens) * c.Hkv * (c.r_k + c.r_v)
+    assert second <= max(2, 1e-3 * total), f"{second} of {total} cache elements needed the accumulation-bound clause"
+    return Kd, Vd
+
+
+def _untouched_rows_still_nan(c: U.Case):
+    """Layout check from the other side: everything the prefill was not asked to write still holds the NaN fill."""
+    used = np.zeros((c.paging.num_pages, 64), dtype=bool)
+    for b in range(c.B):
+        for t in range(int(c.seq_lens[b])):
+            used[c.paging.block_table[b, t // 64], t % 64] = True
+    for pool in (c.layer.k_pool, c.layer.v_pool):
+        pb = U.bits(pool.cpu())                                   # [pages, Hkv, 64, r]
+        untouched = pb[~used[:, None, :].repeat(c.Hkv, 1)]
+        assert np.all(untouched == U.NAN_BITS)
+        assert not np.any(pb[used[:, None, :].repeat(c.Hkv, 1)] == U.NAN_BITS)
+
+
+def _decode(c: U.Case, num_splits, len_add=0, q=None):
+    ws = U.workspace_for(c, num_splits if num_splits else S.stief_decode_num_splits(c.B, c.Hkv, c.batch.block_table.shape[1]))
+    out = torch.full((c.B, c.Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((c.B, c.Hq), float("nan"), dtype=torch.float32, device="cuda")
+    S.stief_decode_attention(c.layer, c.batch, (c.q if q is None else q).cuda(), ws, num_splits, out, lse, len_add=len_add,
+                             status=c.status)
+    assert _sync_status(c) == 0
+    return out, lse
+
+
+def test_config1_prefill_then_decode():
+    # B=1, Hq=4, Hkv=1, T=512, r=64/64, seed 0
+    c = U.make_case(0, 1, 4, 1, 64, 64, [512])
+    Kd, Vd = _prefill_and_check(c)
+    _untouched_rows_still_nan(c)
+    ref, ref_lse = U.oracle_decode(c, Kd, Vd)
+    for ns in (1, 2, 8, 0):
+        out, lse = _decode(c, ns)
+        U.check_out(out, ref)
+        assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 2e-3
+
+
+@pytest.mark.parametrize("r_k", RANKS)
+@pytest.mark.parametrize("r_v", RANKS)
+def test_every_rank_pair_ragged(r_k, r_v):
+    c = U.make_case(100 + r_k + 7 * r_v, 3, 8, 2, r_k, r_v, [200, 64, 129])
+    Kd, Vd = _prefill_and_check(c)
+    ref, ref_lse = U.oracle_decode(c, Kd, Vd)
+    for ns in (1, 3):
+        out, lse = _decode(c, ns)
+        U.check_out(out, ref)
+        assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 2e-3
+
+
+def test_decode_on_the_oracles_own_cache_is_tight():
+    # same cache bits on both sides: what is left is fp32 accumulation, the two-word bf16 operands and the
+    # bf16 rounding of the output (2^-9 relative per element)
+    c = U.make_case(5, 2, 8, 2, 64, 96, [700, 333], lowrank=True)
+    Kd, Vd = U.oracle_cache(c)
+    U.upload_cache(c, Kd, Vd)
+    ref, ref_lse = U.oracle_decode(c, Kd, Vd)
+    for ns in (1, 4, 11):
+        out, lse = _decode(c, ns)
+        ea, rl = U.check_out(out, ref, max_abs=4e-3, rel_l2=2.5e-3)
+        assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 2e-4
+
+
+def test_sharp_softmax_large_scores():
+    # queries 8x larger: scores of magnitude ~10, one or two tokens dominate
+    c = U.make_case(6, 1, 4, 1, 64, 64, [1000], lowrank=True, q_scale=8.0)
+    Kd, Vd = _prefill_and_check(c)
+    ref, ref_lse = U.oracle_decode(c, Kd, Vd)
+    out, lse = _decode(c, 5)
+    U.check_out(out, ref)
+    assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 5e-3
+
+
+@pytest.mark.parametrize("lens", [[1], [63], [64], [65], [0, 5], [128, 0, 1, 640]])
+def test_edge_lengths(lens):
+    c = U.make_case(7 + len(lens) + lens[0], len(lens), 4, 1, 48, 64, lens)
+    Kd, Vd = _prefill_and_check(c)
+    _untouched_rows_still_nan(c)
+    ref, ref_lse = U.oracle_decode(c, Kd, Vd)
+    out, lse = _decode(c, 2)
+    U.check_out(out, ref)
+    g = lse.cpu().numpy()
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert np.all(out[b].float().cpu().numpy() == 0) and np.all(np.isneginf(g[b]))
+        else:
+            assert np.abs(g[b] - ref_lse[b]).max() < 2e-3
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (6, 2), (16, 2), (32, 2), (8, 1)])
+def test_group_sizes(Hq, Hkv):
+    # G = 1 (MHA), 3, 8, 16 (two query tiles), 8 with a single KV head
+    c = U.make_case(20 + Hq, 2, Hq, Hkv, 64, 32, [150, 90])
+    Kd, Vd = _prefill_and_check(c)
+    ref, _ = U.oracle_decode(c, Kd, Vd)
+    out, _ = _decode(c, 2)
+    U.check_out(out, ref)
+
+
+def test_shared_key_basis_and_full_rank_sides():
+    # one key basis per layer shared by all heads (head stride 0)
+    c = U.make_case(30, 2, 8, 2, 64, 64, [100, 260], shared_key_basis=True)
+    Kd, Vd = _prefill_and_check(c)
+    ref, _ = U.oracle_decode(c, Kd, Vd)
+    U.check_out(_decode(c, 3)[0], ref)
+    # keys kept full rank (no basis), values compressed; then the reverse; then nothing compressed
+    for fk, fv, rk, rv in ((True, False, 128, 48), (False, True, 96, 128), (True, True, 128, 128)):
+        c = U.make_case(31, 2, 8, 2, rk, rv, [100, 260], full_rank_k=fk, full_rank_v=fv)
+        Kd, Vd = _prefill_and_check(c)
+        if fk:   # rows stored unprojected must be bit-identical to the input rows
+            assert np.array_equal(U.bits(U.gpu_cache_rows(c, c.layer.k_pool, 1, 260)), U.bits(c.K[1, :260]))
+        ref, _ = U.oracle_decode(c, Kd, Vd)
+        U.check_out(_decode(c, 2)[0], ref)
+
+
+def test_rank_128_with_orthogonal_basis_is_exact_attention():
+    # r = d_h: compressed attention equals plain softmax attention on K, V (up to the bf16 cache rounding)
+    c = U.make_case(32, 1, 4, 1, 128, 128, [300])
+    _prefill_and_check(c)
+    out, _ = _decode(c, 2)
+    q, K, V = U.f64(c.q), U.f64(c.K), U.f64(c.V)
+    ref, _ = O.decode_layer(q, [K[0, :300]], [V[0, :300]], None, None, "a")
+    # U is orthogonal only to bf16 precision (|U^T U - I| ~ 1e-3), so this is looser than oracle parity
+    U.check_out(out, ref, max_abs=3e-2, rel_l2=2e-2)
+
+
+def test_append_and_decode_step_across_a_page_boundary():
+    B, Hq, Hkv = 2, 8, 2
+    c = U.make_case(40, B, Hq, Hkv, 48, 96, [62, 127], reserve=8)
+    Kd, Vd = _prefill_and_check(c)
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    lens = c.seq_lens.copy()
+    ws = U.workspace_for(c, 4)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    for step in range(5):
+        k_new, v_new = I.new_token_kv(40, 0, B, Hkv, step=step)
+        q = I.queries(40, 0, B, Hq, step=step + 1)
+        if step % 2 == 0:      # fused step
+            S.stief_decode_step(c.layer, c.batch, q.cuda(), k_new.cuda(), v_new.cuda(), ws, out, num_splits=4, status=c.status)
+        else:                  # the same thing as separate calls
+            S.stief_append(c.layer, c.batch, k_new.cuda(), v_new.cuda(), status=c.status)
+            S.stief_decode_attention(c.layer, c.batch, q.cuda(), ws, 4, out, len_add=1, status=c.status)
+        S.stief_advance_seq_lens(c.batch.seq_lens, 1)
+        assert _sync_status(c) == 0
+        kn, vn = U.f64(k_new), U.f64(v_new)
+        for b in range(B):
+            Kd[b] = np.concatenate([Kd[b], np.stack([O.compress(kn[b, h][None], O.basis_of(Uk, h))[0] for h in range(Hkv)])[None]], 0)
+            Vd[b] = np.concatenate([Vd[b], np.stack([O.compress(vn[b, h][None], O.basis_of(Uv, h))[0] for h in range(Hkv)])[None]], 0)
+        lens += 1
+        assert np.array_equal(c.batch.seq_lens.cpu().numpy(), lens)
+        # appended rows: 1 ulp; position: the row must be where the address formula says
+        for b in range(B):
+            n = int(lens[b])
+            gk = U.gpu_cache_rows(c, c.layer.k_pool, b, n)
+            gv = U.gpu_cache_rows(c, c.layer.v_pool, b, n)
+            for h in range(Hkv):
+                U.check_cache(gk[n - 1:, h], kn[b, h][None], O.basis_of(Uk, h), Kd[b][n - 1:, h])
+                U.check_cache(gv[n - 1:, h], vn[b, h][None], O.basis_of(Uv, h), Vd[b][n - 1:, h])
+        ref, _ = O.decode_layer(U.f64(q), Kd, Vd, Uk, Uv, "b")
+        U.check_out(out, ref)
+
+
+def test_split_count_invariance_and_span():
+    c = U.make_case(50, 1, 8, 2, 64, 48, [2000])
+    _prefill_and_check(c)
+    outs = [_decode(c, ns)[0].float().cpu().numpy() for ns in (1, 2, 7, 32)]
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() < 4e-3
+    # output lies in span(U_v) up to the bf16 rounding of out and of U_v
+    Uv = U.f64(c.U_v)
+    o = outs[0][0].astype(np.float64)
+    for g in range(8):
+        P = Uv[g // 4] @ Uv[g // 4].T
+        assert np.linalg.norm(o[g] - o[g] @ P) <= 1e-2 * np.linalg.norm(o[g])
+
+
+def test_separate_combine_call_matches_fused_call():
+    c = U.make_case(51, 2, 8, 2, 64, 64, [500, 131])
+    _prefill_and_check(c)
+    ws = U.workspace_for(c, 6)
+    out1 = torch.empty(2, 8, 128, dtype=torch.bfloat16, device="cuda")
+    out2 = torch.empty_like(out1)
+    S.stief_decode_attention(c.layer, c.batch, c.q.cuda(), ws, 6, out1, status=c.status)
+    S.stief_decode_attention(c.layer, c.batch, c.q.cuda(), ws, 6, None, status=c.status)
+    S.stief_split_combine(c.layer, c.batch, ws, 6, out2)
+    assert _sync_status(c) == 0
+    assert torch.equal(out1, out2)
+
+
+def test_host_staged_step():
+    B, Hq, Hkv = 2, 8, 2
+    c = U.make_case(60, B, Hq, Hkv, 64, 64, [100, 70], reserve=4)
+    Kd, Vd = _prefill_and_check(c)
+    k_new, v_new = I.new_token_kv(60, 0, B, Hkv)
+    q = c.q.pin_memory()
+    kh, vh = k_new.pin_memory(), v_new.pin_memory()
+    out_h = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(S.stief_host_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device="cuda")
+    ws = U.workspace_for(c, 2)
+    S.stief_decode_step_host(c.layer, c.batch, q, kh, vh, staging, ws, out_h, num_splits=2, status=c.status)
+    assert _sync_status(c) == 0
+    out_d = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    S.stief_decode_step(c.layer, c.batch, c.q.cuda(), k_new.cuda(), v_new.cuda(), ws, out_d, num_splits=2, status=c.status)
+    assert _sync_status(c) == 0
+    assert torch.equal(out_h, out_d.cpu())
+
+
+def test_errors_are_reported_not_trapped():
+    c = U.make_case(70, 1, 4, 1, 64, 64, [100])
+    ws = U.workspace_for(c, 2)
+    out = torch.empty(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    # host-visible problems come back as return codes
+    bad = S.Layer(4, 1, 40, 64, c.layer.U_k, c.layer.U_v, c.layer.k_pool, c.layer.v_pool)
+    with pytest.raises(S.StiefError) as e:
+        S.stief_decode_attention(bad, c.batch, c.q.cuda(), ws, 2, out)
+    assert e.value.code == S.STIEF_ERR_UNSUPPORTED
+    with pytest.raises(S.StiefError) as e:
+        S.stief_decode_attention(c.layer, c.batch, c.q.cuda(), ws[:64], 2, out)
+    assert e.value.code == S.STIEF_ERR_WORKSPACE
+    with pytest.raises(S.StiefError) as e:
+        S.stief_decode_attention(c.layer, c.batch, c.q.cuda().view(-1)[1:513], ws, 2, out)      # misaligned q
+    assert e.value.code == S.STIEF_ERR_INVALID_ARG
+    bad = S.Layer(5, 2, 64, 64, c.layer.U_k, c.layer.U_v, c.layer.k_pool, c.layer.v_pool)       # Hq % Hkv != 0
+    with pytest.raises(S.StiefError) as e:
+        S.stief_decode_attention(bad, c.batch, c.q.cuda(), ws, 2, out)
+    assert e.value.code == S.STIEF_ERR_INVALID_ARG
+    # a page id outside the pool: the kernels redirect the access, finish, and flag the status word
+    S.stief_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    bt = c.batch.block_table.clone()
+    bt[0, 1] = c.paging.num_pages + 5
+    badb = S.Batch(bt, c.batch.seq_lens)
+    S.stief_decode_attention(c.layer, badb, c.q.cuda(), ws, 2, out, status=c.status)
+    assert _sync_status(c) == S.STIEF_ERR_BOUNDS
+    c.status.zero_()
+    S.stief_prefill_compress(c.layer, badb, c.K.cuda(), c.V.cuda(), status=c.status)
+    assert _sync_status(c) == S.STIEF_ERR_BOUNDS
+    c.status.zero_()
+    # a sequence longer than its block table
+    long = S.Batch(c.batch.block_table, torch.tensor([64 * c.batch.block_table.shape[1] + 3], dtype=torch.int32, device="cuda"))
+    S.stief_decode_attention(c.layer, long, c.q.cuda(), ws, 2, out, status=c.status)
+    assert _sync_status(c) == S.STIEF_ERR_BOUNDS
+    c.status.zero_()
+    k_new, v_new = I.new_token_kv(70, 0, 1, 1)
+    S.stief_append(c.layer, long, k_new.cuda(), v_new.cuda(), status=c.status)
+    assert _sync_status(c) == S.STIEF_ERR_BOUNDS
+    # and the context is still healthy
+    c.status.zero_()
+    S.stief_decode_attention(c.layer, c.batch, c.q.cuda(), ws, 2, out, status=c.status)
+    assert _sync_status(c) == 0
