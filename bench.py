@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the compressed-cache decode hot path on B200.
+
+Workload (N = 1): Llama3-8B-shaped single-layer decode, B=4 sequences, 32 query heads, 8 KV heads,
+d_h=128, T=32768 tokens of context per sequence, r_k=r_v=64, bf16 compressed cache in 64-token pages
+handed out from a shuffled pool.  Keys are a rank-48 Gaussian signal plus 0.1 N(0,1) noise, values and
+queries Gaussian, bases from seeded QR -- all synthetic.
+
+A step = one decode step of one layer: project and append the new token's k, v into the cache, project the
+queries, split-T attention over the T+1 cached tokens in the compressed space, merge the chunks and
+back-project (every kernel of the path).  The cache itself is built once, before timing, by the library's
+own prefill-compression kernel, which is timed separately and reported under "prefill".  Steps rotate over
+several independent layer caches, each larger than L2, so no step finds its cache in L2.
+
+metric  = effective HBM bandwidth over the compressed cache bytes a step must read
+          (B * Hkv * (T+1) * 2 * (r_k + r_v) bytes per step); tokens/s is reported next to it.
+Prints one JSON line (see the design doc for every key).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+SEED = 0
+CFG2 = dict(B=4, Hq=32, Hkv=8, T=32768, r_k=64, r_v=64)
+N_CACHES = 4               # rotating layer caches (each 256 MiB of compressed rows)
+METRIC = "decode_attn_effective_hbm_gbs"
+UNIT = "GB/s"
+
+
+def step_bytes(cfg) -> int:
+    return cfg["B"] * cfg["Hkv"] * (cfg["T"] + 1) * 2 * (cfg["r_k"] + cfg["r_v"])
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), float(d.get("bf16_tflops", 1590.0)), "measured"
+        except Exception:
+            pass
+    return 6650.0, 1590.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.rows:
+            if ts < t0 - 0.05 or ts > t1 + 0.15:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+def build_caches(cfg, n_caches, dev, S, I):
+    """n_caches independent layer caches, filled by the library's prefill kernel from seeded K, V."""
+    B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
+    pg = I.make_paging(SEED, [T] * B, reserve_tokens=1)
+    bt = torch.from_numpy(pg.block_table).to(dev)
+    lens = torch.from_numpy(pg.seq_lens).to(dev)
+    batch = S.Batch(bt, lens)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    layers, prefill_ms = [], []
+    for l in range(n_caches):
+        U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
+        layer = S.Layer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev),
+                        torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.bfloat16, device=dev),
+                        torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.bfloat16, device=dev))
+        K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
+        V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        S.stief_prefill_compress(layer, batch, K, V, status=status)      # warm-up (also the real fill)
+        torch.cuda.synchronize()
+        e0.record()
+        S.stief_prefill_compress(layer, batch, K, V, status=status)
+        e1.record()
+        torch.cuda.synchronize()
+        prefill_ms.append(e0.elapsed_time(e1))
+        layers.append(layer)
+        del K, V
+    assert int(status.item()) == 0, f"device status {int(status.item())} while building the cache"
+    return layers, batch, status, prefill_ms
+
+
+def run_ours(args):
+    import paper_2601_21686_b200 as S
+    from paper_2601_21686_b200 import inputs as I
+    from paper_2601_21686_b200 import build as Bld
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        Bld.build()
+    if world > 1:
+        dist.barrier()
+    S.lib()
+
+    cfg = dict(CFG2)
+    B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
+    layers, batch, status, prefill_ms = build_caches(cfg, N_CACHES, dev, S, I)
+    ns = args.num_splits or S.stief_decode_num_splits(B, Hkv, batch.block_table.shape[1])
+    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, r_k, r_v, ns) // 4, dtype=torch.float32, device=dev)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    n_in = 8
+    qs = [I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for i in range(n_in)]
+    kvs = [I.new_token_kv(SEED, 0, B, Hkv, device=dev, step=i) for i in range(n_in)]
+
+    def step(i):
+        S.stief_decode_step(layers[i % N_CACHES], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
+                            num_splits=ns, status=status)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K_steps, W = args.steps, max(args.warmup, 3)
+    for i in range(W):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- timed region 1: device-resident inputs
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.time()
+    e0.record()
+    for i in range(K_steps):
+        step(W + i)
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1)
+
+    # ---- timed region 2: the split-T kernel alone, per launch (events recorded inside the library call)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
+    for a, b in evs:
+        a.record(); b.record()
+    barrier()
+    for i in range(K_steps):
+        S.stief_time_next_decode_kernel(*evs[i])
+        step(W + i)
+    barrier()
+    kern_ms = [a.elapsed_time(b) for a, b in evs]
+
+    # ---- timed region 3: end to end through the host-buffer entry point
+    staging = torch.empty(S.stief_host_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
+    qh = [q.cpu().pin_memory() for q in qs]
+    kh = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kvs]
+    out_h = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
+
+    def step_host(i):
+        S.stief_decode_step_host(layers[i % N_CACHES], batch, qh[i % n_in], kh[i % n_in][0], kh[i % n_in][1], staging, ws,
+                                 out_h, num_splits=ns, status=status)
+        torch.cuda.current_stream().synchronize()       # the caller reads out_h after every step
+
+    for i in range(W):
+        step_host(i)
+    barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for i in range(K_steps):
+        step_host(W + i)
+    h1.record()
+    barrier()
+    ms_host = h0.elapsed_time(h1)
+    if rank == 0:
+        sampler.stop()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    # ---- max over ranks
+    times = torch.tensor([ms, ms_host, float(np.mean(kern_ms))], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, ms_host, kern_avg_ms = (float(x) for x in times.tolist())
+
+    if rank == 0:
+        hbm_peak, tf_peak, peak_kind = measured_peaks()
+        sb = step_bytes(cfg)
+        value = world * sb * K_steps / (ms * 1e-3) / 1e9
+        e2e = world * sb * K_steps / (ms_host * 1e-3) / 1e9
+        achieved = sb / (kern_avg_ms * 1e-3) / 1e9
+        pf_ms = float(np.median(prefill_ms))
+        pf_bytes = B * T * Hkv * (2 * 128 * 2 + 2 * (r_k + r_v))
+        pf_flops = 2.0 * B * T * Hkv * 128 * (r_k + r_v)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
+            "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 cache, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": "config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64, "
+                                   "64-token pages, shuffled block tables; step = append + query projection + split-T attention + combine",
+                       "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_splits": ns,
+                       "l2": f"steps rotate over {N_CACHES} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
+                       "parallelism": f"replicas x{world} (independent batches, no collective)"},
+            "tokens_per_s": world * B * K_steps / (ms * 1e-3),
+            "frac_of_hbm_peak": value / world / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
+            "frac_of_hbm_spec_8000": value / world / 8000.0,
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
+                    "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
+                    "tokens_per_s": world * B * K_steps / (ms_host * 1e-3)},
+            "gpu_launches": 3 * K_steps,
+            "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<64,64>", "achieved": achieved, "peak": hbm_peak,
+                         "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": peak_kind, "traffic": args.traffic,
+                         "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms, "min_launch_ms": float(min(kern_ms))},
+            "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak,
+                        "tflops": pf_flops / (pf_ms * 1e-3) / 1e12, "frac_of_bf16_peak": pf_flops / (pf_ms * 1e-3) / 1e12 / tf_peak,
+                        "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache, one layer"},
+            "clocks": sampler.summary(t0, t1),
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=20.0)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle, timed on the host cores (a reported baseline, and the `--impl reference` arm)
+# ------------------------------------------------------------------------------------------------
+def _oracle_sample(cfg, n_seq):
+    """Inputs and oracle cache for the first n_seq sequences of the workload (CPU, fp64)."""
+    from oracle import stief_oracle as O
+    from paper_2601_21686_b200 import inputs as I
+    Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("Hq", "Hkv", "T", "r_k", "r_v"))
+    K = I.lowrank_keys(SEED, 0, n_seq, T, Hkv).double().numpy()
+    V = I.gaussian_kv(SEED, I.TAG_V, 0, n_seq, T, Hkv).double().numpy()
+    U_k, U_v = I.stiefel_bases(SEED, 0, Hkv, r_k, r_v)
+    U_k, U_v = U_k.double().numpy(), U_v.double().numpy()
+    Kd, Vd = O.compress_layer(K, V, U_k, U_v, [T] * n_seq)
+    return O, I, Kd, Vd, U_k, U_v
+
+
+def _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, i):
+    """One decode step of the oracle on the sample: append the new token's projected rows, then attend."""
+    Hq, Hkv = cfg["Hq"], cfg["Hkv"]
+    q = I.queries(SEED, 0, n_seq, Hq, scale=1.0 / np.sqrt(128.0), step=i).double().numpy()
+    k_new, v_new = I.new_token_kv(SEED, 0, n_seq, Hkv, step=i)
+    k_new, v_new = k_new.double().numpy(), v_new.double().numpy()
+    t0 = time.perf_counter()
+    Kd2, Vd2 = [], []
+    for b in range(n_seq):
+        kr = np.stack([O.compress(k_new[b, h][None], O.basis_of(U_k, h))[0] for h in range(Hkv)])[None]
+        vr = np.stack([O.compress(v_new[b, h][None], O.basis_of(U_v, h))[0] for h in range(Hkv)])[None]
+        Kd2.append(np.concatenate([Kd[b], kr], 0))
+        Vd2.append(np.concatenate([Vd[b], vr], 0))
+    out, _ = O.decode_layer(q, Kd2, Vd2, U_k, U_v, "b")
+    return time.perf_counter() - t0, out
+
+
+def _threads_used() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else 1
+    except Exception:
+        return 1
+
+
+def cpu_baseline(cfg, seconds_budget=20.0):
+    n_seq = 1
+    O, I, Kd, Vd, U_k, U_v = _oracle_sample(cfg, n_seq)
+    sb = step_bytes(cfg) * n_seq // cfg["B"]
+    dts = []
+    t_start = time.perf_counter()
+    i = 0
+    while i < 3 or (time.perf_counter() - t_start < seconds_budget and i < 20):
+        dt, _ = _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, i)
+        dts.append(dt)
+        i += 1
+    best = min(dts)
+    return {"value": sb / best / 1e9, "unit": UNIT, "cores": _threads_used(), "host_cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{n_seq} of {cfg['B']} sequences of the same workload (all {cfg['Hq']} query heads, T={cfg['T']}), "
+                      f"{len(dts)} decode steps (append + attention, fp64 numpy), best step",
+            "s_per_step_sample": best, "tokens_per_s": n_seq / best}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = dict(CFG2)
+    n_seq = 1
+    O, I, Kd, Vd, U_k, U_v = _oracle_sample(cfg, n_seq)
+    sb = step_bytes(cfg) * n_seq // cfg["B"]
+    W, K_steps = max(args.warmup, 1), args.steps
+    for i in range(W):
+        _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, i)
+    total = 0.0
+    for i in range(K_steps):
+        dt, _ = _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, W + i)
+        total += dt
+    value = sb * K_steps / total / 1e9
+    sample = (f"each step = one decode step (append + attention, fp64 numpy) on {n_seq} of {cfg['B']} sequences of the workload "
+              f"(all {cfg['Hq']} query heads, T={cfg['T']})")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": K_steps, "warmup": W, "ms_per_step": total / K_steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64 (bounded sample)",
+                       "sample": sample},
+            "tokens_per_s": n_seq * K_steps / total,
+            "cpu_baseline": {"value": value, "unit": UNIT, "kind": "oracle", "cores": _threads_used(), "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -146,6 +146,13 @@ int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, c
 /* seq_lens[b] += delta on the device (so a captured step can be replayed). */
 int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream);
 
+/* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
+ * stief_decode_step_host call made by this host thread records `start_event` just before and
+ * `stop_event` just after its split-T kernel on the call's stream (both cudaEvent_t passed as void*),
+ * so the kernel can be timed alone inside a longer step.  One-shot: cleared by that call.  Passing NULLs
+ * cancels a pending request. */
+int stief_time_next_decode_kernel(void* start_event, void* stop_event);
+
 const char* stief_status_string(int status);
 int stief_version(void);
 

@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
             "stief_host_staging_bytes": (SZ, [I32, I32, I32]),
             "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, P, P]),
             "stief_advance_seq_lens": (ctypes.c_int, [P, I32, I32, P]),
+            "stief_time_next_decode_kernel": (ctypes.c_int, [P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -197,3 +198,14 @@ def stief_decode_step_host(layer: Layer, batch: Batch, q_host: torch.Tensor, k_n
 
 def stief_advance_seq_lens(seq_lens: torch.Tensor, delta: int = 1):
     _check(lib().stief_advance_seq_lens(_ptr(seq_lens), seq_lens.numel(), delta, _stream()), "stief_advance_seq_lens")
+
+
+def stief_time_next_decode_kernel(start_event: Optional[torch.cuda.Event], stop_event: Optional[torch.cuda.Event]):
+    """Have the next decode call of this thread record the two (timing-enabled) events around its split-T kernel."""
+    if start_event is None:
+        _check(lib().stief_time_next_decode_kernel(None, None), "stief_time_next_decode_kernel")
+        return
+    for ev in (start_event, stop_event):
+        if not ev.cuda_event:                 # torch creates the handle lazily, on first record
+            ev.record()
+    _check(lib().stief_time_next_decode_kernel(start_event.cuda_event, stop_event.cuda_event), "stief_time_next_decode_kernel")

@@ -144,6 +144,8 @@ bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
   return rc == CUDA_SUCCESS;
 }
 
+thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+
 int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
                const uint16_t* v_new, int len_add, void* workspace, size_t workspace_bytes, int num_splits, uint16_t* out,
                float* out_lse, int32_t* status, cudaStream_t st) {
@@ -182,7 +184,11 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   DecodeLaunch da;
   da.L = L; da.Bt = Bt; da.q_proj = w.q_proj; da.partial_o = w.partial_o; da.partial_lse = w.partial_lse;
   da.S = S; da.chunk_pages = chunk_pages; da.len_add = len_add; da.status = status;
+  cudaEvent_t ev0 = g_ev_start, ev1 = g_ev_stop;
+  g_ev_start = g_ev_stop = nullptr;
+  if (ev0) cudaEventRecord(ev0, st);
   if (launch_decode(da, tmK, tmV, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  if (ev1) cudaEventRecord(ev1, st);
 
   if (out) {
     CombineArgs ca;
@@ -320,6 +326,13 @@ int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, c
 int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream) {
   if (!seq_lens || B <= 0) return STIEF_ERR_INVALID_ARG;
   return launch_advance(seq_lens, B, delta, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+int stief_time_next_decode_kernel(void* start_event, void* stop_event) {
+  if ((start_event == nullptr) != (stop_event == nullptr)) return STIEF_ERR_INVALID_ARG;
+  g_ev_start = static_cast<cudaEvent_t>(start_event);
+  g_ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return STIEF_OK;
 }
 
 const char* stief_status_string(int status) {

@@ -2,10 +2,15 @@
 //
 // Work item = (sequence b, KV head h, chunk of pages).  One producer warp streams the chunk's
 // compressed page tiles K_down[64 x RK], V_down[64 x RV] from HBM into a ring of shared-memory
-// stages with TMA (hardware swizzle, completion on mbarriers); four consumer warps each take every
-// fourth page, compute the scores S = q' K_down^T of the group's query heads against the 64 tokens on
+// stages with TMA (hardware swizzle, completion on mbarriers); NW consumer warps each take every
+// NW-th page, compute the scores S = q' K_down^T of the group's query heads against the 64 tokens on
 // the tensor cores, keep an online softmax in registers, and accumulate P V_down.  Warps merge their
 // running (max, sum, accumulator) at the end and write one chunk-normalised partial [G][RV] + lse.
+//
+// Every consumer warp owns SPW private stages of the ring and walks them in order, so each mbarrier
+// is only ever waited on by one warp, phase after phase: a parity wait can tell two adjacent phases
+// apart but not more, and a shared ring would let a fast warp wait on a phase that is two ahead of
+// what a slot has completed.
 //
 // Precision: q' (already scaled by log2(e)/sqrt(128)) and P are each carried as a pair of bf16 words
 // (value + remainder) occupying rows 0-7 and 8-15 of the 16-row MMA operand, so the products see
@@ -14,6 +19,10 @@
 #pragma once
 
 #include "stief_common.cuh"
+
+#ifndef STIEF_DECODE_NW
+#define STIEF_DECODE_NW 4
+#endif
 
 namespace stief {
 
@@ -31,19 +40,20 @@ template <int RK, int RV>
 struct DecodeCfg {
   using TK = Tile<RK>;
   using TV = Tile<RV>;
-  static constexpr int NW = 4;                          // consumer warps
+  static constexpr int NW = STIEF_DECODE_NW;            // consumer warps
   static constexpr int THREADS = (NW + 1) * 32;         // + 1 producer warp
   static constexpr int STAGE_BYTES = TK::BYTES + TV::BYTES;
-  static constexpr int NS_RAW = 98304 / STAGE_BYTES;
-  static constexpr int NS = NS_RAW < 2 ? 2 : (NS_RAW > 8 ? 8 : NS_RAW);
+  static constexpr int SPW_RAW = (98304 / STAGE_BYTES) / NW;
+  static constexpr int SPW = SPW_RAW < 1 ? 1 : (SPW_RAW > 4 ? 4 : SPW_RAW);   // private stages per consumer warp
+  static constexpr int NS = NW * SPW;
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
-  static constexpr int CTRL_BYTES = 256;                // full[NS], empty[NS], abort flag
+  static constexpr int CTRL_BYTES = 512;                // full[NS], empty[NS], abort flag
   static constexpr int SMEM_BYTES = RING_BYTES + CTRL_BYTES + 1024;   // + slack to align the ring to 1 KiB
   static_assert(RK % 16 == 0 && RV % 16 == 0 && RK <= 128 && RV <= 128, "ranks are multiples of 16 up to 128");
   static_assert(NW * 8 * (RV + 2) * 4 <= RING_BYTES, "merge scratch must fit in the ring");
 };
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(STIEF_DECODE_NW * 32) : "memory"); }
 
 template <int RK, int RV>
 __global__ void __launch_bounds__(DecodeCfg<RK, RV>::THREADS, 2)
@@ -51,7 +61,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   using C = DecodeCfg<RK, RV>;
   using TK = typename C::TK;
   using TV = typename C::TV;
-  constexpr int NW = C::NW, NS = C::NS;
+  constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW;
 
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -77,6 +87,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const uint32_t ctrl = ring + C::RING_BYTES;
   uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_ptr + C::RING_BYTES + 2 * NS * 8);
+  static_assert(2 * NS * 8 + 4 <= C::CTRL_BYTES, "control block too small");
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (NS + s) * 8; };
 
@@ -107,9 +118,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (lane == 0) report(a.status, STIEF_ERR_BOUNDS);
         page = 0;
       }
-      const int slot = i % NS;
+      const int slot = (i % NW) * SPW + (i / NW) % SPW;    // private stage of the page's consumer warp
+      const int use = (i / NW) / SPW;                      // how often that stage has been filled before
       if (lane == 0) {
-        if (i >= NS) mbar_wait(empty_bar(slot), ((i / NS) - 1) & 1, abort_flag, a.status);
+        if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
         const uint32_t st = ring + slot * C::STAGE_BYTES;
         const int y = (page * a.L.Hkv + h) * kPage;
         mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
@@ -154,8 +166,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int last_valid = len - (npages_seq - 1) * kPage;   // tokens in the sequence's last page (1..64)
 
   for (int i = warp; i < npg; i += NW) {
-    const int slot = i % NS;
-    mbar_wait(full_bar(slot), (i / NS) & 1, abort_flag, a.status);
+    const int slot = warp * SPW + (i / NW) % SPW;
+    mbar_wait(full_bar(slot), ((i / NW) / SPW) & 1, abort_flag, a.status);
     const uint32_t kt = ring + slot * C::STAGE_BYTES;
     const uint32_t vt = kt + TK::BYTES;
     const bool tail = (p0 + i == npages_seq - 1) && (last_valid < kPage);
