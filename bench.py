@@ -164,18 +164,20 @@ def run_ours(args):
     S.lib()
 
     cfg = dict(CFG2)
+    n_caches = args.caches
     B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
-    layers, batch, status, prefill_ms = build_caches(cfg, N_CACHES, dev, S, I)
-    ns = args.num_splits or S.stief_decode_num_splits(B, Hkv, batch.block_table.shape[1])
-    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, r_k, r_v, ns) // 4, dtype=torch.float32, device=dev)
+    layers, batch, status, prefill_ms = build_caches(cfg, n_caches, dev, S, I)
+    ns = args.num_parts or S.stief_decode_num_parts()
+    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, Hkv, r_v, ns) // 4, dtype=torch.float32, device=dev)
+    S.stief_decode_workspace_init(ws)
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     n_in = 8
     qs = [I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for i in range(n_in)]
     kvs = [I.new_token_kv(SEED, 0, B, Hkv, device=dev, step=i) for i in range(n_in)]
 
     def step(i):
-        S.stief_decode_step(layers[i % N_CACHES], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
-                            num_splits=ns, status=status)
+        S.stief_decode_step(layers[i % n_caches], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
+                            num_parts=ns, status=status)
 
     def barrier():
         if world > 1:
@@ -221,8 +223,8 @@ def run_ours(args):
     out_h = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
 
     def step_host(i):
-        S.stief_decode_step_host(layers[i % N_CACHES], batch, qh[i % n_in], kh[i % n_in][0], kh[i % n_in][1], staging, ws,
-                                 out_h, num_splits=ns, status=status)
+        S.stief_decode_step_host(layers[i % n_caches], batch, qh[i % n_in], kh[i % n_in][0], kh[i % n_in][1], staging, ws,
+                                 out_h, num_parts=ns, status=status)
         torch.cuda.current_stream().synchronize()       # the caller reads out_h after every step
 
     for i in range(W):
@@ -259,9 +261,9 @@ def run_ours(args):
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 cache, fp32 accumulate", "data": "synthetic",
             "config": {"workload": "config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64, "
-                                   "64-token pages, shuffled block tables; step = append + query projection + split-T attention + combine",
-                       "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_splits": ns,
-                       "l2": f"steps rotate over {N_CACHES} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
+                                   "64-token pages, shuffled block tables; step = append + query projection + split-T attention + combine, one launch",
+                       "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_parts": ns,
+                       "l2": f"steps rotate over {n_caches} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
                        "parallelism": f"replicas x{world} (independent batches, no collective)"},
             "tokens_per_s": world * B * K_steps / (ms * 1e-3),
             "frac_of_hbm_peak": value / world / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
@@ -269,14 +271,14 @@ def run_ours(args):
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
                     "tokens_per_s": world * B * K_steps / (ms_host * 1e-3)},
-            "gpu_launches": 3 * K_steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<64,64>", "achieved": achieved, "peak": hbm_peak,
+            "gpu_launches": K_steps,
+            "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel<64,64>", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": peak_kind, "traffic": args.traffic,
                          "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms, "min_launch_ms": float(min(kern_ms))},
             "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak,
                         "tflops": pf_flops / (pf_ms * 1e-3) / 1e12, "frac_of_bf16_peak": pf_flops / (pf_ms * 1e-3) / 1e12 / tf_peak,
                         "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache, one layer"},
-            "clocks": sampler.summary(t0, t1),
+            "clocks": sampler.summary(t0, time.time()),
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=20.0)
@@ -379,11 +381,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--num-parts", type=int, default=0, help="CTAs of the persistent decode kernel (0 = one per SM)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -95,42 +95,50 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
 int stief_append(const stief_layer* layer, const stief_batch* batch, const uint16_t* k_new,
                  const uint16_t* v_new, int32_t* status, void* stream);
 
-/* Split-T planning.  The context of every sequence is cut into at most S chunks of
- * chunk_pages = ceil(max_pages_per_seq / S) pages; chunk s covers pages [s*chunk_pages, (s+1)*chunk_pages)
- * clipped to the sequence.  stief_decode_num_splits proposes S for the current device;
- * stief_decode_workspace_bytes sizes the scratch buffer for a given S.  Workspace layout (fp32):
- *   q_proj      [B][Hq][r_k]        scaled projected queries (q U_k) * log2(e)/sqrt(128)
- *   partial_o   [B][Hq][S][r_v]     chunk-normalised mixes p V_down (compressed space)
- *   partial_lse [B][Hq][S]          natural-log sum-exp of each chunk's scores
- * The buffer must be 128-byte aligned. */
-int32_t stief_decode_num_splits(int32_t B, int32_t Hkv, int32_t max_pages_per_seq);
-size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t r_k, int32_t r_v, int32_t num_splits);
+/* Split-T planning.  The page tiles of the whole batch (one tile = 64 tokens of one KV head) are laid
+ * end to end -- units (sequence, KV head, tile of up to 8 query heads) in that order -- and cut into
+ * num_parts contiguous ranges of equal size, one per CTA of a persistent kernel; a range cuts one
+ * "segment" out of every unit it overlaps and each segment yields one chunk-normalised partial
+ * result.  num_parts = 0 lets the library choose (one CTA per SM of the current device, which is also
+ * what stief_decode_num_parts returns); it must not exceed 65535.  The same num_parts must be given
+ * to stief_decode_workspace_bytes and to every call that shares the workspace.
+ * Workspace layout, n_units = B * Hkv * ceil((Hq/Hkv) / 8):
+ *   counters    int32 [n_units]                    arrivals per unit; zero between calls
+ *   partial_o   fp32  [num_parts + n_units][8][r_v]  chunk-normalised mixes p V_down (compressed space)
+ *   partial_lse fp32  [num_parts + n_units][8]       natural-log sum-exp of each segment's scores
+ * The buffer must be 128-byte aligned and must be cleared once with stief_decode_workspace_init
+ * (a cudaMemsetAsync of the whole buffer) before its first use; calls that end normally leave the
+ * counters zero again.  Calls that share a workspace must not overlap on the GPU.  B <= 1024. */
+int32_t stief_decode_num_parts(void);
+size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t r_v, int32_t num_parts);
+int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Decode attention (Eq. 18 on the reconstructions of Eq. 7, one query row per head): q [B][Hq][128]
  * bf16 attends to tokens [0, seq_lens[b] + len_add) of every sequence; len_add is 0, or 1 when the
- * token of this step was appended on the same stream and seq_lens not yet advanced.  Runs the query
- * projection, the split-T kernel (scores, online softmax, mix, all in the compressed space) and, when
- * `out` is not NULL, stief_split_combine.  out [B][Hq][128] bf16; out_lse [B][Hq] fp32 natural-log
- * sum-exp, optional.  A sequence of length 0 yields a zero row and lse = -inf.
- * num_splits 0 lets the library choose (the workspace must then hold stief_decode_num_splits splits). */
+ * token of this step was appended on the same stream and seq_lens not yet advanced.  One kernel
+ * launch: query projection q U_k (the projection that compressing keys induces on queries, Sec. 2.2),
+ * scores, online softmax and mix in the compressed space, and, when `out` is not NULL, the merge and
+ * back-projection of stief_split_combine done by whichever CTA delivers a unit's last partial.
+ * out [B][Hq][128] bf16; out_lse [B][Hq] fp32 natural-log sum-exp, optional.  A sequence of length 0
+ * yields a zero row and lse = -inf.  With out == NULL only the partials are written. */
 int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
-                           int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_splits,
+                           int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
                            uint16_t* out, float* out_lse, int32_t* status, void* stream);
 
-/* Merge of the per-chunk results by log-sum-exp (an exact re-association of Eq. 18) followed by the
+/* Merge of the per-segment results by log-sum-exp (an exact re-association of Eq. 18) followed by the
  * back-projection o = o_down U_v^T (Eq. 7 applied to the mixed values; linear, so done once after the
- * merge).  Reads the workspace written by stief_decode_attention with the same batch, len_add and
- * num_splits.  Chunks beyond a sequence's length weigh nothing and are never read. */
+ * merge).  Reads the workspace written by stief_decode_attention (called with out == NULL) with the
+ * same batch, len_add and num_parts.  Only segments that hold tokens are read. */
 int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int32_t len_add,
-                        const void* workspace, int32_t num_splits, uint16_t* out, float* out_lse,
+                        const void* workspace, int32_t num_parts, uint16_t* out, float* out_lse,
                         int32_t* status, void* stream);
 
-/* One decode step of one layer: append (k_new, v_new) at seq_lens[b], then attend over
- * seq_lens[b] + 1 tokens.  Same result as stief_append followed by stief_decode_attention with
- * len_add = 1, in fewer launches. */
+/* One decode step of one layer in one kernel launch: project and store (k_new, v_new) at position
+ * seq_lens[b] (Eq. 1), then attend over seq_lens[b] + 1 tokens.  Same result as stief_append followed
+ * by stief_decode_attention with len_add = 1. */
 int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
                       const uint16_t* k_new, const uint16_t* v_new, void* workspace,
-                      size_t workspace_bytes, int32_t num_splits, uint16_t* out, float* out_lse,
+                      size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
                       int32_t* status, void* stream);
 
 /* The same step for callers whose activations live in host memory: q_host, k_new_host, v_new_host
@@ -140,7 +148,7 @@ int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const 
 size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
                            const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging,
-                           void* workspace, size_t workspace_bytes, int32_t num_splits,
+                           void* workspace, size_t workspace_bytes, int32_t num_parts,
                            uint16_t* out_host, int32_t* status, void* stream);
 
 /* seq_lens[b] += delta on the device (so a captured step can be replayed). */
@@ -148,7 +156,7 @@ int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* st
 
 /* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
  * stief_decode_step_host call made by this host thread records `start_event` just before and
- * `stop_event` just after its split-T kernel on the call's stream (both cudaEvent_t passed as void*),
+ * `stop_event` just after its decode kernel on the call's stream (both cudaEvent_t passed as void*),
  * so the kernel can be timed alone inside a longer step.  One-shot: cleared by that call.  Passing NULLs
  * cancels a pending request. */
 int stief_time_next_decode_kernel(void* start_event, void* stop_event);

@@ -58,8 +58,9 @@ def lib() -> ctypes.CDLL:
         sig = {
             "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, P, P]),
             "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
-            "stief_decode_num_splits": (I32, [I32, I32, I32]),
+            "stief_decode_num_parts": (I32, []),
             "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
+            "stief_decode_workspace_init": (ctypes.c_int, [P, SZ, P]),
             "stief_decode_attention": (ctypes.c_int, [LP, BP, P, I32, P, SZ, I32, P, P, P, P]),
             "stief_split_combine": (ctypes.c_int, [LP, BP, I32, P, I32, P, P, P, P]),
             "stief_decode_step": (ctypes.c_int, [LP, BP, P, P, P, P, SZ, I32, P, P, P, P]),
@@ -148,36 +149,41 @@ def stief_append(layer: Layer, batch: Batch, k_new: torch.Tensor, v_new: torch.T
            "stief_append")
 
 
-def stief_decode_num_splits(B: int, Hkv: int, max_pages_per_seq: int) -> int:
-    return lib().stief_decode_num_splits(B, Hkv, max_pages_per_seq)
+def stief_decode_num_parts() -> int:
+    return lib().stief_decode_num_parts()
 
 
-def stief_decode_workspace_bytes(B: int, Hq: int, r_k: int, r_v: int, num_splits: int) -> int:
-    return lib().stief_decode_workspace_bytes(B, Hq, r_k, r_v, num_splits)
+def stief_decode_workspace_bytes(B: int, Hq: int, Hkv: int, r_v: int, num_parts: int = 0) -> int:
+    return lib().stief_decode_workspace_bytes(B, Hq, Hkv, r_v, num_parts)
 
 
-def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, num_splits: int = 0,
+def stief_decode_workspace_init(workspace: torch.Tensor):
+    _check(lib().stief_decode_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+           "stief_decode_workspace_init")
+
+
+def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, num_parts: int = 0,
                            out: Optional[torch.Tensor] = None, out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
                            status: Optional[torch.Tensor] = None):
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
-                                        workspace.numel() * workspace.element_size(), num_splits, _ptr(out), _ptr(out_lse),
+                                        workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
                                         _ptr(status), _stream()), "stief_decode_attention")
 
 
-def stief_split_combine(layer: Layer, batch: Batch, workspace: torch.Tensor, num_splits: int, out: torch.Tensor,
+def stief_split_combine(layer: Layer, batch: Batch, workspace: torch.Tensor, num_parts: int, out: torch.Tensor,
                         out_lse: Optional[torch.Tensor] = None, len_add: int = 0, status: Optional[torch.Tensor] = None):
     cl, cb = layer.c(), batch.c()
-    _check(lib().stief_split_combine(ctypes.byref(cl), ctypes.byref(cb), len_add, _ptr(workspace), num_splits, _ptr(out),
+    _check(lib().stief_split_combine(ctypes.byref(cl), ctypes.byref(cb), len_add, _ptr(workspace), num_parts, _ptr(out),
                                      _ptr(out_lse), _ptr(status), _stream()), "stief_split_combine")
 
 
 def stief_decode_step(layer: Layer, batch: Batch, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
-                      workspace: torch.Tensor, out: torch.Tensor, num_splits: int = 0, out_lse: Optional[torch.Tensor] = None,
+                      workspace: torch.Tensor, out: torch.Tensor, num_parts: int = 0, out_lse: Optional[torch.Tensor] = None,
                       status: Optional[torch.Tensor] = None):
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_step(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
-                                   workspace.numel() * workspace.element_size(), num_splits, _ptr(out), _ptr(out_lse),
+                                   workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
                                    _ptr(status), _stream()), "stief_decode_step")
 
 
@@ -186,14 +192,14 @@ def stief_host_staging_bytes(B: int, Hq: int, Hkv: int) -> int:
 
 
 def stief_decode_step_host(layer: Layer, batch: Batch, q_host: torch.Tensor, k_new_host: torch.Tensor, v_new_host: torch.Tensor,
-                           staging: torch.Tensor, workspace: torch.Tensor, out_host: torch.Tensor, num_splits: int = 0,
+                           staging: torch.Tensor, workspace: torch.Tensor, out_host: torch.Tensor, num_parts: int = 0,
                            status: Optional[torch.Tensor] = None):
     """Host (pinned) q/k/v/out buffers; copies and kernels are enqueued, nothing is synchronised."""
     assert not q_host.is_cuda and not out_host.is_cuda
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_step_host(ctypes.byref(cl), ctypes.byref(cb), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
                                         _ptr(staging), _ptr(workspace), workspace.numel() * workspace.element_size(),
-                                        num_splits, _ptr(out_host), _ptr(status), _stream()), "stief_decode_step_host")
+                                        num_parts, _ptr(out_host), _ptr(status), _stream()), "stief_decode_step_host")
 
 
 def stief_advance_seq_lens(seq_lens: torch.Tensor, delta: int = 1):

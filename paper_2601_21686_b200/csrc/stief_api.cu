@@ -1,8 +1,9 @@
-// C-ABI entry points: argument checks, split planning, workspace carving, tensor-map encoding and
-// kernel launches.  No allocation, no synchronisation; everything is enqueued on the caller's stream.
+// C-ABI entry points: argument checks, workspace carving, tensor-map encoding and kernel launches.
+// No allocation, no synchronisation; everything is enqueued on the caller's stream.
 #include <cstring>
 
 #include "stief_kernels.h"
+#include "stief_partition.cuh"
 
 namespace stief {
 
@@ -13,7 +14,7 @@ cudaError_t launch_decode_rk96(const DecodeLaunch&, const CUtensorMap&, const CU
 cudaError_t launch_decode_rk128(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
 
 cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st) {
-  switch (a.L.r_k) {
+  switch (a.args.L.r_k) {
     case 32: return launch_decode_rk32(a, tmK, tmV, st);
     case 48: return launch_decode_rk48(a, tmK, tmV, st);
     case 64: return launch_decode_rk64(a, tmK, tmV, st);
@@ -46,7 +47,7 @@ int check_layer(const stief_layer* l) {
 }
 int check_batch(const stief_batch* b) {
   if (!b || b->B <= 0 || b->max_pages_per_seq <= 0 || !b->block_table || !b->seq_lens) return STIEF_ERR_INVALID_ARG;
-  if (b->B > 65535) return STIEF_ERR_INVALID_ARG;
+  if (b->B > kMaxBatch) return STIEF_ERR_INVALID_ARG;
   return STIEF_OK;
 }
 
@@ -82,32 +83,27 @@ int sm_count() {
   return cached[dev];
 }
 
-// The one place that turns (max_pages, requested splits) into (chunk_pages, S): decode and combine
-// must agree on it because it fixes the workspace layout.
-void plan_splits(int max_pages, int requested, int* chunk_pages, int* S) {
-  int s = requested < 1 ? 1 : requested;
-  if (s > max_pages) s = max_pages;
-  const int cp = (max_pages + s - 1) / s;
-  *chunk_pages = cp;
-  *S = (max_pages + cp - 1) / cp;
-}
+int resolve_parts(int num_parts) { return num_parts > 0 ? num_parts : sm_count(); }
+int query_tiles(int Hq, int Hkv) { return (Hq / Hkv + kGroupTile - 1) / kGroupTile; }
 
 struct Workspace {
-  float* q_proj;
+  int* counters;
   float* partial_o;
   float* partial_lse;
   size_t bytes;
 };
-Workspace carve(void* base, int B, int Hq, int r_k, int r_v, int S) {
+Workspace carve(void* base, int B, int Hq, int Hkv, int r_v, int n_cta) {
   Workspace w;
+  const size_t n_units = (size_t)B * Hkv * query_tiles(Hq, Hkv);
+  const size_t slots = n_units + (size_t)n_cta;
   size_t off = 0;
   uint8_t* p = static_cast<uint8_t*>(base);
-  w.q_proj = reinterpret_cast<float*>(p + off);
-  off += align_up((size_t)B * Hq * r_k * 4, 128);
+  w.counters = reinterpret_cast<int*>(p + off);
+  off += align_up(n_units * 4, 128);
   w.partial_o = reinterpret_cast<float*>(p + off);
-  off += align_up((size_t)B * Hq * S * r_v * 4, 128);
+  off += align_up(slots * kGroupTile * r_v * 4, 128);
   w.partial_lse = reinterpret_cast<float*>(p + off);
-  off += align_up((size_t)B * Hq * S * 4, 128);
+  off += align_up(slots * kGroupTile * 4, 128);
   w.bytes = off;
   return w;
 }
@@ -147,7 +143,7 @@ bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
 thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 
 int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
-               const uint16_t* v_new, int len_add, void* workspace, size_t workspace_bytes, int num_splits, uint16_t* out,
+               const uint16_t* v_new, int len_add, void* workspace, size_t workspace_bytes, int num_parts, uint16_t* out,
                float* out_lse, int32_t* status, cudaStream_t st) {
   int rc = check_layer(layer);
   if (rc) return rc;
@@ -157,46 +153,41 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   if ((k_new == nullptr) != (v_new == nullptr)) return STIEF_ERR_INVALID_ARG;
   if (k_new && (!aligned(k_new, 16) || !aligned(v_new, 16))) return STIEF_ERR_INVALID_ARG;
   if (out && !aligned(out, 16)) return STIEF_ERR_INVALID_ARG;
-  if (len_add < 0 || len_add > 1) return STIEF_ERR_INVALID_ARG;
-  if (num_splits < 0) return STIEF_ERR_INVALID_ARG;
-  if (num_splits == 0) num_splits = stief_decode_num_splits(batch->B, layer->Hkv, batch->max_pages_per_seq);
-  int chunk_pages, S;
-  plan_splits(batch->max_pages_per_seq, num_splits, &chunk_pages, &S);
-  if (S > 65535 || (long long)layer->Hkv * ((layer->Hq / layer->Hkv + 7) / 8) > 65535) return STIEF_ERR_INVALID_ARG;
-  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->r_k, layer->r_v, S);
+  if (len_add < 0 || len_add > 1 || (k_new && len_add != 1)) return STIEF_ERR_INVALID_ARG;
+  if (num_parts < 0 || num_parts > 65535) return STIEF_ERR_INVALID_ARG;
+  const int n_cta = resolve_parts(num_parts);
+  const int QT = query_tiles(layer->Hq, layer->Hkv);
+  if ((long long)batch->B * batch->max_pages_per_seq * layer->Hkv * QT >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
+  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
   if (w.bytes > workspace_bytes) return STIEF_ERR_WORKSPACE;
 
-  const LayerDev L = to_dev(layer);
-  const BatchDev Bt = to_dev(batch);
   const long long rows = (long long)layer->num_pages * layer->Hkv * kPage;
   CUtensorMap tmK, tmV;
   if (!make_pool_map(&tmK, layer->k_pool, layer->r_k, rows) || !make_pool_map(&tmV, layer->v_pool, layer->r_v, rows))
     return STIEF_ERR_CUDA;
 
-  PreArgs pa;
-  pa.L = L; pa.Bt = Bt;
-  pa.q = reinterpret_cast<const __nv_bfloat16*>(q);
-  pa.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
-  pa.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  pa.q_proj = w.q_proj; pa.status = status;
-  if (launch_pre(pa, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  DecodeLaunch dl;
+  dl.n_cta = n_cta;
+  DecodeArgs& a = dl.args;
+  a.L = to_dev(layer);
+  a.Bt = to_dev(batch);
+  a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
+  a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
+  a.partial_o = w.partial_o;
+  a.partial_lse = w.partial_lse;
+  a.counters = w.counters;
+  a.out = reinterpret_cast<__nv_bfloat16*>(out);
+  a.out_lse = out ? out_lse : nullptr;
+  a.len_add = len_add;
+  a.QT = QT;
+  a.status = status;
 
-  DecodeLaunch da;
-  da.L = L; da.Bt = Bt; da.q_proj = w.q_proj; da.partial_o = w.partial_o; da.partial_lse = w.partial_lse;
-  da.S = S; da.chunk_pages = chunk_pages; da.len_add = len_add; da.status = status;
   cudaEvent_t ev0 = g_ev_start, ev1 = g_ev_stop;
   g_ev_start = g_ev_stop = nullptr;
   if (ev0) cudaEventRecord(ev0, st);
-  if (launch_decode(da, tmK, tmV, st) != cudaSuccess) return STIEF_ERR_CUDA;
+  if (launch_decode(dl, tmK, tmV, st) != cudaSuccess) return STIEF_ERR_CUDA;
   if (ev1) cudaEventRecord(ev1, st);
-
-  if (out) {
-    CombineArgs ca;
-    ca.L = L; ca.Bt = Bt; ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
-    ca.S = S; ca.chunk_pages = chunk_pages; ca.len_add = len_add;
-    ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;
-    if (launch_combine(ca, st) != cudaSuccess) return STIEF_ERR_CUDA;
-  }
   return STIEF_OK;
 }
 
@@ -216,7 +207,6 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
   if (!K || !V || !aligned(K, 16) || !aligned(V, 16)) return STIEF_ERR_INVALID_ARG;
   if (T_max <= 0 || stride_t < (int64_t)layer->Hkv * kD || stride_b < 0 || (stride_t % 8) != 0 || (stride_b % 8) != 0)
     return STIEF_ERR_INVALID_ARG;
-  if (2 * batch->B > 65535) return STIEF_ERR_INVALID_ARG;
   PrefillArgs a;
   a.L = to_dev(layer); a.Bt = to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);
@@ -231,67 +221,59 @@ int stief_append(const stief_layer* layer, const stief_batch* batch, const uint1
   rc = check_batch(batch);
   if (rc) return rc;
   if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return STIEF_ERR_INVALID_ARG;
-  PreArgs pa;
-  pa.L = to_dev(layer); pa.Bt = to_dev(batch);
-  pa.q = nullptr;
-  pa.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
-  pa.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  pa.q_proj = nullptr; pa.status = status;
-  return launch_pre(pa, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+  AppendArgs a;
+  a.L = to_dev(layer); a.Bt = to_dev(batch);
+  a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
+  a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
+  a.status = status;
+  return launch_append(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
-int32_t stief_decode_num_splits(int32_t B, int32_t Hkv, int32_t max_pages_per_seq) {
-  if (B <= 0 || Hkv <= 0 || max_pages_per_seq <= 0) return 1;
-  // aim at ~8 work items per SM (two resident CTAs, four rounds), at least 4 pages per item
-  const long long units = (long long)B * Hkv;
-  const long long target = (long long)sm_count() * 8;
-  long long s = (target + units - 1) / units;
-  const long long smax = (max_pages_per_seq + 3) / 4;
-  if (s > smax) s = smax;
-  if (s < 1) s = 1;
-  int chunk_pages, S;
-  plan_splits(max_pages_per_seq, (int)s, &chunk_pages, &S);
-  return S;
+int32_t stief_decode_num_parts(void) { return sm_count(); }
+
+size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t r_v, int32_t num_parts) {
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || r_v <= 0 || num_parts < 0) return 0;
+  return carve(nullptr, B, Hq, Hkv, r_v, resolve_parts(num_parts)).bytes;
 }
 
-size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t r_k, int32_t r_v, int32_t num_splits) {
-  if (B <= 0 || Hq <= 0 || r_k <= 0 || r_v <= 0 || num_splits <= 0) return 0;
-  return carve(nullptr, B, Hq, r_k, r_v, num_splits).bytes;
+int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace || workspace_bytes == 0) return STIEF_ERR_INVALID_ARG;
+  return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
 int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int32_t len_add,
-                           void* workspace, size_t workspace_bytes, int32_t num_splits, uint16_t* out, float* out_lse,
+                           void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
                            int32_t* status, void* stream) {
-  return run_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_splits, out, out_lse, status,
+  return run_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_parts, out, out_lse, status,
                     static_cast<cudaStream_t>(stream));
 }
 
 int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int32_t len_add, const void* workspace,
-                        int32_t num_splits, uint16_t* out, float* out_lse, int32_t* status, void* stream) {
+                        int32_t num_parts, uint16_t* out, float* out_lse, int32_t* status, void* stream) {
   (void)status;
   int rc = check_layer(layer);
   if (rc) return rc;
   rc = check_batch(batch);
   if (rc) return rc;
-  if (!workspace || !aligned(workspace, 128) || !out || !aligned(out, 16) || num_splits < 0 || len_add < 0 || len_add > 1)
+  if (!workspace || !aligned(workspace, 128) || !out || !aligned(out, 16) || num_parts < 0 || num_parts > 65535 || len_add < 0 ||
+      len_add > 1)
     return STIEF_ERR_INVALID_ARG;
-  if (num_splits == 0) num_splits = stief_decode_num_splits(batch->B, layer->Hkv, batch->max_pages_per_seq);
-  int chunk_pages, S;
-  plan_splits(batch->max_pages_per_seq, num_splits, &chunk_pages, &S);
-  const Workspace w = carve(const_cast<void*>(workspace), batch->B, layer->Hq, layer->r_k, layer->r_v, S);
+  const int n_cta = resolve_parts(num_parts);
+  const Workspace w = carve(const_cast<void*>(workspace), batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
   CombineArgs ca;
   ca.L = to_dev(layer); ca.Bt = to_dev(batch);
   ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
-  ca.S = S; ca.chunk_pages = chunk_pages; ca.len_add = len_add;
+  ca.n_cta = n_cta; ca.QT = query_tiles(layer->Hq, layer->Hkv); ca.len_add = len_add;
   ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;
+  if ((long long)layer->Hkv * ca.QT > 2147483647ll || batch->B > 65535) return STIEF_ERR_INVALID_ARG;
   return launch_combine(ca, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
 int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
-                      const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_splits, uint16_t* out,
+                      const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out,
                       float* out_lse, int32_t* status, void* stream) {
   if (!k_new || !v_new || !out) return STIEF_ERR_INVALID_ARG;
-  return run_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_splits, out, out_lse, status,
+  return run_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_parts, out, out_lse, status,
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -303,7 +285,7 @@ size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv) {
 
 int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
                            const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging, void* workspace,
-                           size_t workspace_bytes, int32_t num_splits, uint16_t* out_host, int32_t* status, void* stream) {
+                           size_t workspace_bytes, int32_t num_parts, uint16_t* out_host, int32_t* status, void* stream) {
   if (!layer || !batch || !q_host || !k_new_host || !v_new_host || !staging || !out_host || !aligned(staging, 128))
     return STIEF_ERR_INVALID_ARG;
   if (batch->B <= 0 || layer->Hq <= 0 || layer->Hkv <= 0) return STIEF_ERR_INVALID_ARG;
@@ -317,7 +299,7 @@ int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, c
   if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
   if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
   if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
-  const int rc = stief_decode_step(layer, batch, dq, dk, dv, workspace, workspace_bytes, num_splits, dout, nullptr, status, stream);
+  const int rc = stief_decode_step(layer, batch, dq, dk, dv, workspace, workspace_bytes, num_parts, dout, nullptr, status, stream);
   if (rc) return rc;
   if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return STIEF_ERR_CUDA;
   return STIEF_OK;
@@ -348,6 +330,6 @@ const char* stief_status_string(int status) {
   }
 }
 
-int stief_version(void) { return 100; }
+int stief_version(void) { return 200; }
 
 }  // extern "C"

@@ -1,105 +1,151 @@
-// Split-T decode attention in the compressed space (scores, online softmax, mix) for one GQA group.
+// Persistent split-T decode attention in the compressed space: one launch does the whole decode step
+// of a layer -- (optional) projection + append of the new token's k, v (Eq. 1), query projection
+// q' = q U_k, scores q' K_down^T, online softmax, mix P V_down, and (optional) the log-sum-exp merge
+// over chunks with the back-projection by U_v^T (Eq. 7, Eq. 18).
 //
-// Work item = (sequence b, KV head h, chunk of pages).  One producer warp streams the chunk's
-// compressed page tiles K_down[64 x RK], V_down[64 x RV] from HBM into a ring of shared-memory
-// stages with TMA (hardware swizzle, completion on mbarriers); NW consumer warps each take every
-// NW-th page, compute the scores S = q' K_down^T of the group's query heads against the 64 tokens on
-// the tensor cores, keep an online softmax in registers, and accumulate P V_down.  Warps merge their
-// running (max, sum, accumulator) at the end and write one chunk-normalised partial [G][RV] + lse.
+// One CTA per SM.  The batch's page tiles are split evenly over the CTAs (stief_partition.cuh); a CTA
+// walks the segments of its range.  A producer warp streams the page tiles K_down[64 x RK],
+// V_down[64 x RV] from HBM into a ring of shared-memory stages with TMA (hardware swizzle, completion
+// on mbarriers) and never stops at segment borders, so the next segment's tiles are already in
+// flight while the consumers finish the current one.  NW consumer warps each take every NW-th page:
+// scores of the group's query heads against the 64 tokens on the tensor cores, online softmax in
+// registers, P V_down accumulated in registers.  At a segment's end the warps merge their running
+// (max, sum, accumulator) and write one chunk-normalised partial; the CTA that delivers a unit's last
+// partial merges all of them and back-projects.
 //
 // Every consumer warp owns SPW private stages of the ring and walks them in order, so each mbarrier
-// is only ever waited on by one warp, phase after phase: a parity wait can tell two adjacent phases
-// apart but not more, and a shared ring would let a fast warp wait on a phase that is two ahead of
-// what a slot has completed.
+// is only ever waited on by one warp, phase after phase (a parity wait can tell two adjacent phases
+// apart but not more).
 //
 // Precision: q' (already scaled by log2(e)/sqrt(128)) and P are each carried as a pair of bf16 words
 // (value + remainder) occupying rows 0-7 and 8-15 of the 16-row MMA operand, so the products see
-// ~16 significant bits of q' and P; accumulation is fp32.  Up to 8 query heads per KV head share one
-// pass; larger groups are tiled over blockIdx.y.
+// ~16 significant bits of q' and P; accumulation is fp32.  Up to 8 query heads of a KV head form one
+// unit; larger groups become several units.
 #pragma once
 
-#include "stief_common.cuh"
-
-#ifndef STIEF_DECODE_NW
-#define STIEF_DECODE_NW 4
-#endif
+#include "stief_decode_args.h"
+#include "stief_partition.cuh"
 
 namespace stief {
-
-struct DecodeArgs {
-  LayerDev L;
-  BatchDev Bt;
-  const float* q_proj;     // [B][Hq][RK]
-  float* partial_o;        // [B][Hq][S][RV]
-  float* partial_lse;      // [B][Hq][S]
-  int S, chunk_pages, len_add;
-  int32_t* status;
-};
 
 template <int RK, int RV>
 struct DecodeCfg {
   using TK = Tile<RK>;
   using TV = Tile<RV>;
-  static constexpr int NW = STIEF_DECODE_NW;            // consumer warps
-  static constexpr int THREADS = (NW + 1) * 32;         // + 1 producer warp
   static constexpr int STAGE_BYTES = TK::BYTES + TV::BYTES;
-  static constexpr int SPW_RAW = (98304 / STAGE_BYTES) / NW;
-  static constexpr int SPW = SPW_RAW < 1 ? 1 : (SPW_RAW > 4 ? 4 : SPW_RAW);   // private stages per consumer warp
+  static constexpr int RING_BUDGET = 192 * 1024;
+  static constexpr int NSTAGE_MAX = RING_BUDGET / STAGE_BYTES;
+  static constexpr int NW = NSTAGE_MAX >= 8 ? 4 : (NSTAGE_MAX >= 6 ? 3 : 2);      // consumer warps
+  static constexpr int SPW = (NSTAGE_MAX / NW) > 4 ? 4 : (NSTAGE_MAX / NW);        // private stages per consumer warp
   static constexpr int NS = NW * SPW;
+  static constexpr int NT = NW * 32;                     // consumer threads
+  static constexpr int THREADS = NT + 32;                // + 1 producer warp
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
-  static constexpr int CTRL_BYTES = 512;                // full[NS], empty[NS], abort flag
-  static constexpr int SMEM_BYTES = RING_BYTES + CTRL_BYTES + 1024;   // + slack to align the ring to 1 KiB
+  // scratch after the ring
+  static constexpr int CTRL_BYTES = 512;                 // full[NS], empty[NS], append barrier, flags
+  static constexpr int PREF_BYTES = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
+  static constexpr int QP_BYTES = kGroupTile * kD * 4;   // q' fp32 [8][RK]
+  static constexpr int ROWS_BYTES = 9 * kD * 4;          // vectors to project: 8 queries + the new key (or value)
+  static constexpr int RED_BYTES = NW * 9 * kD * 4;      // per-warp partial projections
+  static constexpr int UNION_BYTES = ROWS_BYTES + RED_BYTES;   // also: merge scratch [NW][8][RV]+[2][NW][8]; combine scratch [8][128]
+  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + CTRL_BYTES + PREF_BYTES + QP_BYTES + UNION_BYTES;
   static_assert(RK % 16 == 0 && RV % 16 == 0 && RK <= 128 && RV <= 128, "ranks are multiples of 16 up to 128");
-  static_assert(NW * 8 * (RV + 2) * 4 <= RING_BYTES, "merge scratch must fit in the ring");
+  static_assert(SPW >= 1 && NS <= 16, "ring shape");
+  static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= UNION_BYTES, "merge scratch must fit");
+  static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KiB shared memory of an SM");
 };
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(STIEF_DECODE_NW * 32) : "memory"); }
+// sums[r][j] = sum_d rows[r][d] * U[d][j] for r < 9, j < R, by NW warps (warp w contracts d = w, w+NW, ...).
+// rows: shared fp32 [9][128]; red: shared fp32 [NW][9][128]; result left in red[0][r][j].
+template <int NW>
+__device__ __forceinline__ void cta_project(const float* rows, const __nv_bfloat16* __restrict__ U, int R, float* red, int warp, int lane) {
+  for (int cp = lane; cp < R / 2; cp += 32) {
+    float acc[9][2];
+#pragma unroll
+    for (int r = 0; r < 9; ++r) acc[r][0] = acc[r][1] = 0.f;
+    constexpr int ND = (kD + NW - 1) / NW;                // d values per warp
+#pragma unroll 1
+    for (int i0 = 0; i0 < ND; i0 += 8) {
+      uint32_t u[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int d = warp + (i0 + i) * NW;
+        u[i] = (d < kD) ? __ldg(reinterpret_cast<const uint32_t*>(U + (size_t)d * R + 2 * cp)) : 0u;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int d = warp + (i0 + i) * NW;
+        if (d < kD) {
+          const float u0 = bf16_lo(u[i]), u1 = bf16_hi(u[i]);
+#pragma unroll
+          for (int r = 0; r < 9; ++r) {
+            const float x = rows[r * kD + d];
+            acc[r][0] = fmaf(x, u0, acc[r][0]);
+            acc[r][1] = fmaf(x, u1, acc[r][1]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 9; ++r) *reinterpret_cast<float2*>(red + (warp * 9 + r) * kD + 2 * cp) = make_float2(acc[r][0], acc[r][1]);
+  }
+  bar1(NW * 32);
+  for (int idx = warp * 32 + lane; idx < 9 * R; idx += NW * 32) {
+    const int r = idx / R, j = idx % R;
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) s += red[(w * 9 + r) * kD + j];
+    red[r * kD + j] = s;                                  // slot of warp 0; only this thread touches (r, j)
+  }
+  bar1(NW * 32);
+}
 
 template <int RK, int RV>
-__global__ void __launch_bounds__(DecodeCfg<RK, RV>::THREADS, 2)
-decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeArgs a) {
+__global__ void __launch_bounds__(DecodeCfg<RK, RV>::THREADS, 1)
+decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeArgs a) {
   using C = DecodeCfg<RK, RV>;
   using TK = typename C::TK;
   using TV = typename C::TV;
-  constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW;
+  constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW, NT = C::NT;
 
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x;
-  const int h = blockIdx.y % a.L.Hkv;
-  const int qt = blockIdx.y / a.L.Hkv;
-  const int b = blockIdx.z;
-
-  int len = a.Bt.seq_lens[b] + a.len_add;
-  if (len < 0) len = 0;
-  int npages_seq = (len + kPage - 1) / kPage;
-  if (npages_seq > a.Bt.max_pages) {
-    if (tid == 0) report(a.status, STIEF_ERR_BOUNDS);
-    npages_seq = a.Bt.max_pages;
-    len = npages_seq * kPage;
-  }
-  const int p0 = split * a.chunk_pages;
-  const int p1 = min(p0 + a.chunk_pages, npages_seq);
-  if (p0 >= p1) return;                                  // chunk beyond this sequence: nothing to do
-  const int npg = p1 - p0;
+  const int c = blockIdx.x, n_cta = gridDim.x;
 
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t ctrl = ring + C::RING_BYTES;
   uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_ptr + C::RING_BYTES + 2 * NS * 8);
-  static_assert(2 * NS * 8 + 4 <= C::CTRL_BYTES, "control block too small");
+  uint8_t* ctrl_ptr = ring_ptr + C::RING_BYTES;
+  const uint32_t ctrl = ring + C::RING_BYTES;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
-  auto empty_bar = [&](int s) { return ctrl + (NS + s) * 8; };
+  auto empty_bar = [&](int s) { return ctrl + (16 + s) * 8; };
+  const uint32_t append_bar = ctrl + 32 * 8;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);
+  int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
+  float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
+  float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
+    mbar_init(append_bar, 1);
     *abort_flag = 0;
+    *last_flag = 0;
     mbar_fence_init();
   }
-  __syncthreads();
+  build_page_prefix(pref, a.Bt, a.len_add, c == 0 ? a.status : nullptr);   // ends with __syncthreads
+
+  const int B = a.Bt.B, Hkv = a.L.Hkv, QT = a.QT, G = a.L.G;
+  const int upb = Hkv * QT;
+  const int total = pref[B] * upb;
+  const int P = pages_per_cta(total, n_cta);
+  const bool appending = a.k_new != nullptr;
+
+  SegmentWalker walk;
+  walk.init(pref, B, upb, c, P, total);
+  Segment seg;
 
   // ------------------------------------------------------------------ producer warp
   if (warp == NW) {
@@ -107,184 +153,313 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
     }
-    int tbl = 0;
-    for (int i = 0; i < npg; ++i) {
-      if ((i & 31) == 0) {
-        const int idx = p0 + i + lane;
-        tbl = (idx < p1) ? a.Bt.block_table[(size_t)b * a.Bt.max_pages + idx] : 0;
+    int i = 0;                 // pages issued by this CTA so far (across segments)
+    int n_append = 0;          // segments so far that had to wait for the new token's rows
+    while (walk.next(seg)) {
+      const int h = seg.j / QT;
+      const int npg = seg.p1 - seg.p0;
+      bool wait_append = false;
+      if (appending && seg.p1 == seg.npages) {
+        const int pos = a.Bt.seq_lens[seg.b];
+        wait_append = pos >= 0 && pos / kPage < a.Bt.max_pages;
       }
-      int page = __shfl_sync(0xffffffffu, tbl, i & 31);
-      if (page < 0 || page >= a.L.num_pages) {
-        if (lane == 0) report(a.status, STIEF_ERR_BOUNDS);
-        page = 0;
-      }
-      const int slot = (i % NW) * SPW + (i / NW) % SPW;    // private stage of the page's consumer warp
-      const int use = (i / NW) / SPW;                      // how often that stage has been filled before
-      if (lane == 0) {
-        if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
-        const uint32_t st = ring + slot * C::STAGE_BYTES;
-        const int y = (page * a.L.Hkv + h) * kPage;
-        mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
+      int tbl = 0;
+      for (int k = 0; k < npg; ++k, ++i) {
+        if ((k & 31) == 0) {
+          const int idx = seg.p0 + k + lane;
+          tbl = (idx < seg.p1) ? a.Bt.block_table[(size_t)seg.b * a.Bt.max_pages + idx] : 0;
+        }
+        int page = __shfl_sync(0xffffffffu, tbl, k & 31);
+        if (page < 0 || page >= a.L.num_pages) {
+          if (lane == 0) report(a.status, STIEF_ERR_BOUNDS);
+          page = 0;
+        }
+        const int cw = i % NW, kw = i / NW;               // consumer warp of this page, its k-th page
+        const int slot = cw * SPW + kw % SPW;
+        const int use = kw / SPW;
+        if (lane == 0) {
+          if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
+          if (wait_append && k == npg - 1) {
+            // the sequence's last page receives the new token's rows from this CTA's consumers first
+            mbar_wait(append_bar, n_append & 1, abort_flag, a.status);
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+          }
+          const uint32_t st = ring + slot * C::STAGE_BYTES;
+          const int y = (page * Hkv + h) * kPage;
+          mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
 #pragma unroll
-        for (int nb = 0; nb < TK::NB; ++nb) tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, nb * TK::BW, y, full_bar(slot));
+          for (int nb = 0; nb < TK::NB; ++nb) tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, nb * TK::BW, y, full_bar(slot));
 #pragma unroll
-        for (int nb = 0; nb < TV::NB; ++nb)
-          tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, nb * TV::BW, y, full_bar(slot));
+          for (int nb = 0; nb < TV::NB; ++nb)
+            tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, nb * TV::BW, y, full_bar(slot));
+        }
+        __syncwarp();
       }
-      __syncwarp();
+      if (wait_append) ++n_append;
     }
     return;
   }
 
   // ------------------------------------------------------------------ consumer warps
-  const int gid = lane >> 2, tid4 = lane & 3;
-  const int G = a.L.G;
-  const int g = qt * 8 + gid;                            // query head inside the group (row of the MMA)
-  const bool row_ok = g < G;
+  const int gid = lane >> 2, tid4 = lane & 3, l7 = lane & 7;
+  const float qscale = kLog2e * 0.08838834764831845f;     // log2(e) / sqrt(128)
 
-  // A operand of the score MMA: rows 0-7 = bf16(q'), rows 8-15 = bf16(q' - bf16(q'))
-  uint32_t qa[RK / 16][4];
-  {
-    const float* qp = a.q_proj + ((size_t)b * a.L.Hq + (size_t)h * G + (row_ok ? g : 0)) * RK;
+  // units of empty sequences get their zero rows from CTA (u mod n_cta)
+  if (a.out != nullptr) {
+    for (int u = c; u < B * upb; u += n_cta) {
+      const int b = u / upb, j = u % upb;
+      if (pref[b + 1] != pref[b]) continue;
+      const int h = j / QT, qt = j % QT;
+      const int ng = min(kGroupTile, G - qt * kGroupTile);
+      const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
+      for (int idx = tid; idx < ng * kD; idx += NT) a.out[head0 * kD + idx] = __float2bfloat16_rn(0.f);
+      if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
+    }
+  }
+
+  // per-lane pieces of the ldmatrix addresses (the swizzle term depends on the lane only)
+  constexpr int NCH = RK / 8;
+  uint32_t koff[(NCH + 3) / 4];
+#pragma unroll
+  for (int q4 = 0; q4 < (NCH + 3) / 4; ++q4) {
+    const int cc = (4 * q4 + 4 <= NCH) ? 4 * q4 + (lane >> 3) : 4 * q4 + ((lane >> 3) & 1);
+    koff[q4] = TK::chunk(l7, cc);
+  }
+  uint32_t voff[RV / 16];
+#pragma unroll
+  for (int np = 0; np < RV / 16; ++np) voff[np] = TV::chunk(l7 + ((lane >> 3) & 1) * 8, 2 * np + (lane >> 4));
+
+  int i_base = 0;              // pages of this CTA before the current segment
+
+  while (walk.next(seg)) {
+    const int b = seg.b, h = seg.j / QT, qt = seg.j % QT;
+    const int npg = seg.p1 - seg.p0;
+    const int ng = min(kGroupTile, G - qt * kGroupTile);
+    const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
+    const int len_raw = a.Bt.seq_lens[b] + a.len_add;
+    const int len = min(max(len_raw, 0), seg.npages * kPage);
+    const int last_valid = len - (seg.npages - 1) * kPage;          // tokens in the sequence's last page (1..64)
+    const bool has_final = seg.p1 == seg.npages;
+    bool do_append = false;
+    size_t new_row = 0;
+    if (appending && has_final) {
+      const int pos = a.Bt.seq_lens[b];
+      if (pos >= 0 && pos / kPage < a.Bt.max_pages) {
+        do_append = true;                                            // the producer waits for our signal
+        const int page = a.Bt.block_table[(size_t)b * a.Bt.max_pages + pos / kPage];
+        if (page < 0 || page >= a.L.num_pages) {
+          new_row = ~(size_t)0;                                      // bad page: signal, but store nothing
+        } else {
+          new_row = ((size_t)page * Hkv + h) * kPage + (pos % kPage);
+        }
+      }
+    }
+
+    // ---- vectors contracted with U_k: the unit's queries (rows 0..7) and the new key (row 8)
+    float* rows = un;
+    float* red = un + 9 * kD;
+    for (int idx = tid; idx < 9 * kD; idx += NT) {
+      const int r = idx / kD, d = idx % kD;
+      float x = 0.f;
+      if (r < ng) x = __bfloat162float(a.q[(head0 + r) * kD + d]);
+      else if (r == 8 && do_append) x = __bfloat162float(a.k_new[((size_t)b * Hkv + h) * kD + d]);
+      rows[idx] = x;
+    }
+    bar1(NT);
+    const __nv_bfloat16* Uk = a.L.U_k ? a.L.U_k + (size_t)h * a.L.uk_stride : nullptr;
+    const float* res = rows;
+    if (Uk) {
+      cta_project<NW>(rows, Uk, RK, red, warp, lane);
+      res = red;
+    }
+    for (int idx = tid; idx < 9 * RK; idx += NT) {
+      const int r = idx / RK, j = idx % RK;
+      const float x = res[r * kD + j];
+      if (r < 8) qp[r * RK + j] = x * qscale;
+      else if (do_append && new_row != ~(size_t)0) a.L.k_pool[new_row * RK + j] = __float2bfloat16_rn(x);
+    }
+    if (do_append) {
+      bar1(NT);
+      for (int idx = tid; idx < 9 * kD; idx += NT)
+        rows[idx] = idx < kD ? __bfloat162float(a.v_new[((size_t)b * Hkv + h) * kD + idx]) : 0.f;
+      bar1(NT);
+      const __nv_bfloat16* Uv = a.L.U_v ? a.L.U_v + (size_t)h * a.L.uv_stride : nullptr;
+      res = rows;
+      if (Uv) {
+        cta_project<NW>(rows, Uv, RV, red, warp, lane);
+        res = red;
+      }
+      if (new_row != ~(size_t)0) {
+        for (int j = tid; j < RV; j += NT) a.L.v_pool[new_row * RV + j] = __float2bfloat16_rn(res[j]);
+      } else if (tid == 0) {
+        report(a.status, STIEF_ERR_BOUNDS);
+      }
+      __threadfence();
+      asm volatile("fence.proxy.async.global;" ::: "memory");
+    }
+    bar1(NT);
+    if (do_append && tid == 0) mbar_arrive(append_bar);               // rows are in the pool: the last page may be fetched
+
+    // A operand of the score MMA: rows 0-7 = bf16(q'), rows 8-15 = bf16(q' - bf16(q'))
+    uint32_t qa[RK / 16][4];
 #pragma unroll
     for (int ks = 0; ks < RK / 16; ++ks) {
-      float2 x = make_float2(0.f, 0.f), y = make_float2(0.f, 0.f);
-      if (row_ok) {
-        x = *reinterpret_cast<const float2*>(qp + 16 * ks + 2 * tid4);
-        y = *reinterpret_cast<const float2*>(qp + 16 * ks + 8 + 2 * tid4);
-      }
+      const float2 x = *reinterpret_cast<const float2*>(qp + gid * RK + 16 * ks + 2 * tid4);
+      const float2 y = *reinterpret_cast<const float2*>(qp + gid * RK + 16 * ks + 8 + 2 * tid4);
       split_bf16(x.x, x.y, qa[ks][0], qa[ks][1]);
       split_bf16(y.x, y.y, qa[ks][2], qa[ks][3]);
     }
-  }
 
-  float m = -INFINITY, l = 0.f;
-  float o[RV / 8][4];
+    float m = -INFINITY, l = 0.f;
+    float o[RV / 8][4];
 #pragma unroll
-  for (int n = 0; n < RV / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    for (int n = 0; n < RV / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
 
-  const int last_valid = len - (npages_seq - 1) * kPage;   // tokens in the sequence's last page (1..64)
+    // first page of this segment that belongs to this warp: global index i = i_base + k, i % NW == warp
+    int k0 = (warp - i_base % NW + NW) % NW;
+    for (int k = k0; k < npg; k += NW) {
+      const int kw = (i_base + k) / NW;
+      const int slot = warp * SPW + kw % SPW;
+      mbar_wait(full_bar(slot), (kw / SPW) & 1, abort_flag, a.status);
+      const uint32_t kt = ring + slot * C::STAGE_BYTES;
+      const uint32_t vt = kt + TK::BYTES;
+      const bool tail = (seg.p0 + k == seg.npages - 1) && (last_valid < kPage);
 
-  for (int i = warp; i < npg; i += NW) {
-    const int slot = warp * SPW + (i / NW) % SPW;
-    mbar_wait(full_bar(slot), ((i / NW) / SPW) & 1, abort_flag, a.status);
-    const uint32_t kt = ring + slot * C::STAGE_BYTES;
-    const uint32_t vt = kt + TK::BYTES;
-    const bool tail = (p0 + i == npages_seq - 1) && (last_valid < kPage);
-
-    // ---- scores of the page: s[j] covers tokens 8j..8j+7; c0,c1 from bf16(q'), c2,c3 from the remainder
-    float sc[16];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float s[4] = {0.f, 0.f, 0.f, 0.f};
-      constexpr int NCH = RK / 8;
-#pragma unroll
-      for (int kc = 0; kc + 4 <= NCH; kc += 4) {
-        uint32_t r0, r1, r2, r3;
-        ldsm_x4(kt + TK::chunk(8 * j + (lane & 7), kc + (lane >> 3)), r0, r1, r2, r3);
-        mma_bf16(s, qa[kc / 2], r0, r1);
-        mma_bf16(s, qa[kc / 2 + 1], r2, r3);
-      }
-      if constexpr (NCH % 4 == 2) {
-        uint32_t r0, r1;
-        ldsm_x2(kt + TK::chunk(8 * j + (lane & 7), NCH - 2 + ((lane >> 3) & 1)), r0, r1);
-        mma_bf16(s, qa[NCH / 2 - 1], r0, r1);
-      }
-      sc[2 * j] = s[0] + s[2];
-      sc[2 * j + 1] = s[1] + s[3];
-    }
-    if (tail) {
+      // ---- scores of the page: n-tile j covers tokens 8j..8j+7; c0,c1 from bf16(q'), c2,c3 from the remainder
+      float sc[16];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const int t = 8 * j + 2 * tid4;
-        if (t >= last_valid) sc[2 * j] = -INFINITY;
-        if (t + 1 >= last_valid) sc[2 * j + 1] = -INFINITY;
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int q4 = 0; 4 * q4 + 4 <= NCH; ++q4) {
+          uint32_t r0, r1, r2, r3;
+          ldsm_x4(kt + koff[q4] + j * 8 * TK::RB, r0, r1, r2, r3);
+          mma_bf16(s, qa[2 * q4], r0, r1);
+          mma_bf16(s, qa[2 * q4 + 1], r2, r3);
+        }
+        if constexpr (NCH % 4 == 2) {
+          uint32_t r0, r1;
+          ldsm_x2(kt + koff[NCH / 4] + j * 8 * TK::RB, r0, r1);
+          mma_bf16(s, qa[NCH / 2 - 1], r0, r1);
+        }
+        sc[2 * j] = s[0] + s[2];
+        sc[2 * j + 1] = s[1] + s[3];
       }
-      // rows past the end hold unspecified bits: zero them in V so that 0 * garbage cannot make a NaN
-      constexpr int NCV = RV / 8;
-      for (int idx = lane; idx < (kPage - last_valid) * NCV; idx += 32) {
-        const int t = last_valid + idx / NCV, c = idx % NCV;
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vt + TV::chunk(t, c)), "r"(0u) : "memory");
+      if (tail) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = 8 * j + 2 * tid4;
+          if (t >= last_valid) sc[2 * j] = -INFINITY;
+          if (t + 1 >= last_valid) sc[2 * j + 1] = -INFINITY;
+        }
+        // rows past the end hold unspecified bits: zero them in V so that 0 * garbage cannot make a NaN
+        constexpr int NCV = RV / 8;
+        for (int idx = lane; idx < (kPage - last_valid) * NCV; idx += 32) {
+          const int t = last_valid + idx / NCV, cc = idx % NCV;
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vt + TV::chunk(t, cc)), "r"(0u) : "memory");
+        }
+        __syncwarp();
       }
-      __syncwarp();
-    }
 
-    // ---- online softmax (base 2; the scale is folded into q')
-    float mx = sc[0];
+      // ---- online softmax (base 2; the scale is folded into q')
+      float mx = sc[0];
 #pragma unroll
-    for (int e = 1; e < 16; ++e) mx = fmaxf(mx, sc[e]);
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    const float m_new = fmaxf(m, mx);
-    const float alpha = fast_exp2(m - m_new);
-    m = m_new;
-    uint32_t pa[4][4];
-    float ps = 0.f;
+      for (int e = 1; e < 16; ++e) mx = fmaxf(mx, sc[e]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m, mx);
+      const float alpha = fast_exp2(m - m_new);
+      m = m_new;
+      uint32_t pa[4][4];
+      float ps = 0.f;
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      const float p0_ = fast_exp2(sc[4 * kk + 0] - m), p1_ = fast_exp2(sc[4 * kk + 1] - m);
-      const float p2_ = fast_exp2(sc[4 * kk + 2] - m), p3_ = fast_exp2(sc[4 * kk + 3] - m);
-      ps += (p0_ + p1_) + (p2_ + p3_);
-      split_bf16(p0_, p1_, pa[kk][0], pa[kk][1]);
-      split_bf16(p2_, p3_, pa[kk][2], pa[kk][3]);
+      for (int kk = 0; kk < 4; ++kk) {
+        const float p0_ = fast_exp2(sc[4 * kk + 0] - m), p1_ = fast_exp2(sc[4 * kk + 1] - m);
+        const float p2_ = fast_exp2(sc[4 * kk + 2] - m), p3_ = fast_exp2(sc[4 * kk + 3] - m);
+        ps += (p0_ + p1_) + (p2_ + p3_);
+        split_bf16(p0_, p1_, pa[kk][0], pa[kk][1]);
+        split_bf16(p2_, p3_, pa[kk][2], pa[kk][3]);
+      }
+      l = l * alpha + ps;
+#pragma unroll
+      for (int n = 0; n < RV / 8; ++n) {
+        o[n][0] *= alpha; o[n][1] *= alpha; o[n][2] *= alpha; o[n][3] *= alpha;
+      }
+
+      // ---- mix: o += P V_down (tokens are the contraction index; V tile read transposed)
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+        for (int np = 0; np < RV / 16; ++np) {
+          uint32_t r0, r1, r2, r3;
+          ldsm_x4_t(vt + voff[np] + kk * 16 * TV::RB, r0, r1, r2, r3);
+          mma_bf16(o[2 * np], pa[kk], r0, r1);
+          mma_bf16(o[2 * np + 1], pa[kk], r2, r3);
+        }
+      }
+
+      if (tail) fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar(slot));
     }
-    l = l * alpha + ps;
+    i_base += npg;
+
+    // ------------------------------------------------------------------ merge the warps of this segment
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    float* wo = un;                      // [NW][8][RV]
+    float* wm = wo + NW * 8 * RV;        // [NW][8]
+    float* wl = wm + NW * 8;             // [NW][8]
 #pragma unroll
     for (int n = 0; n < RV / 8; ++n) {
-      o[n][0] *= alpha; o[n][1] *= alpha; o[n][2] *= alpha; o[n][3] *= alpha;
+      *reinterpret_cast<float2*>(wo + (warp * 8 + gid) * RV + 8 * n + 2 * tid4) = make_float2(o[n][0] + o[n][2], o[n][1] + o[n][3]);
+    }
+    if (tid4 == 0) {
+      wm[warp * 8 + gid] = m;
+      wl[warp * 8 + gid] = l;
+    }
+    bar1(NT);
+    const int u = b * upb + seg.j;
+    const int slot_id = c + u;
+    for (int idx = tid; idx < ng * RV; idx += NT) {
+      const int gg = idx / RV, j = idx % RV;
+      float M = wm[gg];
+#pragma unroll
+      for (int w = 1; w < NW; ++w) M = fmaxf(M, wm[w * 8 + gg]);
+      float num = 0.f, den = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const float e = fast_exp2(wm[w * 8 + gg] - M);
+        num += e * wo[(w * 8 + gg) * RV + j];
+        den += e * wl[w * 8 + gg];
+      }
+      __stcg(a.partial_o + ((size_t)slot_id * kGroupTile + gg) * RV + j, num / den);
+      if (j == 0) __stcg(a.partial_lse + (size_t)slot_id * kGroupTile + gg, (M + log2f(den)) * kLn2);
     }
 
-    // ---- mix: o += P V_down (tokens are the contraction index; V tile read transposed)
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-      for (int np = 0; np < RV / 16; ++np) {
-        uint32_t r0, r1, r2, r3;
-        ldsm_x4_t(vt + TV::chunk(16 * kk + (lane & 7) + ((lane >> 3) & 1) * 8, 2 * np + (lane >> 4)), r0, r1, r2, r3);
-        mma_bf16(o[2 * np], pa[kk], r0, r1);
-        mma_bf16(o[2 * np + 1], pa[kk], r2, r3);
+    // ------------------------------------------------------------------ the unit's last partial triggers the combine
+    if (a.out != nullptr) {
+      int first, last;
+      unit_cta_span(pref, upb, P, b, seg.j, &first, &last);
+      const int nseg = last - first + 1;
+      __threadfence();
+      bar1(NT);
+      if (tid == 0) {
+        int is_last = 1;
+        if (nseg > 1) {
+          const int prev = atomicAdd(a.counters + u, 1);
+          is_last = (prev == nseg - 1);
+          if (is_last) a.counters[u] = 0;                  // leave the counter clean for the next call
+        }
+        *last_flag = is_last;
+      }
+      bar1(NT);
+      if (*last_flag) {
+        __threadfence();
+        combine_unit(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, tid, NT);
       }
     }
-
-    if (tail) fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(empty_bar(slot));
-  }
-
-  // ------------------------------------------------------------------ merge the four warps
-  l += __shfl_xor_sync(0xffffffffu, l, 1);
-  l += __shfl_xor_sync(0xffffffffu, l, 2);
-  consumer_bar();                                        // every tile has been consumed: the ring is free
-  float* wo = reinterpret_cast<float*>(ring_ptr);        // [NW][8][RV]
-  float* wm = wo + NW * 8 * RV;                          // [NW][8]
-  float* wl = wm + NW * 8;                               // [NW][8]
-#pragma unroll
-  for (int n = 0; n < RV / 8; ++n) {
-    *reinterpret_cast<float2*>(wo + (warp * 8 + gid) * RV + 8 * n + 2 * tid4) =
-        make_float2(o[n][0] + o[n][2], o[n][1] + o[n][3]);
-  }
-  if (tid4 == 0) {
-    wm[warp * 8 + gid] = m;
-    wl[warp * 8 + gid] = l;
-  }
-  consumer_bar();
-  for (int idx = tid; idx < 8 * RV; idx += NW * 32) {
-    const int gg = idx / RV, j = idx % RV;
-    const int gq = qt * 8 + gg;
-    if (gq >= G) break;
-    float M = wm[gg];
-#pragma unroll
-    for (int w = 1; w < NW; ++w) M = fmaxf(M, wm[w * 8 + gg]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const float e = exp2f(wm[w * 8 + gg] - M);
-      num += e * wo[(w * 8 + gg) * RV + j];
-      den += e * wl[w * 8 + gg];
-    }
-    const size_t row = ((size_t)b * a.L.Hq + (size_t)h * G + gq) * a.S + split;
-    a.partial_o[row * RV + j] = num / den;
-    if (j == 0) a.partial_lse[row] = (M + log2f(den)) * kLn2;
+    bar1(NT);
   }
 }
 

@@ -1,5 +1,5 @@
-// Instantiations of the split-T decode kernel for one key rank (STIEF_RK, given on the command line)
-// and every supported value rank.  Compiled once per key rank so the build parallelises.
+// Instantiations of the persistent decode kernel for one key rank (STIEF_RK, given on the command
+// line) and every supported value rank.  Compiled once per key rank so the build parallelises.
 #include "stief_decode.cuh"
 #include "stief_kernels.h"
 
@@ -12,7 +12,7 @@ namespace stief {
 template <int RK, int RV>
 static cudaError_t launch_one(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st) {
   using C = DecodeCfg<RK, RV>;
-  auto kern = decode_split_kernel<RK, RV>;
+  auto kern = decode_persistent_kernel<RK, RV>;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -21,18 +21,7 @@ static cudaError_t launch_one(const DecodeLaunch& a, const CUtensorMap& tmK, con
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  DecodeArgs k;
-  k.L = a.L;
-  k.Bt = a.Bt;
-  k.q_proj = a.q_proj;
-  k.partial_o = a.partial_o;
-  k.partial_lse = a.partial_lse;
-  k.S = a.S;
-  k.chunk_pages = a.chunk_pages;
-  k.len_add = a.len_add;
-  k.status = a.status;
-  dim3 grid(a.S, a.L.Hkv * ((a.L.G + 7) / 8), a.Bt.B);
-  kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tmK, tmV, k);
+  kern<<<a.n_cta, C::THREADS, C::SMEM_BYTES, st>>>(tmK, tmV, a.args);
   return cudaGetLastError();
 }
 
@@ -41,7 +30,7 @@ static cudaError_t launch_one(const DecodeLaunch& a, const CUtensorMap& tmK, con
 
 cudaError_t STIEF_CAT(launch_decode_rk, STIEF_RK)(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                                   cudaStream_t st) {
-  switch (a.L.r_v) {
+  switch (a.args.L.r_v) {
     case 32: return launch_one<STIEF_RK, 32>(a, tmK, tmV, st);
     case 48: return launch_one<STIEF_RK, 48>(a, tmK, tmV, st);
     case 64: return launch_one<STIEF_RK, 64>(a, tmK, tmV, st);

@@ -1,17 +1,15 @@
 // Internal interface between the C-ABI layer (stief_api.cu) and the kernel translation units.
 #pragma once
 
-#include "stief_common.cuh"
+#include "stief_decode_args.h"
 
 namespace stief {
 
-struct PreArgs {
+struct AppendArgs {
   LayerDev L;
   BatchDev Bt;
-  const __nv_bfloat16* q;       // [B][Hq][128] or NULL (append only)
-  const __nv_bfloat16* k_new;   // [B][Hkv][128] or NULL (query projection only)
+  const __nv_bfloat16* k_new;   // [B][Hkv][128]
   const __nv_bfloat16* v_new;
-  float* q_proj;                // [B][Hq][r_k]
   int32_t* status;
 };
 
@@ -20,7 +18,7 @@ struct CombineArgs {
   BatchDev Bt;
   const float* partial_o;
   const float* partial_lse;
-  int S, chunk_pages, len_add;
+  int n_cta, QT, len_add;
   __nv_bfloat16* out;           // [B][Hq][128]
   float* out_lse;               // [B][Hq] or NULL
 };
@@ -36,16 +34,11 @@ struct PrefillArgs {
 };
 
 struct DecodeLaunch {
-  LayerDev L;
-  BatchDev Bt;
-  const float* q_proj;
-  float* partial_o;
-  float* partial_lse;
-  int S, chunk_pages, len_add;
-  int32_t* status;
+  DecodeArgs args;
+  int n_cta;
 };
 
-cudaError_t launch_pre(const PreArgs& a, cudaStream_t st);
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
 cudaError_t launch_combine(const CombineArgs& a, cudaStream_t st);
 cudaError_t launch_advance(int32_t* seq_lens, int B, int delta, cudaStream_t st);
 cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st);

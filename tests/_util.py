@@ -124,9 +124,11 @@ def check_out(gpu_out: torch.Tensor, ref: np.ndarray, max_abs=1e-2, rel_l2=5e-3)
     return ea, rl
 
 
-def workspace_for(c: Case, num_splits: int) -> torch.Tensor:
-    n = S.stief_decode_workspace_bytes(c.B, c.Hq, c.r_k, c.r_v, max(num_splits, 1))
-    return torch.full((n // 4,), float("nan"), dtype=torch.float32, device="cuda")
+def workspace_for(c: Case, num_parts: int) -> torch.Tensor:
+    n = S.stief_decode_workspace_bytes(c.B, c.Hq, c.Hkv, c.r_v, num_parts)
+    ws = torch.full((n // 4,), float("nan"), dtype=torch.float32, device="cuda")
+    S.stief_decode_workspace_init(ws)          # the one-time clearing the library asks for
+    return ws
 
 
 def upload_cache(c: Case, Kd, Vd):

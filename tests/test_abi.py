@@ -32,21 +32,25 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings_and_version(lib):
-    assert S.stief_version() >= 100
+    assert S.stief_version() >= 200
     assert S.status_string(0) == "ok"
     assert "workspace" in S.status_string(S.STIEF_ERR_WORKSPACE)
     assert all(S.status_string(i) for i in range(8))
 
 
-def test_workspace_and_split_planning(lib):
-    # q_proj + partial_o + partial_lse, each section padded to 128 bytes
-    n = S.stief_decode_workspace_bytes(4, 32, 64, 64, 37)
-    assert n == 4 * 32 * 64 * 4 + 4 * 32 * 37 * 64 * 4 + ((4 * 32 * 37 * 4 + 127) // 128) * 128
-    assert S.stief_decode_workspace_bytes(0, 32, 64, 64, 1) == 0
-    s = S.stief_decode_num_splits(4, 8, 514)
-    assert 1 <= s <= 514
-    assert S.stief_decode_num_splits(1, 8, 1) == 1
-    assert S.stief_decode_num_splits(1000, 8, 64) >= 1
+def test_workspace_planning(lib):
+    # counters [n_units] int32 | partial_o [parts + n_units][8][r_v] fp32 | partial_lse [parts + n_units][8] fp32
+    up = lambda x: (x + 127) // 128 * 128
+    n_units = 4 * 8 * 1
+    n = S.stief_decode_workspace_bytes(4, 32, 8, 64, 148)
+    assert n == up(n_units * 4) + up((148 + n_units) * 8 * 64 * 4) + up((148 + n_units) * 8 * 4)
+    # a group of 16 query heads per KV head is two units per (sequence, KV head)
+    n_units = 2 * 2 * 2
+    assert S.stief_decode_workspace_bytes(2, 32, 2, 96, 10) == up(n_units * 4) + up((10 + n_units) * 8 * 96 * 4) + up((10 + n_units) * 8 * 4)
+    assert S.stief_decode_workspace_bytes(0, 32, 8, 64, 1) == 0
+    assert S.stief_decode_workspace_bytes(4, 30, 8, 64, 1) == 0          # Hq not a multiple of Hkv
+    assert S.stief_decode_num_parts() >= 1                                  # 148 when no device is present
+    assert S.stief_decode_workspace_bytes(4, 32, 8, 64, 0) == S.stief_decode_workspace_bytes(4, 32, 8, 64, S.stief_decode_num_parts())
     assert S.stief_host_staging_bytes(4, 32, 8) == 2 * 4 * 32 * 128 * 2 + 2 * 4 * 8 * 128 * 2
 
 

@@ -59,7 +59,7 @@ def _untouched_rows_still_nan(c: U.Case):
 
 
 def _decode(c: U.Case, num_splits, len_add=0, q=None):
-    ws = U.workspace_for(c, num_splits if num_splits else S.stief_decode_num_splits(c.B, c.Hkv, c.batch.block_table.shape[1]))
+    ws = U.workspace_for(c, num_splits)
     out = torch.full((c.B, c.Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
     lse = torch.full((c.B, c.Hq), float("nan"), dtype=torch.float32, device="cuda")
     S.stief_decode_attention(c.layer, c.batch, (c.q if q is None else q).cuda(), ws, num_splits, out, lse, len_add=len_add,
@@ -180,7 +180,7 @@ def test_append_and_decode_step_across_a_page_boundary():
         k_new, v_new = I.new_token_kv(40, 0, B, Hkv, step=step)
         q = I.queries(40, 0, B, Hq, step=step + 1)
         if step % 2 == 0:      # fused step
-            S.stief_decode_step(c.layer, c.batch, q.cuda(), k_new.cuda(), v_new.cuda(), ws, out, num_splits=4, status=c.status)
+            S.stief_decode_step(c.layer, c.batch, q.cuda(), k_new.cuda(), v_new.cuda(), ws, out, num_parts=4, status=c.status)
         else:                  # the same thing as separate calls
             S.stief_append(c.layer, c.batch, k_new.cuda(), v_new.cuda(), status=c.status)
             S.stief_decode_attention(c.layer, c.batch, q.cuda(), ws, 4, out, len_add=1, status=c.status)
@@ -241,10 +241,10 @@ def test_host_staged_step():
     out_h = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
     staging = torch.empty(S.stief_host_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device="cuda")
     ws = U.workspace_for(c, 2)
-    S.stief_decode_step_host(c.layer, c.batch, q, kh, vh, staging, ws, out_h, num_splits=2, status=c.status)
+    S.stief_decode_step_host(c.layer, c.batch, q, kh, vh, staging, ws, out_h, num_parts=2, status=c.status)
     assert _sync_status(c) == 0
     out_d = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device="cuda")
-    S.stief_decode_step(c.layer, c.batch, c.q.cuda(), k_new.cuda(), v_new.cuda(), ws, out_d, num_splits=2, status=c.status)
+    S.stief_decode_step(c.layer, c.batch, c.q.cuda(), k_new.cuda(), v_new.cuda(), ws, out_d, num_parts=2, status=c.status)
     assert _sync_status(c) == 0
     assert torch.equal(out_h, out_d.cpu())
 
