@@ -154,6 +154,31 @@ int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, c
 /* seq_lens[b] += delta on the device (so a captured step can be replayed). */
 int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream);
 
+/* stief_decode_attention for callers that cannot supply a workspace.  The paper has no counterpart:
+ * this exists for integration only.  Who needs it: code that runs as a plug-in inside an engine which
+ * has already claimed all device memory for its own pool and offers no allocator to plug-ins, and
+ * code on a latency-critical path where cudaMalloc is ruled out because it synchronises the whole
+ * device.  The split-T scratch (arrival counters and per-segment partials, same layout as the
+ * workspace above) is a fixed device array of STIEF_STATIC_WORKSPACE_BYTES inside the library; every
+ * GPU that loads the library holds that much memory until the process exits.  This entry point never
+ * calls cudaMalloc, cudaFree or any allocating routine.
+ *  - Same arguments and result as stief_decode_attention, without the workspace; `out` must not be NULL
+ *    (the partials are not reachable from outside).
+ *  - Limit: stief_decode_workspace_bytes(B, Hq, Hkv, r_v, num_parts) must not exceed
+ *    STIEF_STATIC_WORKSPACE_BYTES, else STIEF_ERR_WORKSPACE is returned and nothing is launched
+ *    (with one part per SM of a B200 and r_v = 128 that allows up to 359 (sequence, KV head) pairs
+ *    of groups of at most 8 query heads).
+ *  - The first call on each device looks up the array's device address (this loads the module if it
+ *    is not loaded yet); make that first call outside any stream capture, with the device current.
+ *  - All calls on a device share the one array and it keeps the previous call's contents.  Each call
+ *    clears the counters it relies on (a cudaMemsetAsync on `stream`) before its kernel.  Two calls
+ *    that overlap on the GPU -- different streams, or different host threads -- race on the array
+ *    and give wrong results: serialise them. */
+#define STIEF_STATIC_WORKSPACE_BYTES (2u << 20)
+int stief_decode_attention_static(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
+                                  int32_t len_add, int32_t num_parts, uint16_t* out, float* out_lse,
+                                  int32_t* status, void* stream);
+
 /* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
  * stief_decode_step_host call made by this host thread records `start_event` just before and
  * `stop_event` just after its decode kernel on the call's stream (both cudaEvent_t passed as void*),

@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
             "stief_decode_workspace_init": (ctypes.c_int, [P, SZ, P]),
             "stief_decode_attention": (ctypes.c_int, [LP, BP, P, I32, P, SZ, I32, P, P, P, P]),
             "stief_split_combine": (ctypes.c_int, [LP, BP, I32, P, I32, P, P, P, P]),
+            "stief_decode_attention_static": (ctypes.c_int, [LP, BP, P, I32, I32, P, P, P, P]),
             "stief_decode_step": (ctypes.c_int, [LP, BP, P, P, P, P, SZ, I32, P, P, P, P]),
             "stief_host_staging_bytes": (SZ, [I32, I32, I32]),
             "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, P, P]),
@@ -169,6 +170,23 @@ def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspac
     _check(lib().stief_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
                                         _ptr(status), _stream()), "stief_decode_attention")
+
+
+STATIC_WORKSPACE_BYTES = 2 << 20
+
+
+def stief_decode_attention_static(layer: Layer, batch: Batch, q: torch.Tensor, out: torch.Tensor, num_parts: int = 0,
+                                  out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
+                                  status: Optional[torch.Tensor] = None):
+    """stief_decode_attention without a workspace argument, for callers that have no means of allocating one
+    (a plug-in inside an engine that owns all device memory; a path where cudaMalloc's device-wide
+    synchronisation is not acceptable).  The scratch is a fixed STATIC_WORKSPACE_BYTES array inside the
+    library, shared by every call on the device: calls must not overlap on the GPU, and shapes whose
+    workspace would be larger raise StiefError(STIEF_ERR_WORKSPACE).  Make the first call on a device
+    outside any stream capture."""
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_decode_attention_static(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, num_parts, _ptr(out),
+                                               _ptr(out_lse), _ptr(status), _stream()), "stief_decode_attention_static")
 
 
 def stief_split_combine(layer: Layer, batch: Batch, workspace: torch.Tensor, num_parts: int, out: torch.Tensor,
