@@ -97,9 +97,10 @@ int stief_append(const stief_layer* layer, const stief_batch* batch, const uint1
 
 /* Split-T planning.  The page tiles of the whole batch (one tile = 64 tokens of one KV head) are laid
  * end to end -- units (sequence, KV head, tile of up to 8 query heads) in that order -- and cut into
- * num_parts contiguous ranges of equal size, one per CTA of a persistent kernel; a range cuts one
- * "segment" out of every unit it overlaps and each segment yields one chunk-normalised partial
- * result.  num_parts = 0 lets the library choose (one CTA per SM of the current device, which is also
+ * num_parts contiguous ranges of equal cost, one per CTA of a persistent kernel (cost = page tiles,
+ * plus a fixed charge for every unit a range enters, which stands for the work of starting a
+ * segment); a range cuts one "segment" out of every unit it overlaps and each segment yields one
+ * chunk-normalised partial result.  num_parts = 0 lets the library choose (one CTA per SM of the current device, which is also
  * what stief_decode_num_parts returns); it must not exceed 65535.  The same num_parts must be given
  * to stief_decode_workspace_bytes and to every call that shares the workspace.
  * Workspace layout, n_units = B * Hkv * ceil((Hq/Hkv) / 8):

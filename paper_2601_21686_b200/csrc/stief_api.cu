@@ -157,7 +157,8 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   if (num_parts < 0 || num_parts > 65535) return STIEF_ERR_INVALID_ARG;
   const int n_cta = resolve_parts(num_parts);
   const int QT = query_tiles(layer->Hq, layer->Hkv);
-  if ((long long)batch->B * batch->max_pages_per_seq * layer->Hkv * QT >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
+  if ((long long)batch->B * (batch->max_pages_per_seq + seg_pad_pages(layer->r_k, layer->r_v)) * layer->Hkv * QT >= (1ll << 31))
+    return STIEF_ERR_INVALID_ARG;
   const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
   if (w.bytes > workspace_bytes) return STIEF_ERR_WORKSPACE;
 

@@ -45,59 +45,79 @@ struct DecodeCfg {
   static constexpr int CTRL_BYTES = 512;                 // full[NS], empty[NS], append barrier, flags
   static constexpr int PREF_BYTES = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
   static constexpr int QP_BYTES = kGroupTile * kD * 4;   // q' fp32 [8][RK]
-  static constexpr int ROWS_BYTES = 9 * kD * 4;          // vectors to project: 8 queries + the new key (or value)
+  static constexpr int ROWS_BYTES = 10 * kD * 4;         // vectors to project: 8 queries, the new key, the new value
   static constexpr int RED_BYTES = NW * 9 * kD * 4;      // per-warp partial projections
   static constexpr int UNION_BYTES = ROWS_BYTES + RED_BYTES;   // also: merge scratch [NW][8][RV]+[2][NW][8]; combine scratch [8][128]
   static constexpr int SMEM_BYTES = 1024 + RING_BYTES + CTRL_BYTES + PREF_BYTES + QP_BYTES + UNION_BYTES;
   static_assert(RK % 16 == 0 && RV % 16 == 0 && RK <= 128 && RV <= 128, "ranks are multiples of 16 up to 128");
   static_assert(SPW >= 1 && NS <= 16, "ring shape");
   static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= UNION_BYTES, "merge scratch must fit");
+  static_assert(kCombineScratchFloats * 4 <= UNION_BYTES && NT >= 96, "combine scratch must fit; combine_unit wants >= 96 threads");
   static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KiB shared memory of an SM");
 };
 
-// sums[r][j] = sum_d rows[r][d] * U[d][j] for r < 9, j < R, by NW warps (warp w contracts d = w, w+NW, ...).
-// rows: shared fp32 [9][128]; red: shared fp32 [NW][9][128]; result left in red[0][r][j].
-template <int NW>
-__device__ __forceinline__ void cta_project(const float* rows, const __nv_bfloat16* __restrict__ U, int R, float* red, int warp, int lane) {
-  for (int cp = lane; cp < R / 2; cp += 32) {
-    float acc[9][2];
+// Projection of a few rows onto a basis, X U with X fp32 [rows][128] in shared memory and U bf16
+// [128][R] in global memory, by NW warps.  Warp w contracts the d-range [w*DPW, (w+1)*DPW); lane l owns
+// the column pairs l and l+32.  The kernel runs while the whole GPU streams the cache, so a dependent
+// global load costs microseconds: a thread therefore fetches its whole slice of U into registers with
+// independent loads (one round trip) before any arithmetic.
+template <int NW, int R>
+struct BasisSlice {
+  static constexpr int DPW = ((kD + NW - 1) / NW + 3) / 4 * 4;   // d values per warp (multiple of 4)
+  static constexpr int NP = (R / 2 + 31) / 32;                   // column-pair passes per lane
+  uint32_t u[NP][DPW];
+
+  __device__ __forceinline__ void load(const __nv_bfloat16* __restrict__ U, int warp, int lane) {
 #pragma unroll
-    for (int r = 0; r < 9; ++r) acc[r][0] = acc[r][1] = 0.f;
-    constexpr int ND = (kD + NW - 1) / NW;                // d values per warp
-#pragma unroll 1
-    for (int i0 = 0; i0 < ND; i0 += 8) {
-      uint32_t u[8];
+    for (int p = 0; p < NP; ++p) {
+      const int cp = lane + 32 * p;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int d = warp + (i0 + i) * NW;
-        u[i] = (d < kD) ? __ldg(reinterpret_cast<const uint32_t*>(U + (size_t)d * R + 2 * cp)) : 0u;
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int d = warp + (i0 + i) * NW;
-        if (d < kD) {
-          const float u0 = bf16_lo(u[i]), u1 = bf16_hi(u[i]);
-#pragma unroll
-          for (int r = 0; r < 9; ++r) {
-            const float x = rows[r * kD + d];
-            acc[r][0] = fmaf(x, u0, acc[r][0]);
-            acc[r][1] = fmaf(x, u1, acc[r][1]);
-          }
-        }
+      for (int i = 0; i < DPW; ++i) {
+        const int d = warp * DPW + i;
+        u[p][i] = (cp < R / 2 && d < kD) ? __ldg(reinterpret_cast<const uint32_t*>(U + (size_t)d * R + 2 * cp)) : 0u;
       }
     }
-#pragma unroll
-    for (int r = 0; r < 9; ++r) *reinterpret_cast<float2*>(red + (warp * 9 + r) * kD + 2 * cp) = make_float2(acc[r][0], acc[r][1]);
   }
-  bar1(NW * 32);
-  for (int idx = warp * 32 + lane; idx < 9 * R; idx += NW * 32) {
-    const int r = idx / R, j = idx % R;
-    float s = 0.f;
+
+  // red[(warp*9 + r)*128 + j] = this warp's share of sum_d rows[r][d] U[d][j], for the rows whose bit is
+  // set in row_mask (bit r <-> row r, r < 9)
+  __device__ __forceinline__ void contract(const float* rows, uint32_t row_mask, float* red, int warp, int lane) const {
 #pragma unroll
-    for (int w = 0; w < NW; ++w) s += red[(w * 9 + r) * kD + j];
-    red[r * kD + j] = s;                                  // slot of warp 0; only this thread touches (r, j)
+    for (int r = 0; r < 9; ++r) {
+      if (!((row_mask >> r) & 1u)) continue;               // uniform over the CTA
+      float acc[NP][2];
+#pragma unroll
+      for (int p = 0; p < NP; ++p) acc[p][0] = acc[p][1] = 0.f;
+#pragma unroll
+      for (int i = 0; i < DPW; i += 4) {
+        const int d = warp * DPW + i;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (d < kD) x = *reinterpret_cast<const float4*>(rows + r * kD + d);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+          for (int p = 0; p < NP; ++p) {
+            acc[p][0] = fmaf(xs[e], bf16_lo(u[p][i + e]), acc[p][0]);
+            acc[p][1] = fmaf(xs[e], bf16_hi(u[p][i + e]), acc[p][1]);
+          }
+      }
+#pragma unroll
+      for (int p = 0; p < NP; ++p) {
+        const int cp = lane + 32 * p;
+        if (cp < R / 2) *reinterpret_cast<float2*>(red + (warp * 9 + r) * kD + 2 * cp) = make_float2(acc[p][0], acc[p][1]);
+      }
+    }
   }
-  bar1(NW * 32);
+};
+
+// sum over the warps' shares of (row r, column j)
+template <int NW>
+__device__ __forceinline__ float warp_shares(const float* red, int r, int j) {
+  float s = 0.f;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) s += red[(w * 9 + r) * kD + j];
+  return s;
 }
 
 template <int RK, int RV>
@@ -135,7 +155,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     *last_flag = 0;
     mbar_fence_init();
   }
-  build_page_prefix(pref, a.Bt, a.len_add, c == 0 ? a.status : nullptr);   // ends with __syncthreads
+  const int pad = seg_pad_pages(RK, RV);
+  build_page_prefix(pref, a.Bt, a.len_add, pad, c == 0 ? a.status : nullptr);   // ends with __syncthreads
 
   const int B = a.Bt.B, Hkv = a.L.Hkv, QT = a.QT, G = a.L.G;
   const int upb = Hkv * QT;
@@ -144,7 +165,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const bool appending = a.k_new != nullptr;
 
   SegmentWalker walk;
-  walk.init(pref, B, upb, c, P, total);
+  walk.init(pref, B, upb, pad, c, P, total);
   Segment seg;
 
   // ------------------------------------------------------------------ producer warp
@@ -255,42 +276,68 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       }
     }
 
-    // ---- vectors contracted with U_k: the unit's queries (rows 0..7) and the new key (row 8)
-    float* rows = un;
-    float* red = un + 9 * kD;
-    for (int idx = tid; idx < 9 * kD; idx += NT) {
-      const int r = idx / kD, d = idx % kD;
-      float x = 0.f;
-      if (r < ng) x = __bfloat162float(a.q[(head0 + r) * kD + d]);
-      else if (r == 8 && do_append) x = __bfloat162float(a.k_new[((size_t)b * Hkv + h) * kD + d]);
-      rows[idx] = x;
-    }
-    bar1(NT);
+    // ---- prologue: q' = q U_k for the unit's queries (rows 0..7), the new key's row k U_k (row 8) and the
+    // new value's row v U_v.  All global loads are issued before the first use of any of them.
+    float* rows = un;                    // [9][128] fp32
+    float* vrow = un + 9 * kD;           // [128]
+    float* red = un + 10 * kD;           // [NW][9][128]
     const __nv_bfloat16* Uk = a.L.U_k ? a.L.U_k + (size_t)h * a.L.uk_stride : nullptr;
-    const float* res = rows;
-    if (Uk) {
-      cta_project<NW>(rows, Uk, RK, red, warp, lane);
-      res = red;
+    const __nv_bfloat16* Uv = a.L.U_v ? a.L.U_v + (size_t)h * a.L.uv_stride : nullptr;
+    const uint32_t row_mask = ((1u << ng) - 1u) | (do_append ? 0x100u : 0u);
+    {
+      BasisSlice<NW, RK> sk;
+      if (Uk) sk.load(Uk, warp, lane);
+      // rows as 16-byte pieces: piece idx -> row idx / 16, elements 8 * (idx % 16) ..
+      constexpr int NPC = (9 * 16 + NT - 1) / NT;
+      uint4 pc[NPC];
+#pragma unroll
+      for (int i = 0; i < NPC; ++i) {
+        const int idx = tid + i * NT, r = idx / 16, c = idx % 16;
+        pc[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < ng) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (head0 + r) * kD) + c);
+        else if (r == 8 && do_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * kD) + c);
+      }
+      uint4 pv = make_uint4(0u, 0u, 0u, 0u);
+      if (do_append && tid < 16) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * kD) + tid);
+#pragma unroll
+      for (int i = 0; i < NPC; ++i) {
+        const int idx = tid + i * NT;
+        if (idx < 9 * 16) {
+          const uint32_t w[4] = {pc[i].x, pc[i].y, pc[i].z, pc[i].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(rows + idx * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
+        }
+      }
+      if (do_append && tid < 16) {
+        const uint32_t w[4] = {pv.x, pv.y, pv.z, pv.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(vrow + tid * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
+      }
+      bar1(NT);
+      if (Uk) sk.contract(rows, row_mask, red, warp, lane);
     }
+    BasisSlice<NW, RV> sv;
+    if (do_append && Uv) sv.load(Uv, warp, lane);          // in flight while the key side is reduced
+    bar1(NT);
     for (int idx = tid; idx < 9 * RK; idx += NT) {
       const int r = idx / RK, j = idx % RK;
-      const float x = res[r * kD + j];
+      if (!((row_mask >> r) & 1u)) {
+        if (r < 8) qp[r * RK + j] = 0.f;
+        continue;
+      }
+      const float x = Uk ? warp_shares<NW>(red, r, j) : rows[r * kD + j];
       if (r < 8) qp[r * RK + j] = x * qscale;
-      else if (do_append && new_row != ~(size_t)0) a.L.k_pool[new_row * RK + j] = __float2bfloat16_rn(x);
+      else if (new_row != ~(size_t)0) a.L.k_pool[new_row * RK + j] = __float2bfloat16_rn(x);
     }
     if (do_append) {
-      bar1(NT);
-      for (int idx = tid; idx < 9 * kD; idx += NT)
-        rows[idx] = idx < kD ? __bfloat162float(a.v_new[((size_t)b * Hkv + h) * kD + idx]) : 0.f;
-      bar1(NT);
-      const __nv_bfloat16* Uv = a.L.U_v ? a.L.U_v + (size_t)h * a.L.uv_stride : nullptr;
-      res = rows;
+      bar1(NT);                                            // the key side has left `red`
       if (Uv) {
-        cta_project<NW>(rows, Uv, RV, red, warp, lane);
-        res = red;
+        // the value row sits where row 0 is expected: contract one row
+        sv.contract(vrow, 1u, red, warp, lane);
+        bar1(NT);
       }
       if (new_row != ~(size_t)0) {
-        for (int j = tid; j < RV; j += NT) a.L.v_pool[new_row * RV + j] = __float2bfloat16_rn(res[j]);
+        for (int j = tid; j < RV; j += NT) a.L.v_pool[new_row * RV + j] = __float2bfloat16_rn(Uv ? warp_shares<NW>(red, 0, j) : vrow[j]);
       } else if (tid == 0) {
         report(a.status, STIEF_ERR_BOUNDS);
       }
@@ -440,7 +487,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     // ------------------------------------------------------------------ the unit's last partial triggers the combine
     if (a.out != nullptr) {
       int first, last;
-      unit_cta_span(pref, upb, P, b, seg.j, &first, &last);
+      unit_cta_span(pref, upb, pad, P, b, seg.j, &first, &last);
       const int nseg = last - first + 1;
       __threadfence();
       bar1(NT);
@@ -456,7 +503,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       bar1(NT);
       if (*last_flag) {
         __threadfence();
-        combine_unit(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, tid, NT);
+        combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, un + kGroupTile * kD, tid, NT);
       }
     }
     bar1(NT);

@@ -80,20 +80,29 @@ constexpr int kCombThreads = 128;
 __global__ void __launch_bounds__(kCombThreads)
 combine_kernel(const CombineArgs a) {
   __shared__ int pref[kMaxBatch + 1];
-  __shared__ float od[kGroupTile * kD];
+  __shared__ __align__(16) float od[kCombineScratchFloats];
   const int j = blockIdx.x, b = blockIdx.y;
   const int upb = a.L.Hkv * a.QT;
-  build_page_prefix(pref, a.Bt, a.len_add, nullptr);
+  const int pad = seg_pad_pages(a.L.r_k, a.L.r_v);
+  build_page_prefix(pref, a.Bt, a.len_add, pad, nullptr);
   const int total = pref[a.Bt.B] * upb;
   const int P = pages_per_cta(total, a.n_cta);
   const int h = j / a.QT, qt = j % a.QT;
   int first = 0, nseg = 0;
   if (pref[b + 1] != pref[b]) {
     int last;
-    unit_cta_span(pref, upb, P, b, j, &first, &last);
+    unit_cta_span(pref, upb, pad, P, b, j, &first, &last);
     nseg = last - first + 1;
   }
-  combine_unit(a.L, b, h, qt, first + b * upb + j, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads);
+  const int slot0 = first + b * upb + j;
+  switch (a.L.r_v) {
+    case 32: combine_unit<32>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    case 48: combine_unit<48>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    case 64: combine_unit<64>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    case 96: combine_unit<96>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    case 128: combine_unit<128>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    default: break;
+  }
 }
 
 __global__ void advance_kernel(int32_t* seq_lens, int B, int delta) {
