@@ -175,9 +175,13 @@ def run_ours(args):
     qs = [I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for i in range(n_in)]
     kvs = [I.new_token_kv(SEED, 0, B, Hkv, device=dev, step=i) for i in range(n_in)]
 
-    def step(i):
+    # Consecutive steps work on different layer caches and their inputs are resident before the loop, which
+    # is what STIEF_DECODE_OVERLAP_PREVIOUS asks for: each launch may take over SMs as the previous one drains.
+    overlap = S.STIEF_DECODE_OVERLAP_PREVIOUS if (args.overlap and n_caches >= 2) else 0
+
+    def step(i, flags=overlap):
         S.stief_decode_step(layers[i % n_caches], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
-                            num_parts=ns, status=status)
+                            num_parts=ns, status=status, flags=flags)
 
     def barrier():
         if world > 1:
@@ -205,6 +209,16 @@ def run_ours(args):
     t1 = time.time()
     ms = e0.elapsed_time(e1)
 
+    # ---- the same loop with plainly serialised launches
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    s0.record()
+    for i in range(K_steps):
+        step(W + i, 0)
+    s1.record()
+    barrier()
+    ms_serial = s0.elapsed_time(s1)
+
     # ---- timed region 2: the split-T kernel alone, per launch (events recorded inside the library call)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
     for a, b in evs:
@@ -212,7 +226,7 @@ def run_ours(args):
     barrier()
     for i in range(K_steps):
         S.stief_time_next_decode_kernel(*evs[i])
-        step(W + i)
+        step(W + i, 0)
     barrier()
     kern_ms = [a.elapsed_time(b) for a, b in evs]
 
@@ -224,7 +238,7 @@ def run_ours(args):
 
     def step_host(i):
         S.stief_decode_step_host(layers[i % n_caches], batch, qh[i % n_in], kh[i % n_in][0], kh[i % n_in][1], staging, ws,
-                                 out_h, num_parts=ns, status=status)
+                                 out_h, num_parts=ns, status=status, flags=0)
         torch.cuda.current_stream().synchronize()       # the caller reads out_h after every step
 
     for i in range(W):
@@ -242,10 +256,11 @@ def run_ours(args):
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
     # ---- max over ranks
-    times = torch.tensor([ms, ms_host, float(np.mean(kern_ms))], dtype=torch.float64, device=dev)
+    times = torch.tensor([ms, ms_host, float(np.mean(kern_ms)), ms_serial], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, ms_host, kern_avg_ms = (float(x) for x in times.tolist())
+    ms, ms_host, kern_isolated_ms, ms_serial = (float(x) for x in times.tolist())
+    kern_avg_ms = ms / K_steps          # one launch per step: the timed region divided by its launches
 
     if rank == 0:
         hbm_peak, tf_peak, peak_kind = measured_peaks()
@@ -263,6 +278,8 @@ def run_ours(args):
             "config": {"workload": "config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64, "
                                    "64-token pages, shuffled block tables; step = append + query projection + split-T attention + combine, one launch",
                        "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_parts": ns,
+                       "launch": ("programmatic dependent launch: each step's kernel may start while the previous step's drains"
+                                  if overlap else "serialised launches"),
                        "l2": f"steps rotate over {n_caches} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
                        "parallelism": f"replicas x{world} (independent batches, no collective)"},
             "tokens_per_s": world * B * K_steps / (ms * 1e-3),
@@ -274,7 +291,12 @@ def run_ours(args):
             "gpu_launches": K_steps,
             "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel<64,64>", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": peak_kind, "traffic": args.traffic,
-                         "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms, "min_launch_ms": float(min(kern_ms))},
+                         "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms,
+                         "isolated_launch_ms": kern_isolated_ms, "isolated_min_launch_ms": float(min(kern_ms)),
+                         "isolated_frac": sb / (kern_isolated_ms * 1e-3) / 1e9 / hbm_peak},
+            "serial_launches": {"value": world * sb * K_steps / (ms_serial * 1e-3) / 1e9, "unit": UNIT,
+                                "ms_per_step": ms_serial / K_steps,
+                                "frac_of_hbm_peak": sb * K_steps / (ms_serial * 1e-3) / 1e9 / hbm_peak},
             "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak,
                         "tflops": pf_flops / (pf_ms * 1e-3) / 1e12, "frac_of_bf16_peak": pf_flops / (pf_ms * 1e-3) / 1e12 / tf_peak,
                         "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache, one layer"},
@@ -386,6 +408,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--num-parts", type=int, default=0, help="CTAs of the persistent decode kernel (0 = one per SM)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", dest="overlap", action="store_false",
+                    help="launch every step's kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()

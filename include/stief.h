@@ -114,6 +114,19 @@ int32_t stief_decode_num_parts(void);
 size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t r_v, int32_t num_parts);
 int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
+/* Flags of the decode calls.
+ * STIEF_DECODE_OVERLAP_PREVIOUS: the kernel may start before the kernel that precedes it on the stream
+ * has finished (programmatic dependent launch): it takes over each SM as the earlier kernel's work there
+ * ends, reads its inputs, appends this step's rows and streams the cache, and only then waits for the
+ * earlier kernel to complete before it first touches `workspace`, `out` and `out_lse`.  Back-to-back
+ * decode kernels (the layers of one step) then run without an idle gap between them.  By setting the
+ * flag the caller promises that the preceding kernel on the stream writes none of this call's inputs
+ * (q, k_new, v_new, seq_lens, block_table, the bases, this layer's pools) and does not read the cache
+ * rows this call appends.  Two consecutive decode calls of this library on different layers satisfy
+ * that; a call that follows stief_advance_seq_lens, or whose q is produced by the preceding kernel,
+ * does not.  If the preceding stream operation is not a kernel the flag has no effect. */
+#define STIEF_DECODE_OVERLAP_PREVIOUS 1u
+
 /* Decode attention (Eq. 18 on the reconstructions of Eq. 7, one query row per head): q [B][Hq][128]
  * bf16 attends to tokens [0, seq_lens[b] + len_add) of every sequence; len_add is 0, or 1 when the
  * token of this step was appended on the same stream and seq_lens not yet advanced.  One kernel
@@ -124,7 +137,7 @@ int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* s
  * yields a zero row and lse = -inf.  With out == NULL only the partials are written. */
 int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
                            int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
-                           uint16_t* out, float* out_lse, int32_t* status, void* stream);
+                           uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
 
 /* Merge of the per-segment results by log-sum-exp (an exact re-association of Eq. 18) followed by the
  * back-projection o = o_down U_v^T (Eq. 7 applied to the mixed values; linear, so done once after the
@@ -140,7 +153,7 @@ int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int3
 int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
                       const uint16_t* k_new, const uint16_t* v_new, void* workspace,
                       size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
-                      int32_t* status, void* stream);
+                      uint32_t flags, int32_t* status, void* stream);
 
 /* The same step for callers whose activations live in host memory: q_host, k_new_host, v_new_host
  * are copied to `staging` (device, stief_host_staging_bytes) with cudaMemcpyAsync on `stream`, the
@@ -150,7 +163,7 @@ size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
                            const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging,
                            void* workspace, size_t workspace_bytes, int32_t num_parts,
-                           uint16_t* out_host, int32_t* status, void* stream);
+                           uint16_t* out_host, uint32_t flags, int32_t* status, void* stream);
 
 /* seq_lens[b] += delta on the device (so a captured step can be replayed). */
 int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* stream);

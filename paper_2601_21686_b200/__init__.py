@@ -21,6 +21,7 @@ STIEF_OK, STIEF_ERR_INVALID_ARG, STIEF_ERR_UNSUPPORTED, STIEF_ERR_WORKSPACE = 0,
 STIEF_ERR_CUDA, STIEF_ERR_BOUNDS, STIEF_ERR_TIMEOUT = 4, 5, 6
 PAGE = 64
 D_HEAD = 128
+STIEF_DECODE_OVERLAP_PREVIOUS = 1
 
 
 class StiefError(RuntimeError):
@@ -53,7 +54,7 @@ def lib() -> ctypes.CDLL:
             raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_21686_b200.build` "
                                "(there is no non-CUDA path)")
         L = ctypes.CDLL(LIB_PATH)
-        P, I32, I64, SZ = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        P, I32, I64, SZ, U32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32
         LP, BP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch)
         sig = {
             "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, P, P]),
@@ -61,12 +62,12 @@ def lib() -> ctypes.CDLL:
             "stief_decode_num_parts": (I32, []),
             "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
             "stief_decode_workspace_init": (ctypes.c_int, [P, SZ, P]),
-            "stief_decode_attention": (ctypes.c_int, [LP, BP, P, I32, P, SZ, I32, P, P, P, P]),
+            "stief_decode_attention": (ctypes.c_int, [LP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
             "stief_split_combine": (ctypes.c_int, [LP, BP, I32, P, I32, P, P, P, P]),
             "stief_decode_attention_static": (ctypes.c_int, [LP, BP, P, I32, I32, P, P, P, P]),
-            "stief_decode_step": (ctypes.c_int, [LP, BP, P, P, P, P, SZ, I32, P, P, P, P]),
+            "stief_decode_step": (ctypes.c_int, [LP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
             "stief_host_staging_bytes": (SZ, [I32, I32, I32]),
-            "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, P, P]),
+            "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, U32, P, P]),
             "stief_advance_seq_lens": (ctypes.c_int, [P, I32, I32, P]),
             "stief_time_next_decode_kernel": (ctypes.c_int, [P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -165,11 +166,11 @@ def stief_decode_workspace_init(workspace: torch.Tensor):
 
 def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, num_parts: int = 0,
                            out: Optional[torch.Tensor] = None, out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
-                           status: Optional[torch.Tensor] = None):
+                           status: Optional[torch.Tensor] = None, flags: int = 0):
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
-                                        _ptr(status), _stream()), "stief_decode_attention")
+                                        flags, _ptr(status), _stream()), "stief_decode_attention")
 
 
 STATIC_WORKSPACE_BYTES = 2 << 20
@@ -198,11 +199,11 @@ def stief_split_combine(layer: Layer, batch: Batch, workspace: torch.Tensor, num
 
 def stief_decode_step(layer: Layer, batch: Batch, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                       workspace: torch.Tensor, out: torch.Tensor, num_parts: int = 0, out_lse: Optional[torch.Tensor] = None,
-                      status: Optional[torch.Tensor] = None):
+                      status: Optional[torch.Tensor] = None, flags: int = 0):
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_step(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
-                                   _ptr(status), _stream()), "stief_decode_step")
+                                   flags, _ptr(status), _stream()), "stief_decode_step")
 
 
 def stief_host_staging_bytes(B: int, Hq: int, Hkv: int) -> int:
@@ -211,13 +212,13 @@ def stief_host_staging_bytes(B: int, Hq: int, Hkv: int) -> int:
 
 def stief_decode_step_host(layer: Layer, batch: Batch, q_host: torch.Tensor, k_new_host: torch.Tensor, v_new_host: torch.Tensor,
                            staging: torch.Tensor, workspace: torch.Tensor, out_host: torch.Tensor, num_parts: int = 0,
-                           status: Optional[torch.Tensor] = None):
+                           status: Optional[torch.Tensor] = None, flags: int = 0):
     """Host (pinned) q/k/v/out buffers; copies and kernels are enqueued, nothing is synchronised."""
     assert not q_host.is_cuda and not out_host.is_cuda
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_decode_step_host(ctypes.byref(cl), ctypes.byref(cb), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
                                         _ptr(staging), _ptr(workspace), workspace.numel() * workspace.element_size(),
-                                        num_parts, _ptr(out_host), _ptr(status), _stream()), "stief_decode_step_host")
+                                        num_parts, _ptr(out_host), flags, _ptr(status), _stream()), "stief_decode_step_host")
 
 
 def stief_advance_seq_lens(seq_lens: torch.Tensor, delta: int = 1):

@@ -144,7 +144,8 @@ thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 
 int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
                const uint16_t* v_new, int len_add, void* workspace, size_t workspace_bytes, int num_parts, uint16_t* out,
-               float* out_lse, int32_t* status, cudaStream_t st) {
+               float* out_lse, uint32_t flags, int32_t* status, cudaStream_t st) {
+  if (flags & ~STIEF_DECODE_OVERLAP_PREVIOUS) return STIEF_ERR_INVALID_ARG;
   int rc = check_layer(layer);
   if (rc) return rc;
   rc = check_batch(batch);
@@ -169,6 +170,7 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
 
   DecodeLaunch dl;
   dl.n_cta = n_cta;
+  dl.overlap_previous = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0;
   DecodeArgs& a = dl.args;
   a.L = to_dev(layer);
   a.Bt = to_dev(batch);
@@ -244,9 +246,9 @@ int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* s
 
 int stief_decode_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int32_t len_add,
                            void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
-                           int32_t* status, void* stream) {
-  return run_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_parts, out, out_lse, status,
-                    static_cast<cudaStream_t>(stream));
+                           uint32_t flags, int32_t* status, void* stream) {
+  return run_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_parts, out, out_lse, flags,
+                    status, static_cast<cudaStream_t>(stream));
 }
 
 int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int32_t len_add, const void* workspace,
@@ -272,9 +274,9 @@ int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int3
 
 int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
                       const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out,
-                      float* out_lse, int32_t* status, void* stream) {
+                      float* out_lse, uint32_t flags, int32_t* status, void* stream) {
   if (!k_new || !v_new || !out) return STIEF_ERR_INVALID_ARG;
-  return run_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_parts, out, out_lse, status,
+  return run_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_parts, out, out_lse, flags, status,
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -286,7 +288,8 @@ size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv) {
 
 int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
                            const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging, void* workspace,
-                           size_t workspace_bytes, int32_t num_parts, uint16_t* out_host, int32_t* status, void* stream) {
+                           size_t workspace_bytes, int32_t num_parts, uint16_t* out_host, uint32_t flags, int32_t* status,
+                           void* stream) {
   if (!layer || !batch || !q_host || !k_new_host || !v_new_host || !staging || !out_host || !aligned(staging, 128))
     return STIEF_ERR_INVALID_ARG;
   if (batch->B <= 0 || layer->Hq <= 0 || layer->Hkv <= 0) return STIEF_ERR_INVALID_ARG;
@@ -300,7 +303,7 @@ int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, c
   if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
   if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
   if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STIEF_ERR_CUDA;
-  const int rc = stief_decode_step(layer, batch, dq, dk, dv, workspace, workspace_bytes, num_parts, dout, nullptr, status, stream);
+  const int rc = stief_decode_step(layer, batch, dq, dk, dv, workspace, workspace_bytes, num_parts, dout, nullptr, flags, status, stream);
   if (rc) return rc;
   if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return STIEF_ERR_CUDA;
   return STIEF_OK;

@@ -68,6 +68,13 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   report(status, STIEF_ERR_TIMEOUT);
 }
 
+// Programmatic dependent launch.  launch_dependents lets the next kernel on the stream (if it was
+// launched with programmatic stream serialization) start as soon as every CTA of this grid has passed
+// this point or exited; grid_dependency_wait blocks until the grids this one depends on have completed
+// and their writes are visible (a no-op for a normally launched kernel).
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }

@@ -145,6 +145,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
 
+  // The next kernel on the stream may take over each SM as soon as this grid's CTA leaves it.
+  launch_dependents();
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(full_bar(s), 1);
@@ -224,19 +226,6 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   // ------------------------------------------------------------------ consumer warps
   const int gid = lane >> 2, tid4 = lane & 3, l7 = lane & 7;
   const float qscale = kLog2e * 0.08838834764831845f;     // log2(e) / sqrt(128)
-
-  // units of empty sequences get their zero rows from CTA (u mod n_cta)
-  if (a.out != nullptr) {
-    for (int u = c; u < B * upb; u += n_cta) {
-      const int b = u / upb, j = u % upb;
-      if (pref[b + 1] != pref[b]) continue;
-      const int h = j / QT, qt = j % QT;
-      const int ng = min(kGroupTile, G - qt * kGroupTile);
-      const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
-      for (int idx = tid; idx < ng * kD; idx += NT) a.out[head0 * kD + idx] = __float2bfloat16_rn(0.f);
-      if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
-    }
-  }
 
   // per-lane pieces of the ldmatrix addresses (the swizzle term depends on the lane only)
   constexpr int NCH = RK / 8;
@@ -468,6 +457,9 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     bar1(NT);
     const int u = b * upb + seg.j;
     const int slot_id = c + u;
+    // Everything up to here only read inputs (and appended this step's rows); the workspace and the
+    // outputs may still be in use by the kernel before this one when the launch overlaps it.
+    grid_dependency_wait();
     for (int idx = tid; idx < ng * RV; idx += NT) {
       const int gg = idx / RV, j = idx % RV;
       float M = wm[gg];
@@ -507,6 +499,20 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       }
     }
     bar1(NT);
+  }
+
+  // units of empty sequences get their zero rows from CTA (u mod n_cta)
+  if (a.out != nullptr) {
+    grid_dependency_wait();
+    for (int u = c; u < B * upb; u += n_cta) {
+      const int b = u / upb, j = u % upb;
+      if (pref[b + 1] != pref[b]) continue;
+      const int h = j / QT, qt = j % QT;
+      const int ng = min(kGroupTile, G - qt * kGroupTile);
+      const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
+      for (int idx = tid; idx < ng * kD; idx += NT) a.out[head0 * kD + idx] = __float2bfloat16_rn(0.f);
+      if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
+    }
   }
 }
 

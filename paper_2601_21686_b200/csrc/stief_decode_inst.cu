@@ -21,8 +21,17 @@ static cudaError_t launch_one(const DecodeLaunch& a, const CUtensorMap& tmK, con
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  kern<<<a.n_cta, C::THREADS, C::SMEM_BYTES, st>>>(tmK, tmV, a.args);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.n_cta);
+  cfg.blockDim = dim3(C::THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.overlap_previous ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, tmK, tmV, a.args);
 }
 
 #define STIEF_CAT_(a, b) a##b

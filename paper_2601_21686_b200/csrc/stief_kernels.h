@@ -36,6 +36,7 @@ struct PrefillArgs {
 struct DecodeLaunch {
   DecodeArgs args;
   int n_cta;
+  bool overlap_previous;        // launch with programmatic stream serialization
 };
 
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);

@@ -57,5 +57,5 @@ extern "C" int stief_decode_attention_static(const stief_layer* layer, const sti
   const size_t counter_bytes = ((size_t)batch->B * layer->Hkv * groups * 4 + 127) / 128 * 128;
   if (cudaMemsetAsync(ws, 0, counter_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return STIEF_ERR_CUDA;
   return stief_decode_attention(layer, batch, q, len_add, ws, (size_t)STIEF_STATIC_WORKSPACE_BYTES, num_parts, out, out_lse,
-                                status, stream);
+                                0u, status, stream);
 }

@@ -57,7 +57,7 @@ def test_workspace_planning(lib):
 def test_host_side_argument_checks_need_no_gpu(lib):
     # NULL descriptors are rejected before anything touches CUDA
     assert lib.stief_append(None, None, None, None, None, None) == S.STIEF_ERR_INVALID_ARG
-    assert lib.stief_decode_attention(None, None, None, 0, None, 0, 0, None, None, None, None) == S.STIEF_ERR_INVALID_ARG
+    assert lib.stief_decode_attention(None, None, None, 0, None, 0, 0, None, None, 0, None, None) == S.STIEF_ERR_INVALID_ARG
     assert lib.stief_advance_seq_lens(None, 4, 1, None) == S.STIEF_ERR_INVALID_ARG
 
 

@@ -231,6 +231,47 @@ def test_separate_combine_call_matches_fused_call():
     assert torch.equal(out1, out2)
 
 
+def test_overlapped_launches_match_serial_ones():
+    # decode steps of two layers enqueued back to back with STIEF_DECODE_OVERLAP_PREVIOUS, all sharing ONE
+    # workspace: every kernel may start while its predecessor still runs, but must not touch the workspace
+    # or its output before the predecessor is done.  Results must equal the serially launched ones bit for bit.
+    B, Hq, Hkv = 3, 8, 2
+    cs = [U.make_case(90, B, Hq, Hkv, 64, 64, [900, 300, 1500], reserve=8),
+          U.make_case(91, B, Hq, Hkv, 64, 64, [900, 300, 1500], reserve=8)]
+    for c in cs:
+        _prefill_and_check(c)
+    ws = U.workspace_for(cs[0], 0)
+    n_steps = 8
+    qs = [I.queries(90, 0, B, Hq, step=i).cuda() for i in range(n_steps)]
+    kvs = [tuple(t.cuda() for t in I.new_token_kv(90, 0, B, Hkv, step=i)) for i in range(n_steps)]
+    pools0 = [(c.layer.k_pool.clone(), c.layer.v_pool.clone()) for c in cs]
+    res = {}
+    for flags in (0, S.STIEF_DECODE_OVERLAP_PREVIOUS):
+        for c, (kp, vp) in zip(cs, pools0):
+            c.layer.k_pool.copy_(kp)
+            c.layer.v_pool.copy_(vp)
+        torch.cuda.synchronize()
+        outs = [torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(n_steps)]
+        for i in range(n_steps):
+            c = cs[i % 2]
+            S.stief_decode_step(c.layer, c.batch, qs[i], kvs[i][0], kvs[i][1], ws, outs[i], status=c.status, flags=flags)
+        torch.cuda.synchronize()
+        assert int(cs[0].status.item()) == 0 and int(cs[1].status.item()) == 0
+        res[flags] = [o.clone() for o in outs]
+    for a, b in zip(res[0], res[S.STIEF_DECODE_OVERLAP_PREVIOUS]):
+        assert torch.equal(a, b)
+    # and the last step against the oracle (the row appended by step 7 overwrote those of steps 1, 3, 5)
+    c = cs[1]
+    Kd, Vd = U.oracle_cache(c)
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    kn, vn = U.f64(kvs[7][0]), U.f64(kvs[7][1])
+    for b in range(B):
+        Kd[b] = np.concatenate([Kd[b], np.stack([O.compress(kn[b, h][None], O.basis_of(Uk, h))[0] for h in range(Hkv)])[None]], 0)
+        Vd[b] = np.concatenate([Vd[b], np.stack([O.compress(vn[b, h][None], O.basis_of(Uv, h))[0] for h in range(Hkv)])[None]], 0)
+    ref, _ = O.decode_layer(U.f64(qs[7]), Kd, Vd, Uk, Uv, "b")
+    U.check_out(res[1][7], ref)
+
+
 def test_host_staged_step():
     B, Hq, Hkv = 2, 8, 2
     c = U.make_case(60, B, Hq, Hkv, 64, 64, [100, 70], reserve=4)
