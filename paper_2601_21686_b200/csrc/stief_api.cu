@@ -124,6 +124,27 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+}  // namespace
+
+bool encode_bf16_map(CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box, CUtensorMapSwizzle swizzle) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc || rank < 1 || rank > 5) return false;
+  cuuint64_t gdim[5], gstride[4];
+  cuuint32_t bx[5], estr[5];
+  for (int i = 0; i < rank; ++i) {
+    gdim[i] = dims[i];
+    bx[i] = box[i];
+    estr[i] = 1;
+    if (i > 0) gstride[i - 1] = strides_bytes[i - 1];
+  }
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, bx, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
 // pool viewed as a 2-D bf16 tensor [rows = num_pages*Hkv*64][r]; box = 64 rows x box-width, swizzle span = box row
 bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
   EncodeTiledFn enc = encode_fn();
@@ -210,6 +231,7 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
   if (!K || !V || !aligned(K, 16) || !aligned(V, 16)) return STIEF_ERR_INVALID_ARG;
   if (T_max <= 0 || stride_t < (int64_t)layer->Hkv * kD || stride_b < 0 || (stride_t % 8) != 0 || (stride_b % 8) != 0)
     return STIEF_ERR_INVALID_ARG;
+  if (batch->B > 1 && stride_b == 0) return STIEF_ERR_INVALID_ARG;
   PrefillArgs a;
   a.L = to_dev(layer); a.Bt = to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);

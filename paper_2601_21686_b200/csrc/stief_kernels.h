@@ -46,6 +46,12 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st);
 
 // Returns cudaErrorInvalidValue for a rank pair that is not compiled in.
 cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st);
+// Encodes a tiled bf16 tensor map (rank <= 5; dims/box in elements, strides in bytes for dims 1..rank-1) with the
+// given swizzle.  Returns false when the driver entry point is missing or refuses the arguments.
+bool encode_bf16_map(CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box, CUtensorMapSwizzle swizzle);
+// Full-rank side of the prefill (no basis): the rows are copied to the pool unchanged.  side: 0 = keys, 1 = values.
+cudaError_t launch_prefill_copy(const PrefillArgs& a, int side, cudaStream_t st);
 // Box width (elements) of the TMA tiles the decode kernel expects for rank r.
 int decode_box_width(int r);
 

@@ -1,0 +1,403 @@
+// Prefill compression on the 5th-generation tensor cores (Eq. 1 for a whole prompt):
+//     X_down[t, :] = rnd_bf16( X[t, :] U ),   X = K or V rows of one KV head, U = that head's basis.
+// A streaming GEMM with tokens as M (tiles of 128), the rank as N and d_h = 128 as the whole K extent.
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      producer: one TMA tiled load per half tile (128 tokens x 64 elements, 128-byte swizzle)
+//               of the caller's [B][T][Hkv][128] tensor into a ring of NST stages, completion on mbarriers.
+//   warp 1      MMA: allocates TMEM, and one lane issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32,
+//               M = 128, N = r, 8 instructions of K = 16 per tile) from shared-memory descriptors into one of
+//               two TMEM accumulators; tcgen05.commit frees the ring stage and publishes the accumulator.
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = token row), round to bf16, 16-byte stores to the
+//               paged pool; they also bring the basis into shared memory, transposed to the K-major swizzled
+//               layout the MMA wants, one buffer ahead of the MMA warp.
+// Work is the list of valid tiles ordered (side, head, sequence, tile) and cut into equal contiguous ranges,
+// so a CTA changes basis at most a couple of times.  The projection is HBM-bound (about 43-64 flop per byte
+// against a ridge near 250): the tensor pipe idles most of the time by construction, and what matters is that
+// no issue slot stands between HBM and the MMA.
+//
+// Every wait is bounded: when one runs out the status word says STIEF_ERR_TIMEOUT, later waits of the CTA
+// return at once, every role walks to the end of its loop, and the TMEM allocation is released.
+#include "stief_kernels.h"
+#include "stief_partition.cuh"
+
+namespace stief {
+
+namespace tc {
+
+constexpr int kTileM = 128;                       // tokens per tile
+constexpr int kNST = 4;                           // ring stages
+constexpr int kStageBytes = kTileM * kD * 2;      // 32 KiB: two halves of 128 rows x 128 bytes
+constexpr int kHalfBytes = kStageBytes / 2;
+constexpr int kUBytes = 128 * kD * 2;             // room for a basis of rank 128, K-major
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 256;                    // two accumulators of up to 128 fp32 columns
+constexpr int kCtrlBytes = 256;
+constexpr int kPrefBytes = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
+constexpr int kSmemBytes = 1024 + kNST * kStageBytes + 2 * kUBytes + kCtrlBytes + kPrefBytes;
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
+
+struct Args {
+  PrefillArgs p;
+  int n_side;                // sides that have a basis (1 or 2)
+  int side0;                 // which side comes first: 0 = keys, 1 = values
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]; both operands K-major, described by shared-memory matrix descriptors
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the mbarrier gets one arrival when every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand stored as rows of 128 bytes (64 bf16 of K) with the
+// 128-byte swizzle, 8-row groups 1024 bytes apart.  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4
+// (unused by swizzled K-major layouts, set to 1), [32,46) stride byte offset >> 4, [46,48) version = 1,
+// [61,64) layout = 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t kmajor_sw128_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: D fp32 (bits [4,6) = 1), A and B bf16 (bits [7,10) = [10,13) = 1), both
+// K-major (bits 15, 16 = 0), N >> 3 in bits [17,23), M >> 4 in bits [24,29).
+__device__ __forceinline__ uint32_t idesc_bf16_f32(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// A tile of the work list
+struct WorkTile {
+  int side;     // 0 = keys, 1 = values
+  int h, b, t0; // head, sequence, first token
+  int len;      // tokens of the sequence
+  int unit;     // side slot * Hkv + h: tiles of one unit share a basis
+};
+
+// pref[b] = tiles of sequences before b (one head, one side); tiles_all = pref[B]
+__device__ __forceinline__ WorkTile decode_tile(int w, const int* pref, int B, int Hkv, int tiles_all, int side0, const int* seq_lens, int T_max) {
+  WorkTile t;
+  const int unit = w / tiles_all;
+  int rem = w - unit * tiles_all;
+  t.unit = unit;
+  const int slot = unit / Hkv;
+  t.side = slot == 0 ? side0 : 1 - side0;
+  t.h = unit - slot * Hkv;
+  int lo = 0, hi = B;                                   // largest b with pref[b] <= rem
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (pref[mid] <= rem) lo = mid; else hi = mid;
+  }
+  t.b = lo;
+  t.t0 = (rem - pref[lo]) * kTileM;
+  t.len = min(max(seq_lens[lo], 0), T_max);
+  return t;
+}
+
+}  // namespace tc
+
+using namespace tc;
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Args a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t ring = base;                                   // kNST stages, each 1024-byte aligned
+  const uint32_t ubuf = base + kNST * kStageBytes;              // two basis buffers
+  uint8_t* ubuf_ptr = base_ptr + kNST * kStageBytes;
+  const uint32_t ctrl = ubuf + 2 * kUBytes;
+  uint8_t* ctrl_ptr = ubuf_ptr + 2 * kUBytes;
+  auto full_bar = [&](int s) { return ctrl + s * 8; };
+  auto empty_bar = [&](int s) { return ctrl + (8 + s) * 8; };
+  auto acc_full = [&](int i) { return ctrl + (16 + i) * 8; };
+  auto acc_empty = [&](int i) { return ctrl + (18 + i) * 8; };
+  auto u_ready = [&](int i) { return ctrl + (20 + i) * 8; };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 22 * 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + 22 * 8 + 4);
+  int* pref = reinterpret_cast<int*>(ctrl_ptr + kCtrlBytes);
+
+  const PrefillArgs& p = a.p;
+  const int B = p.Bt.B, Hkv = p.L.Hkv;
+
+  if (tid == 0) {
+    for (int s = 0; s < kNST; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full(i), 1);
+      mbar_init(acc_empty(i), 4);          // one arrival per epilogue warp
+      mbar_init(u_ready(i), 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  // tiles per sequence (one head, one side), exclusive prefix sums
+  if (warp == 0) {
+    int carry = 0;
+    for (int b0 = 0; b0 < B; b0 += 32) {
+      const int b = b0 + lane;
+      int v = 0;
+      if (b < B) v = (min(max(p.Bt.seq_lens[b], 0), p.T_max) + kTileM - 1) / kTileM;
+      int s = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, s, o);
+        if (lane >= o) s += t;
+      }
+      if (b < B) pref[b + 1] = carry + s;
+      carry += __shfl_sync(0xffffffffu, s, 31);
+    }
+    if (lane == 0) pref[0] = 0;
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_all = pref[B];
+  const long long total = (long long)tiles_all * Hkv * a.n_side;
+  const int per_cta = (int)((total + gridDim.x - 1) / gridDim.x);
+  const long long w_begin = (long long)blockIdx.x * per_cta;
+  const int w0 = (int)min(w_begin, total), w1 = (int)min(w_begin + per_cta, total);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmK);
+      tma_prefetch_desc(&tmV);
+      for (int w = w0, i = 0; w < w1; ++w, ++i) {
+        const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
+        const int s = i % kNST, use = i / kNST;
+        if (use > 0) mbar_wait(empty_bar(s), (use - 1) & 1, abort_flag, p.status);
+        const uint32_t dst = ring + s * kStageBytes;
+        const CUtensorMap* tm = t.side ? &tmV : &tmK;
+        mbar_arrive_expect_tx(full_bar(s), kStageBytes);
+        tma_load_4d(dst, tm, 0, t.h, t.t0, t.b, full_bar(s));
+        tma_load_4d(dst + kHalfBytes, tm, 64, t.h, t.t0, t.b, full_bar(s));
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      int cur_unit = -1, gen = -1;
+      uint32_t idesc = 0;
+      int R = 0;
+      for (int w = w0, i = 0; w < w1; ++w, ++i) {
+        const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
+        if (t.unit != cur_unit) {                          // a new basis: wait until the epilogue warps have staged it
+          cur_unit = t.unit;
+          ++gen;
+          R = t.side ? p.L.r_v : p.L.r_k;
+          idesc = idesc_bf16_f32(kTileM, R);
+          mbar_wait(u_ready(gen & 1), (gen >> 1) & 1, abort_flag, p.status);
+        }
+        const int s = i % kNST, acc = i & 1;
+        if (i >= 2) mbar_wait(acc_empty(acc), ((i >> 1) - 1) & 1, abort_flag, p.status);
+        mbar_wait(full_bar(s), (i / kNST) & 1, abort_flag, p.status);
+        tc_fence_after();
+        const uint32_t a_base = ring + s * kStageBytes;
+        const uint32_t b_base = ubuf + (gen & 1) * kUBytes;
+        const uint32_t d_tmem = tmem_base + acc * 128;
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) {
+          const uint32_t koff = (k & 3) * 32;              // 16 bf16 = 32 bytes inside the 128-byte swizzled row
+          const uint64_t da = kmajor_sw128_desc(a_base + (k >> 2) * kHalfBytes + koff);
+          const uint64_t db = kmajor_sw128_desc(b_base + (k >> 2) * (R * 128) + koff);
+          umma_bf16(d_tmem, da, db, idesc, k > 0 ? 1u : 0u);
+        }
+        umma_commit(empty_bar(s));                         // the stage may be refilled once these MMAs have read it
+        umma_commit(acc_full(acc));                        // and the accumulator is complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps (2..5)
+    const int q = warp & 3;                                // TMEM lane quarter this warp may read
+    const int et = tid - 64;                               // 0..127
+    int cur_unit = -1, gen = -1;
+    int R = 0;
+
+    // Stage the basis of `unit` in buffer gen & 1: element (d, j) of U goes to row j of the K-major operand,
+    // 64-element half d / 64, 16-byte piece ((d % 64) / 8) ^ (j % 8) of the 128-byte row.
+    auto stage_basis = [&](const WorkTile& t, int g) {
+      const int Rn = t.side ? p.L.r_v : p.L.r_k;
+      const __nv_bfloat16* Ub = t.side ? p.L.U_v : p.L.U_k;
+      const __nv_bfloat16* U = Ub + (size_t)t.h * (t.side ? p.L.uv_stride : p.L.uk_stride);
+      uint8_t* dst = ubuf_ptr + (g & 1) * kUBytes;
+      const int pairs = Rn / 2;
+      for (int idx0 = 0; idx0 < kD * pairs; idx0 += 128 * 8) {
+        uint32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int idx = idx0 + u * 128 + et;
+          v[u] = idx < kD * pairs ? __ldg(reinterpret_cast<const uint32_t*>(U) + idx) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int idx = idx0 + u * 128 + et;
+          if (idx < kD * pairs) {
+            const int d = idx / pairs, j = 2 * (idx % pairs);
+            const int half = d >> 6, piece = (d & 63) >> 3, e = d & 7;
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+              const int row = j + jj;
+              const uint32_t off = half * (Rn * 128) + (row >> 3) * 1024 + (row & 7) * 128 + ((piece ^ (row & 7)) << 4) + e * 2;
+              *reinterpret_cast<uint16_t*>(dst + off) = (uint16_t)(jj ? (v[u] >> 16) : (v[u] & 0xffffu));
+            }
+          }
+        }
+      }
+      fence_proxy_async_smem();                            // generic-proxy writes -> visible to the tensor core's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(u_ready(g & 1));
+    };
+
+    for (int w = w0, i = 0; w < w1; ++w, ++i) {
+      const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
+      if (t.unit != cur_unit) {
+        if (gen < 0) stage_basis(t, ++gen);                // first tile of the CTA
+        cur_unit = t.unit;
+        R = t.side ? p.L.r_v : p.L.r_k;
+      }
+      if (w + 1 < w1) {                                    // stage the next basis one buffer ahead
+        const WorkTile tn = decode_tile(w + 1, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
+        if (tn.unit != cur_unit) stage_basis(tn, ++gen);
+      }
+      const int acc = i & 1;
+      mbar_wait(acc_full(acc), (i >> 1) & 1, abort_flag, p.status);
+      tc_fence_after();
+
+      const int tok = t.t0 + 32 * q + lane;
+      const int pi = (t.t0 + 32 * q) / kPage;
+      int page = -1;
+      if (t.t0 + 32 * q < t.len) {
+        if (lane == 0) page = pi < p.Bt.max_pages ? p.Bt.block_table[(size_t)t.b * p.Bt.max_pages + pi] : -1;
+        page = __shfl_sync(0xffffffffu, page, 0);
+        if (page < 0 || page >= p.L.num_pages) {
+          if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
+          page = -1;
+        }
+      }
+      __nv_bfloat16* pool = t.side ? p.L.v_pool : p.L.k_pool;
+      const bool store = page >= 0 && tok < t.len;
+      uint4* dst = reinterpret_cast<uint4*>(pool + (((size_t)max(page, 0) * Hkv + t.h) * kPage + (tok % kPage)) * R);
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + acc * 128;
+      for (int c = 0; c < R / 16; ++c) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c * 16, v);
+        tmem_ld_wait();
+        if (store) {
+          uint4 o0, o1;
+          o0.x = pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1]));
+          o0.y = pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3]));
+          o0.z = pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5]));
+          o0.w = pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7]));
+          o1.x = pack_bf16(__uint_as_float(v[8]), __uint_as_float(v[9]));
+          o1.y = pack_bf16(__uint_as_float(v[10]), __uint_as_float(v[11]));
+          o1.z = pack_bf16(__uint_as_float(v[12]), __uint_as_float(v[13]));
+          o1.w = pack_bf16(__uint_as_float(v[14]), __uint_as_float(v[15]));
+          dst[2 * c] = o0;
+          dst[2 * c + 1] = o1;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(acc));          // this warp has read its quarter of the accumulator
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+namespace {
+
+int sm_count_of_current_device() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return 148;
+  }
+  return n;
+}
+
+// [B][T_max][Hkv][128] bf16 with element strides (stride_b, stride_t, 128, 1), boxes of 128 tokens x 64 elements
+bool make_input_map(CUtensorMap* tm, const void* X, const PrefillArgs& a) {
+  const unsigned long long sb = a.stride_b > 0 ? (unsigned long long)a.stride_b : (unsigned long long)a.stride_t * a.T_max;
+  const unsigned long long dims[4] = {(unsigned long long)kD, (unsigned long long)a.L.Hkv, (unsigned long long)a.T_max,
+                                      (unsigned long long)a.Bt.B};
+  const unsigned long long strides[3] = {(unsigned long long)kD * 2, (unsigned long long)a.stride_t * 2, sb * 2};
+  const unsigned box[4] = {64, 1, (unsigned)kTileM, 1};
+  return encode_bf16_map(tm, X, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+}  // namespace
+
+cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
+  const bool proj_k = a.L.U_k != nullptr, proj_v = a.L.U_v != nullptr;
+  if (!proj_k) {
+    cudaError_t e = launch_prefill_copy(a, 0, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (!proj_v) {
+    cudaError_t e = launch_prefill_copy(a, 1, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (!proj_k && !proj_v) return cudaSuccess;
+
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  CUtensorMap tmK, tmV;
+  if (!make_input_map(&tmK, proj_k ? a.K : a.V, a) || !make_input_map(&tmV, proj_v ? a.V : a.K, a)) return cudaErrorInvalidValue;
+  Args args;
+  args.p = a;
+  args.n_side = (proj_k ? 1 : 0) + (proj_v ? 1 : 0);
+  args.side0 = proj_k ? 0 : 1;
+  prefill_tc_kernel<<<sm_count_of_current_device(), kThreads, kSmemBytes, st>>>(tmK, tmV, args);
+  return cudaGetLastError();
+}
+
+}  // namespace stief
