@@ -26,21 +26,23 @@ namespace stief {
 namespace tc {
 
 constexpr int kTileM = 128;                       // tokens per tile
-constexpr int kNST = 4;                           // ring stages
+constexpr int kMaxNST = 4;                        // ring stages (3 when rank 128 and a large batch leave no room)
 constexpr int kStageBytes = kTileM * kD * 2;      // 32 KiB: two halves of 128 rows x 128 bytes
 constexpr int kHalfBytes = kStageBytes / 2;
-constexpr int kUBytes = 128 * kD * 2;             // room for a basis of rank 128, K-major
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;                    // two accumulators of up to 128 fp32 columns
 constexpr int kCtrlBytes = 256;
-constexpr int kPrefBytes = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
-constexpr int kSmemBytes = 1024 + kNST * kStageBytes + 2 * kUBytes + kCtrlBytes + kPrefBytes;
-static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
+constexpr int kSmemLimit = 232448;                // 227 KiB per CTA
+
+// Shared memory, from a 1024-byte aligned base: ring [nst][32 KiB] | two basis buffers [rmax * 256] |
+// output staging [4 warps][32 rows][rmax * 2] | barriers and flags | tile prefix sums [B + 1].
 
 struct Args {
   PrefillArgs p;
   int n_side;                // sides that have a basis (1 or 2)
   int side0;                 // which side comes first: 0 = keys, 1 = values
+  int nst;                   // ring stages
+  int rmax;                  // larger of the ranks that are projected
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -50,6 +52,18 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
+// 2-D tiled store shared -> global (the tensor map undoes the shared-memory swizzle); completion is tracked by
+// the issuing thread's bulk async-group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until the bulk stores committed so far by this thread have finished READING shared memory
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -100,45 +114,99 @@ __device__ __forceinline__ uint32_t idesc_bf16_f32(int M, int N) {
 struct WorkTile {
   int side;     // 0 = keys, 1 = values
   int h, b, t0; // head, sequence, first token
-  int len;      // tokens of the sequence
+  int len;      // tokens of the sequence if this is its last tile, else any value >= t0 + 128
   int unit;     // side slot * Hkv + h: tiles of one unit share a basis
 };
 
-// pref[b] = tiles of sequences before b (one head, one side); tiles_all = pref[B]
-__device__ __forceinline__ WorkTile decode_tile(int w, const int* pref, int B, int Hkv, int tiles_all, int side0, const int* seq_lens, int T_max) {
-  WorkTile t;
-  const int unit = w / tiles_all;
-  int rem = w - unit * tiles_all;
-  t.unit = unit;
-  const int slot = unit / Hkv;
-  t.side = slot == 0 ? side0 : 1 - side0;
-  t.h = unit - slot * Hkv;
-  int lo = 0, hi = B;                                   // largest b with pref[b] <= rem
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (pref[mid] <= rem) lo = mid; else hi = mid;
+// Walks the tiles [w0, w1) of the work list in order.  pref[b] = tiles of the sequences before b (one head, one
+// side); tiles_all = pref[B]; tile w belongs to unit w / tiles_all.  Positioning costs two divisions and a
+// binary search once; every further step is a few adds, because each role runs this on a single thread and a
+// division per tile would show up in the tile rate.
+struct TileWalker {
+  const int* pref;
+  int B, Hkv, side0, left;
+  int unit, side, h, b, k, nb;     // current unit (its side and head), sequence, tile within it, tiles of the sequence
+
+  __device__ __forceinline__ void set_unit(int u) {
+    unit = u;
+    const int slot = u / Hkv;
+    side = slot == 0 ? side0 : 1 - side0;
+    h = u - slot * Hkv;
   }
-  t.b = lo;
-  t.t0 = (rem - pref[lo]) * kTileM;
-  t.len = min(max(seq_lens[lo], 0), T_max);
-  return t;
-}
+  __device__ void init(const int* pref_, int B_, int Hkv_, int side0_, int tiles_all, int w0, int w1) {
+    pref = pref_; B = B_; Hkv = Hkv_; side0 = side0_;
+    left = w1 - w0;
+    unit = side = h = b = k = 0; nb = 1;
+    if (left <= 0) return;
+    set_unit(w0 / tiles_all);
+    const int rem = w0 - unit * tiles_all;
+    int lo = 0, hi = B;                                   // largest b with pref[b] <= rem
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (pref[mid] <= rem) lo = mid; else hi = mid;
+    }
+    b = lo;
+    k = rem - pref[lo];
+    nb = pref[lo + 1] - pref[lo];
+  }
+  __device__ __forceinline__ bool valid() const { return left > 0; }
+  __device__ __forceinline__ WorkTile cur(const int* seq_lens, int T_max) const {
+    WorkTile t;
+    t.side = side; t.h = h; t.b = b; t.unit = unit;
+    t.t0 = k * kTileM;
+    // only a sequence's last tile can be partial; the others never touch global memory here (a dependent
+    // global load per tile would serialise the role on memory latency)
+    t.len = (k + 1 == nb) ? min(max(seq_lens[b], 0), T_max) : t.t0 + kTileM;
+    return t;
+  }
+  __device__ __forceinline__ void advance() {
+    if (--left <= 0) return;
+    if (++k < nb) return;
+    k = 0;
+    do {
+      if (++b == B) {
+        b = 0;
+        set_unit(unit + 1);
+      }
+      nb = pref[b + 1] - pref[b];
+    } while (nb == 0);                                    // left > 0 guarantees a sequence with tiles ahead
+  }
+  // unit of the tile after the current one, or -1 at the end of the range
+  __device__ __forceinline__ int next_unit() const {
+    if (left <= 1) return -1;
+    if (k + 1 < nb) return unit;
+    int bb = b, uu = unit;
+    do {
+      if (++bb == B) {
+        bb = 0;
+        ++uu;
+      }
+    } while (pref[bb + 1] == pref[bb]);
+    return uu;
+  }
+};
 
 }  // namespace tc
 
 using namespace tc;
 
 __global__ void __launch_bounds__(kThreads, 1)
-prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Args a) {
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                  const __grid_constant__ CUtensorMap tmPK, const __grid_constant__ CUtensorMap tmPV, const Args a) {
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t ring = base;                                   // kNST stages, each 1024-byte aligned
+  const int kNST = a.nst;
+  const int kUBytes = a.rmax * 256;                             // one basis, K-major: rmax rows of 256 bytes
+  const int kOutBytes = 32 * a.rmax * 2;                        // one warp's 32 output rows
+  const uint32_t ring = base;                                   // nst stages, each 1024-byte aligned
   const uint32_t ubuf = base + kNST * kStageBytes;              // two basis buffers
   uint8_t* ubuf_ptr = base_ptr + kNST * kStageBytes;
-  const uint32_t ctrl = ubuf + 2 * kUBytes;
-  uint8_t* ctrl_ptr = ubuf_ptr + 2 * kUBytes;
+  const uint32_t obuf = ubuf + 2 * kUBytes;                     // output staging, one region per epilogue warp
+  uint8_t* obuf_ptr = ubuf_ptr + 2 * kUBytes;
+  const uint32_t ctrl = obuf + 4 * kOutBytes;
+  uint8_t* ctrl_ptr = obuf_ptr + 4 * kOutBytes;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (8 + s) * 8; };
   auto acc_full = [&](int i) { return ctrl + (16 + i) * 8; };
@@ -199,15 +267,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     if (lane == 0) {
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
-      for (int w = w0, i = 0; w < w1; ++w, ++i) {
-        const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
-        const int s = i % kNST, use = i / kNST;
+      tma_prefetch_desc(&tmPK);
+      tma_prefetch_desc(&tmPV);
+      TileWalker wk;
+      wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+      int s = 0, use = 0;                                  // ring stage and how often it has been used
+      for (; wk.valid(); wk.advance()) {
+        const int t_side = wk.side, t_h = wk.h, t_b = wk.b, t_t0 = wk.k * kTileM;
         if (use > 0) mbar_wait(empty_bar(s), (use - 1) & 1, abort_flag, p.status);
         const uint32_t dst = ring + s * kStageBytes;
-        const CUtensorMap* tm = t.side ? &tmV : &tmK;
+        const CUtensorMap* tm = t_side ? &tmV : &tmK;
         mbar_arrive_expect_tx(full_bar(s), kStageBytes);
-        tma_load_4d(dst, tm, 0, t.h, t.t0, t.b, full_bar(s));
-        tma_load_4d(dst + kHalfBytes, tm, 64, t.h, t.t0, t.b, full_bar(s));
+        tma_load_4d(dst, tm, 0, t_h, t_t0, t_b, full_bar(s));
+        tma_load_4d(dst + kHalfBytes, tm, 64, t_h, t_t0, t_b, full_bar(s));
+        if (++s == kNST) {
+          s = 0;
+          ++use;
+        }
       }
     }
   } else if (warp == 1) {
@@ -216,18 +292,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       int cur_unit = -1, gen = -1;
       uint32_t idesc = 0;
       int R = 0;
-      for (int w = w0, i = 0; w < w1; ++w, ++i) {
-        const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
-        if (t.unit != cur_unit) {                          // a new basis: wait until the epilogue warps have staged it
-          cur_unit = t.unit;
+      TileWalker wk;
+      wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+      int s = 0, use = 0;
+      for (int i = 0; wk.valid(); wk.advance(), ++i) {
+        if (wk.unit != cur_unit) {                         // a new basis: wait until the epilogue warps have staged it
+          cur_unit = wk.unit;
           ++gen;
-          R = t.side ? p.L.r_v : p.L.r_k;
+          R = wk.side ? p.L.r_v : p.L.r_k;
           idesc = idesc_bf16_f32(kTileM, R);
           mbar_wait(u_ready(gen & 1), (gen >> 1) & 1, abort_flag, p.status);
         }
-        const int s = i % kNST, acc = i & 1;
+        const int acc = i & 1;
         if (i >= 2) mbar_wait(acc_empty(acc), ((i >> 1) - 1) & 1, abort_flag, p.status);
-        mbar_wait(full_bar(s), (i / kNST) & 1, abort_flag, p.status);
+        mbar_wait(full_bar(s), use & 1, abort_flag, p.status);
         tc_fence_after();
         const uint32_t a_base = ring + s * kStageBytes;
         const uint32_t b_base = ubuf + (gen & 1) * kUBytes;
@@ -241,6 +319,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
         umma_commit(empty_bar(s));                         // the stage may be refilled once these MMAs have read it
         umma_commit(acc_full(acc));                        // and the accumulator is complete
+        if (++s == kNST) {
+          s = 0;
+          ++use;
+        }
       }
     }
   } else {
@@ -252,10 +334,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
     // Stage the basis of `unit` in buffer gen & 1: element (d, j) of U goes to row j of the K-major operand,
     // 64-element half d / 64, 16-byte piece ((d % 64) / 8) ^ (j % 8) of the 128-byte row.
-    auto stage_basis = [&](const WorkTile& t, int g) {
-      const int Rn = t.side ? p.L.r_v : p.L.r_k;
-      const __nv_bfloat16* Ub = t.side ? p.L.U_v : p.L.U_k;
-      const __nv_bfloat16* U = Ub + (size_t)t.h * (t.side ? p.L.uv_stride : p.L.uk_stride);
+    auto stage_basis = [&](int side, int h, int g) {
+      const int Rn = side ? p.L.r_v : p.L.r_k;
+      const __nv_bfloat16* Ub = side ? p.L.U_v : p.L.U_k;
+      const __nv_bfloat16* U = Ub + (size_t)h * (side ? p.L.uv_stride : p.L.uk_stride);
       uint8_t* dst = ubuf_ptr + (g & 1) * kUBytes;
       const int pairs = Rn / 2;
       for (int idx0 = 0; idx0 < kD * pairs; idx0 += 128 * 8) {
@@ -285,60 +367,116 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       if (lane == 0) mbar_arrive(u_ready(g & 1));
     };
 
-    for (int w = w0, i = 0; w < w1; ++w, ++i) {
-      const WorkTile t = decode_tile(w, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
+    TileWalker wk;
+    wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+    for (int i = 0; wk.valid(); wk.advance(), ++i) {
+      const WorkTile t = wk.cur(p.Bt.seq_lens, p.T_max);
       if (t.unit != cur_unit) {
-        if (gen < 0) stage_basis(t, ++gen);                // first tile of the CTA
+        if (gen < 0) stage_basis(t.side, t.h, ++gen);      // first tile of the CTA
         cur_unit = t.unit;
         R = t.side ? p.L.r_v : p.L.r_k;
       }
-      if (w + 1 < w1) {                                    // stage the next basis one buffer ahead
-        const WorkTile tn = decode_tile(w + 1, pref, B, Hkv, tiles_all, a.side0, p.Bt.seq_lens, p.T_max);
-        if (tn.unit != cur_unit) stage_basis(tn, ++gen);
+      {                                                    // stage the next basis one buffer ahead
+        const int nu = wk.next_unit();
+        if (nu >= 0 && nu != cur_unit) {
+          const int slot = nu / Hkv;
+          stage_basis(slot == 0 ? a.side0 : 1 - a.side0, nu - slot * Hkv, ++gen);
+        }
       }
+      // the page of this warp's 32 tokens: fetched before the wait so its latency hides behind the accumulator's
+      const int tok0 = t.t0 + 32 * q;                      // the warp's first token; its 32 tokens share a page
+      int page = -1;
+      if (lane == 0 && tok0 < t.len && tok0 / kPage < p.Bt.max_pages)
+        page = p.Bt.block_table[(size_t)t.b * p.Bt.max_pages + tok0 / kPage];
+
       const int acc = i & 1;
       mbar_wait(acc_full(acc), (i >> 1) & 1, abort_flag, p.status);
       tc_fence_after();
 
-      const int tok = t.t0 + 32 * q + lane;
-      const int pi = (t.t0 + 32 * q) / kPage;
-      int page = -1;
-      if (t.t0 + 32 * q < t.len) {
-        if (lane == 0) page = pi < p.Bt.max_pages ? p.Bt.block_table[(size_t)t.b * p.Bt.max_pages + pi] : -1;
-        page = __shfl_sync(0xffffffffu, page, 0);
-        if (page < 0 || page >= p.L.num_pages) {
-          if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
-          page = -1;
-        }
-      }
-      __nv_bfloat16* pool = t.side ? p.L.v_pool : p.L.k_pool;
-      const bool store = page >= 0 && tok < t.len;
-      uint4* dst = reinterpret_cast<uint4*>(pool + (((size_t)max(page, 0) * Hkv + t.h) * kPage + (tok % kPage)) * R);
+      // ---- the warp's 32 rows of the accumulator -> registers (all loads in flight, one wait)
       const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + acc * 128;
-      for (int c = 0; c < R / 16; ++c) {
-        uint32_t v[16];
-        tmem_ld16(taddr + c * 16, v);
-        tmem_ld_wait();
-        if (store) {
-          uint4 o0, o1;
-          o0.x = pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1]));
-          o0.y = pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3]));
-          o0.z = pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5]));
-          o0.w = pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7]));
-          o1.x = pack_bf16(__uint_as_float(v[8]), __uint_as_float(v[9]));
-          o1.y = pack_bf16(__uint_as_float(v[10]), __uint_as_float(v[11]));
-          o1.z = pack_bf16(__uint_as_float(v[12]), __uint_as_float(v[13]));
-          o1.w = pack_bf16(__uint_as_float(v[14]), __uint_as_float(v[15]));
-          dst[2 * c] = o0;
-          dst[2 * c + 1] = o1;
-        }
-      }
+      uint32_t v[8][16];
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        if (c < R / 16) tmem_ld16(taddr + c * 16, v[c]);
+      tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty(acc));          // this warp has read its quarter of the accumulator
+
+      if (tok0 >= t.len) continue;
+      page = __shfl_sync(0xffffffffu, page, 0);
+      if (page < 0 || page >= p.L.num_pages) {
+        if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
+        continue;
+      }
+      const int row0 = (page * Hkv + t.h) * kPage + (tok0 % kPage);          // pool row of the warp's first token
+      if (tok0 + 32 <= t.len) {
+        // ---- all 32 rows valid: round to bf16 into the swizzled staging boxes, then TMA stores.  A box is 32
+        // rows x BW elements (BW = 64, 32 or 16: the largest that divides R), swizzle span = box row.
+        const int lbw = (R % 64 == 0) ? 6 : (R % 32 == 0) ? 5 : 4;       // log2 of the box width
+        const int BW = 1 << lbw, RB = BW * 2, CPB = BW / 8;
+        const uint32_t wbase = obuf + (warp - 2) * kOutBytes;
+        uint8_t* wptr = obuf_ptr + (warp - 2) * kOutBytes;
+        if (lane == 0) bulk_wait_read_all();               // the previous tile's stores have left the staging region
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c < R / 16) {
+            uint4 o[2];
+            o[0].x = pack_bf16(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]));
+            o[0].y = pack_bf16(__uint_as_float(v[c][2]), __uint_as_float(v[c][3]));
+            o[0].z = pack_bf16(__uint_as_float(v[c][4]), __uint_as_float(v[c][5]));
+            o[0].w = pack_bf16(__uint_as_float(v[c][6]), __uint_as_float(v[c][7]));
+            o[1].x = pack_bf16(__uint_as_float(v[c][8]), __uint_as_float(v[c][9]));
+            o[1].y = pack_bf16(__uint_as_float(v[c][10]), __uint_as_float(v[c][11]));
+            o[1].z = pack_bf16(__uint_as_float(v[c][12]), __uint_as_float(v[c][13]));
+            o[1].w = pack_bf16(__uint_as_float(v[c][14]), __uint_as_float(v[c][15]));
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int col = 16 * c + 8 * e;              // first of the 8 columns in this 16-byte piece
+              const int nb = col >> lbw, cc = (col & (BW - 1)) >> 3;
+              uint32_t off = (uint32_t)(lane * RB + cc * 16);
+              off ^= ((off >> 7) & (uint32_t)(CPB - 1)) << 4;
+              *reinterpret_cast<uint4*>(wptr + ((nb * 32) << (lbw + 1)) + off) = o[e];
+            }
+          }
+        }
+        fence_proxy_async_smem();                          // generic-proxy writes -> visible to the TMA store
+        __syncwarp();
+        if (lane == 0) {
+          const CUtensorMap* tmP = t.side ? &tmPV : &tmPK;
+          for (int nb = 0; nb < (R >> lbw); ++nb) tma_store_2d(tmP, nb * BW, row0, wbase + nb * 32 * RB);
+          bulk_commit_group();
+        }
+      } else {
+        // ---- the sequence ends inside these 32 rows: rows at or beyond its length must stay untouched
+        const int tok = tok0 + lane;
+        __nv_bfloat16* pool = t.side ? p.L.v_pool : p.L.k_pool;
+        uint4* dst = reinterpret_cast<uint4*>(pool + ((size_t)row0 + lane) * R);
+        if (tok < t.len) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            if (c < R / 16) {
+              uint4 o0, o1;
+              o0.x = pack_bf16(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]));
+              o0.y = pack_bf16(__uint_as_float(v[c][2]), __uint_as_float(v[c][3]));
+              o0.z = pack_bf16(__uint_as_float(v[c][4]), __uint_as_float(v[c][5]));
+              o0.w = pack_bf16(__uint_as_float(v[c][6]), __uint_as_float(v[c][7]));
+              o1.x = pack_bf16(__uint_as_float(v[c][8]), __uint_as_float(v[c][9]));
+              o1.y = pack_bf16(__uint_as_float(v[c][10]), __uint_as_float(v[c][11]));
+              o1.z = pack_bf16(__uint_as_float(v[c][12]), __uint_as_float(v[c][13]));
+              o1.w = pack_bf16(__uint_as_float(v[c][14]), __uint_as_float(v[c][15]));
+              dst[2 * c] = o0;
+              dst[2 * c + 1] = o1;
+            }
+          }
+        }
+      }
     }
   }
 
+  if (warp >= 2 && lane == 0) bulk_wait_all();            // this lane's TMA stores are complete
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -368,6 +506,20 @@ bool make_input_map(CUtensorMap* tm, const void* X, const PrefillArgs& a) {
   return encode_bf16_map(tm, X, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// pool [num_pages * Hkv * 64 rows][r] bf16, stored in boxes of 32 rows x BW elements, swizzle span = box row
+bool make_pool_store_map(CUtensorMap* tm, const void* pool, int r, const PrefillArgs& a) {
+  const int bw = (r % 64 == 0) ? 64 : (r % 32 == 0) ? 32 : 16;
+  const unsigned long long dims[2] = {(unsigned long long)r, (unsigned long long)a.L.num_pages * a.L.Hkv * kPage};
+  const unsigned long long strides[1] = {(unsigned long long)r * 2};
+  const unsigned box[2] = {(unsigned)bw, 32};
+  const CUtensorMapSwizzle sw = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  return encode_bf16_map(tm, pool, 2, dims, strides, box, sw);
+}
+
+int smem_bytes(int nst, int rmax, int B) {
+  return 1024 + nst * kStageBytes + 2 * rmax * 256 + 4 * 32 * rmax * 2 + kCtrlBytes + ((B + 1) * 4 + 127) / 128 * 128;
+}
+
 }  // namespace
 
 cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
@@ -386,17 +538,27 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   CUtensorMap tmK, tmV;
   if (!make_input_map(&tmK, proj_k ? a.K : a.V, a) || !make_input_map(&tmV, proj_v ? a.V : a.K, a)) return cudaErrorInvalidValue;
+  CUtensorMap tmPK, tmPV;
+  if (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a))
+    return cudaErrorInvalidValue;
   Args args;
   args.p = a;
   args.n_side = (proj_k ? 1 : 0) + (proj_v ? 1 : 0);
   args.side0 = proj_k ? 0 : 1;
-  prefill_tc_kernel<<<sm_count_of_current_device(), kThreads, kSmemBytes, st>>>(tmK, tmV, args);
+  args.rmax = 0;
+  if (proj_k) args.rmax = a.L.r_k;
+  if (proj_v && a.L.r_v > args.rmax) args.rmax = a.L.r_v;
+  args.nst = kMaxNST;
+  while (args.nst > 2 && smem_bytes(args.nst, args.rmax, a.Bt.B) > kSmemLimit) --args.nst;
+  const int smem = smem_bytes(args.nst, args.rmax, a.Bt.B);
+  if (smem > kSmemLimit) return cudaErrorInvalidValue;
+  prefill_tc_kernel<<<sm_count_of_current_device(), kThreads, smem, st>>>(tmK, tmV, tmPK, tmPV, args);
   return cudaGetLastError();
 }
 
