@@ -84,10 +84,17 @@ typedef struct stief_batch {
  * and the same for V, accumulated in fp32, stored to the paged pools.  K, V are bf16 with element
  * strides stride_b (between sequences) and stride_t (between tokens); heads are contiguous blocks of
  * 128 elements; rows must be 16-byte aligned.  T_max bounds seq_lens (it sizes the launch; tokens
- * beyond seq_lens[b] are not read). */
+ * beyond seq_lens[b] are never stored; the input rows of a sequence's last 128-token tile are read up
+ * to T_max).
+ * flags: 0, or STIEF_PREFILL_OVERLAP_PREVIOUS: the kernel may start (and write its pools) before the kernel
+ * that precedes it on the stream has finished, so that the per-layer launches of one prompt run without
+ * idle gaps.  By setting it the caller promises that the preceding kernel neither writes this call's
+ * inputs (K, V, seq_lens, block_table, the bases) nor touches this layer's pools; consecutive calls for
+ * different layers satisfy that.  The kernel still completes only after its predecessor has. */
+#define STIEF_PREFILL_OVERLAP_PREVIOUS 1u
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K,
                            const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
-                           int32_t* status, void* stream);
+                           uint32_t flags, int32_t* status, void* stream);
 
 /* Eq. 1 for one new token per sequence: projects k_new, v_new [B][Hkv][128] and stores the rows at
  * position seq_lens[b] (the page block_table[b][seq_lens[b]/64] must already be assigned).  The

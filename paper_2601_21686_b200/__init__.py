@@ -22,6 +22,7 @@ STIEF_ERR_CUDA, STIEF_ERR_BOUNDS, STIEF_ERR_TIMEOUT = 4, 5, 6
 PAGE = 64
 D_HEAD = 128
 STIEF_DECODE_OVERLAP_PREVIOUS = 1
+STIEF_PREFILL_OVERLAP_PREVIOUS = 1
 
 
 class StiefError(RuntimeError):
@@ -57,7 +58,7 @@ def lib() -> ctypes.CDLL:
         P, I32, I64, SZ, U32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32
         LP, BP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch)
         sig = {
-            "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, P, P]),
+            "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, U32, P, P]),
             "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
             "stief_decode_num_parts": (I32, []),
             "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
@@ -136,12 +137,12 @@ def stief_version() -> int:
 
 
 def stief_prefill_compress(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
-                           status: Optional[torch.Tensor] = None):
+                           status: Optional[torch.Tensor] = None, flags: int = 0):
     """K, V [B, T, Hkv, 128] bf16 (strides over b and t free, heads and d contiguous) -> paged compressed cache."""
     assert K.stride(3) == 1 and K.stride(2) == D_HEAD and V.stride() == K.stride()
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_prefill_compress(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
-                                        K.shape[1] if T_max is None else T_max, _ptr(status), _stream()),
+                                        K.shape[1] if T_max is None else T_max, flags, _ptr(status), _stream()),
            "stief_prefill_compress")
 
 

@@ -223,7 +223,8 @@ using namespace stief;
 extern "C" {
 
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K, const uint16_t* V,
-                           int64_t stride_b, int64_t stride_t, int32_t T_max, int32_t* status, void* stream) {
+                           int64_t stride_b, int64_t stride_t, int32_t T_max, uint32_t flags, int32_t* status, void* stream) {
+  if (flags & ~STIEF_PREFILL_OVERLAP_PREVIOUS) return STIEF_ERR_INVALID_ARG;
   int rc = check_layer(layer);
   if (rc) return rc;
   rc = check_batch(batch);
@@ -236,6 +237,7 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
   a.L = to_dev(layer); a.Bt = to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);
   a.stride_b = stride_b; a.stride_t = stride_t; a.T_max = T_max; a.status = status;
+  a.overlap_previous = (flags & STIEF_PREFILL_OVERLAP_PREVIOUS) != 0;
   return launch_prefill(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 

@@ -514,6 +514,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
     }
   }
+  grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
 }
 
 }  // namespace stief

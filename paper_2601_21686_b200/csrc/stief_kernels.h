@@ -31,6 +31,7 @@ struct PrefillArgs {
   long long stride_b, stride_t;
   int T_max;
   int32_t* status;
+  bool overlap_previous;        // launch with programmatic stream serialization
 };
 
 struct DecodeLaunch {

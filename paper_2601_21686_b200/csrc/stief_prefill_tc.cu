@@ -41,6 +41,7 @@ struct Args {
   PrefillArgs p;
   int n_side;                // sides that have a basis (1 or 2)
   int side0;                 // which side comes first: 0 = keys, 1 = values
+  int n_chunks;              // chunks per unit's tile list (see TileWalker)
   int nst;                   // ring stages
   int rmax;                  // larger of the ranks that are projected
 };
@@ -118,36 +119,52 @@ struct WorkTile {
   int unit;     // side slot * Hkv + h: tiles of one unit share a basis
 };
 
-// Walks the tiles [w0, w1) of the work list in order.  pref[b] = tiles of the sequences before b (one head, one
-// side); tiles_all = pref[B]; tile w belongs to unit w / tiles_all.  Positioning costs two divisions and a
-// binary search once; every further step is a few adds, because each role runs this on a single thread and a
-// division per tile would show up in the tile rate.
+// Work list.  A unit is (side, head): its tiles share a basis.  pref[b] = tiles of the sequences before b within
+// one unit, tiles_all = pref[B].  Every unit's tile list is cut into n_chunks contiguous chunks of (almost) equal
+// size; item j is chunk j / n_units of unit j % n_units, and CTA c works through items c, c + n_cta, ...
+// Units vary fastest, so the CTAs that run side by side read the SAME tokens' rows for different heads at about
+// the same time: the 256-byte slices of one 2 KiB token row are then fetched together instead of minutes of DRAM
+// time apart.  The host picks n_chunks so that the items fill whole waves of CTAs.
+// Each role runs a walker on a single thread, so a step is a few adds; divisions happen once per item.
 struct TileWalker {
   const int* pref;
-  int B, Hkv, side0, left;
+  int B, Hkv, side0, tiles_all, n_units, n_chunks, n_cta;
+  int j;                           // current item (>= n_units * n_chunks: past the end)
+  int left;                        // tiles left in the current item
   int unit, side, h, b, k, nb;     // current unit (its side and head), sequence, tile within it, tiles of the sequence
 
-  __device__ __forceinline__ void set_unit(int u) {
-    unit = u;
-    const int slot = u / Hkv;
-    side = slot == 0 ? side0 : 1 - side0;
-    h = u - slot * Hkv;
-  }
-  __device__ void init(const int* pref_, int B_, int Hkv_, int side0_, int tiles_all, int w0, int w1) {
-    pref = pref_; B = B_; Hkv = Hkv_; side0 = side0_;
-    left = w1 - w0;
-    unit = side = h = b = k = 0; nb = 1;
-    if (left <= 0) return;
-    set_unit(w0 / tiles_all);
-    const int rem = w0 - unit * tiles_all;
-    int lo = 0, hi = B;                                   // largest b with pref[b] <= rem
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (pref[mid] <= rem) lo = mid; else hi = mid;
+  __device__ __forceinline__ void load_item() {
+    left = 0;
+    while (j < n_units * n_chunks) {
+      const int u = j % n_units, chunk = j / n_units;
+      const int c0 = (int)((long long)chunk * tiles_all / n_chunks), c1 = (int)((long long)(chunk + 1) * tiles_all / n_chunks);
+      if (c1 > c0) {
+        unit = u;
+        const int slot = u / Hkv;
+        side = slot == 0 ? side0 : 1 - side0;
+        h = u - slot * Hkv;
+        int lo = 0, hi = B;                               // largest b with pref[b] <= c0
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (pref[mid] <= c0) lo = mid; else hi = mid;
+        }
+        b = lo;
+        k = c0 - pref[lo];
+        nb = pref[lo + 1] - pref[lo];
+        left = c1 - c0;
+        return;
+      }
+      j += n_cta;
     }
-    b = lo;
-    k = rem - pref[lo];
-    nb = pref[lo + 1] - pref[lo];
+  }
+  __device__ void init(const int* pref_, int B_, int Hkv_, int side0_, int n_side, int n_chunks_, int cta, int n_cta_) {
+    pref = pref_; B = B_; Hkv = Hkv_; side0 = side0_; n_cta = n_cta_;
+    tiles_all = pref_[B_];
+    n_units = n_side * Hkv_;
+    n_chunks = max(1, min(n_chunks_, tiles_all));
+    unit = side = h = b = k = 0; nb = 1;
+    j = tiles_all > 0 ? cta : n_units * n_chunks;
+    load_item();
   }
   __device__ __forceinline__ bool valid() const { return left > 0; }
   __device__ __forceinline__ WorkTile cur(const int* seq_lens, int T_max) const {
@@ -160,29 +177,26 @@ struct TileWalker {
     return t;
   }
   __device__ __forceinline__ void advance() {
-    if (--left <= 0) return;
+    if (--left <= 0) {
+      j += n_cta;
+      load_item();
+      return;
+    }
     if (++k < nb) return;
     k = 0;
-    do {
-      if (++b == B) {
-        b = 0;
-        set_unit(unit + 1);
-      }
+    do {                                                  // left > 0: a sequence with tiles lies ahead, inside the unit
+      ++b;
       nb = pref[b + 1] - pref[b];
-    } while (nb == 0);                                    // left > 0 guarantees a sequence with tiles ahead
+    } while (nb == 0);
   }
-  // unit of the tile after the current one, or -1 at the end of the range
+  // unit of the tile after the current one, or -1 when the CTA has no further tile
   __device__ __forceinline__ int next_unit() const {
-    if (left <= 1) return -1;
-    if (k + 1 < nb) return unit;
-    int bb = b, uu = unit;
-    do {
-      if (++bb == B) {
-        bb = 0;
-        ++uu;
-      }
-    } while (pref[bb + 1] == pref[bb]);
-    return uu;
+    if (left > 1) return unit;
+    for (int jj = j + n_cta; jj < n_units * n_chunks; jj += n_cta) {
+      const int chunk = jj / n_units;
+      if ((int)((long long)(chunk + 1) * tiles_all / n_chunks) > (int)((long long)chunk * tiles_all / n_chunks)) return jj % n_units;
+    }
+    return -1;
   }
 };
 
@@ -218,6 +232,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
   const PrefillArgs& p = a.p;
   const int B = p.Bt.B, Hkv = p.L.Hkv;
+  launch_dependents();       // the next kernel on the stream may take over each SM as this grid's CTA leaves it
 
   if (tid == 0) {
     for (int s = 0; s < kNST; ++s) {
@@ -256,11 +271,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int tiles_all = pref[B];
-  const long long total = (long long)tiles_all * Hkv * a.n_side;
-  const int per_cta = (int)((total + gridDim.x - 1) / gridDim.x);
-  const long long w_begin = (long long)blockIdx.x * per_cta;
-  const int w0 = (int)min(w_begin, total), w1 = (int)min(w_begin + per_cta, total);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
@@ -270,7 +280,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       tma_prefetch_desc(&tmPK);
       tma_prefetch_desc(&tmPV);
       TileWalker wk;
-      wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+      wk.init(pref, B, Hkv, a.side0, a.n_side, a.n_chunks, blockIdx.x, gridDim.x);
       int s = 0, use = 0;                                  // ring stage and how often it has been used
       for (; wk.valid(); wk.advance()) {
         const int t_side = wk.side, t_h = wk.h, t_b = wk.b, t_t0 = wk.k * kTileM;
@@ -293,7 +303,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       uint32_t idesc = 0;
       int R = 0;
       TileWalker wk;
-      wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+      wk.init(pref, B, Hkv, a.side0, a.n_side, a.n_chunks, blockIdx.x, gridDim.x);
       int s = 0, use = 0;
       for (int i = 0; wk.valid(); wk.advance(), ++i) {
         if (wk.unit != cur_unit) {                         // a new basis: wait until the epilogue warps have staged it
@@ -339,26 +349,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       const __nv_bfloat16* Ub = side ? p.L.U_v : p.L.U_k;
       const __nv_bfloat16* U = Ub + (size_t)h * (side ? p.L.uv_stride : p.L.uk_stride);
       uint8_t* dst = ubuf_ptr + (g & 1) * kUBytes;
-      const int pairs = Rn / 2;
-      for (int idx0 = 0; idx0 < kD * pairs; idx0 += 128 * 8) {
-        uint32_t v[8];
+      // 16-byte pieces (8 columns of one row d of U): all of a thread's loads are issued before the first is used
+      const int ppr = Rn / 8, total = kD * ppr;            // pieces per row; at most 16 pieces per thread
+      uint4 v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int idx = idx0 + u * 128 + et;
-          v[u] = idx < kD * pairs ? __ldg(reinterpret_cast<const uint32_t*>(U) + idx) : 0u;
-        }
+      for (int n = 0; n < 16; ++n) {
+        const int qi = et + n * 128;
+        v[n] = qi < total ? __ldg(reinterpret_cast<const uint4*>(U) + qi) : make_uint4(0u, 0u, 0u, 0u);
+      }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int idx = idx0 + u * 128 + et;
-          if (idx < kD * pairs) {
-            const int d = idx / pairs, j = 2 * (idx % pairs);
-            const int half = d >> 6, piece = (d & 63) >> 3, e = d & 7;
+      for (int n = 0; n < 16; ++n) {
+        const int qi = et + n * 128;
+        if (qi < total) {
+          const int d = qi / ppr, j0 = 8 * (qi - d * ppr);
+          const int half = d >> 6, piece = (d & 63) >> 3, e = d & 7;
+          const uint32_t w[4] = {v[n].x, v[n].y, v[n].z, v[n].w};
 #pragma unroll
-            for (int jj = 0; jj < 2; ++jj) {
-              const int row = j + jj;
-              const uint32_t off = half * (Rn * 128) + (row >> 3) * 1024 + (row & 7) * 128 + ((piece ^ (row & 7)) << 4) + e * 2;
-              *reinterpret_cast<uint16_t*>(dst + off) = (uint16_t)(jj ? (v[u] >> 16) : (v[u] & 0xffffu));
-            }
+          for (int jj = 0; jj < 8; ++jj) {
+            const int row = j0 + jj;                       // rows j0 .. j0+7 share row >> 3 (j0 is a multiple of 8)
+            const uint32_t off = half * (Rn * 128) + (row >> 3) * 1024 + (row & 7) * 128 + ((piece ^ (row & 7)) << 4) + e * 2;
+            *reinterpret_cast<uint16_t*>(dst + off) = (uint16_t)((jj & 1) ? (w[jj >> 1] >> 16) : (w[jj >> 1] & 0xffffu));
           }
         }
       }
@@ -368,7 +378,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     };
 
     TileWalker wk;
-    wk.init(pref, B, Hkv, a.side0, tiles_all, w0, w1);
+    wk.init(pref, B, Hkv, a.side0, a.n_side, a.n_chunks, blockIdx.x, gridDim.x);
     for (int i = 0; wk.valid(); wk.advance(), ++i) {
       const WorkTile t = wk.cur(p.Bt.seq_lens, p.T_max);
       if (t.unit != cur_unit) {
@@ -477,6 +487,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   }
 
   if (warp >= 2 && lane == 0) bulk_wait_all();            // this lane's TMA stores are complete
+  grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -554,12 +565,39 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
   args.rmax = 0;
   if (proj_k) args.rmax = a.L.r_k;
   if (proj_v && a.L.r_v > args.rmax) args.rmax = a.L.r_v;
+  {
+    // items = units x chunks should fill whole waves of CTAs: the fewest waves whose fill is >= 95 %, else the best seen
+    const int n_units = args.n_side * a.L.Hkv, n_cta = sm_count_of_current_device();
+    int best_chunks = 1;
+    double best_fill = 0.0;
+    for (int waves = 1; waves <= 8; ++waves) {
+      const int chunks = waves * n_cta / n_units;
+      if (chunks < 1) continue;
+      const int items = chunks * n_units;
+      const double fill = (double)items / ((double)((items + n_cta - 1) / n_cta) * n_cta);
+      if (fill > best_fill + 1e-9) {
+        best_fill = fill;
+        best_chunks = chunks;
+      }
+      if (fill >= 0.95) break;
+    }
+    args.n_chunks = best_chunks;
+  }
   args.nst = kMaxNST;
   while (args.nst > 2 && smem_bytes(args.nst, args.rmax, a.Bt.B) > kSmemLimit) --args.nst;
   const int smem = smem_bytes(args.nst, args.rmax, a.Bt.B);
   if (smem > kSmemLimit) return cudaErrorInvalidValue;
-  prefill_tc_kernel<<<sm_count_of_current_device(), kThreads, smem, st>>>(tmK, tmV, tmPK, tmPV, args);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(sm_count_of_current_device());
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.overlap_previous ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, tmK, tmV, tmPK, tmPV, args);
 }
 
 }  // namespace stief

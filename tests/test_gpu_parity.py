@@ -272,6 +272,36 @@ def test_overlapped_launches_match_serial_ones():
     U.check_out(res[1][7], ref)
 
 
+def test_overlapped_prefill_launches_match_serial_ones():
+    # the per-layer prefill launches of one prompt, enqueued back to back with STIEF_PREFILL_OVERLAP_PREVIOUS
+    B, Hq, Hkv = 2, 8, 2
+    ranks = [(64, 64), (32, 128), (96, 48), (128, 32)]
+    cs = [U.make_case(95 + l, B, Hq, Hkv, rk, rv, [1000, 333]) for l, (rk, rv) in enumerate(ranks)]
+    Kd = [c.K.cuda() for c in cs]
+    Vd = [c.V.cuda() for c in cs]
+    pools = {}
+    for flags in (0, S.STIEF_PREFILL_OVERLAP_PREVIOUS):
+        for c in cs:
+            c.layer.k_pool.view(torch.int16).fill_(U.NAN_BITS)
+            c.layer.v_pool.view(torch.int16).fill_(U.NAN_BITS)
+        torch.cuda.synchronize()
+        for c, K, V in zip(cs, Kd, Vd):
+            S.stief_prefill_compress(c.layer, c.batch, K, V, status=c.status, flags=flags)
+        torch.cuda.synchronize()
+        assert all(int(c.status.item()) == 0 for c in cs)
+        pools[flags] = [(c.layer.k_pool.clone(), c.layer.v_pool.clone()) for c in cs]
+    for (k0, v0), (k1, v1) in zip(pools[0], pools[1]):
+        assert torch.equal(k0.view(torch.int16), k1.view(torch.int16)) and torch.equal(v0.view(torch.int16), v1.view(torch.int16))
+    for c in cs:                         # and the overlapped result against the oracle
+        Kr, Vr = U.oracle_cache(c)
+        for b in range(B):
+            n = int(c.seq_lens[b])
+            gk = U.gpu_cache_rows(c, c.layer.k_pool, b, n)
+            for h in range(Hkv):
+                U.check_cache(gk[:, h], U.f64(c.K)[b, :n, h], O.basis_of(U.f64(c.U_k), h), Kr[b][:, h])
+        _untouched_rows_still_nan(c)
+
+
 def test_host_staged_step():
     B, Hq, Hkv = 2, 8, 2
     c = U.make_case(60, B, Hq, Hkv, 64, 64, [100, 70], reserve=4)
