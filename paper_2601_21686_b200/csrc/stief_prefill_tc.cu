@@ -8,9 +8,10 @@
 //   warp 1      MMA: allocates TMEM, and one lane issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32,
 //               M = 128, N = r, 8 instructions of K = 16 per tile) from shared-memory descriptors into one of
 //               two TMEM accumulators; tcgen05.commit frees the ring stage and publishes the accumulator.
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = token row), round to bf16, 16-byte stores to the
-//               paged pool; they also bring the basis into shared memory, transposed to the K-major swizzled
-//               layout the MMA wants, one buffer ahead of the MMA warp.
+//   warps 2..9  epilogue, two groups of four warps that take alternate tiles (group g owns accumulator g):
+//               tcgen05.ld the accumulator (lane = token row), round to bf16 into a swizzled staging box, TMA
+//               store to the paged pool.  The first group also brings the basis into shared memory, transposed
+//               to the K-major swizzled layout the MMA wants, one buffer ahead of the MMA warp.
 // Work is the list of valid tiles ordered (side, head, sequence, tile) and cut into equal contiguous ranges,
 // so a CTA changes basis at most a couple of times.  The projection is HBM-bound (about 43-64 flop per byte
 // against a ridge near 250): the tensor pipe idles most of the time by construction, and what matters is that
@@ -29,13 +30,13 @@ constexpr int kTileM = 128;                       // tokens per tile
 constexpr int kMaxNST = 4;                        // ring stages (3 when rank 128 and a large batch leave no room)
 constexpr int kStageBytes = kTileM * kD * 2;      // 32 KiB: two halves of 128 rows x 128 bytes
 constexpr int kHalfBytes = kStageBytes / 2;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                     // producer warp, MMA warp, two epilogue groups of four warps
 constexpr int kTmemCols = 256;                    // two accumulators of up to 128 fp32 columns
 constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;                // 227 KiB per CTA
 
 // Shared memory, from a 1024-byte aligned base: ring [nst][32 KiB] | two basis buffers [rmax * 256] |
-// output staging [4 warps][32 rows][rmax * 2] | barriers and flags | tile prefix sums [B + 1].
+// output staging [8 warps][32 rows][rmax * 2] | barriers and flags | tile prefix sums [B + 1].
 
 struct Args {
   PrefillArgs p;
@@ -204,6 +205,43 @@ struct TileWalker {
 
 using namespace tc;
 
+// Brings one basis U [128][Rn] (bf16, row-major) into shared memory as the K-major operand the MMA reads:
+// element (d, j) of U goes to row j, 64-element half d / 64, 16-byte piece ((d % 64) / 8) ^ (j % 8) of the
+// 128-byte row.  Called by the 128 threads of the first epilogue group (et = 0..127); each warp's lane 0 then
+// arrives on `ready_bar`.
+__device__ __forceinline__ void stage_basis(const __nv_bfloat16* __restrict__ U, int Rn, uint8_t* dst, uint32_t ready_bar, int et, int lane) {
+  // 16-byte pieces (8 columns of one row d of U), at most 16 per thread, fetched in one or two rounds of
+  // independent loads
+  const int ppr = Rn / 8, total = kD * ppr;            // pieces per row, pieces in all
+#pragma unroll 1
+  for (int n0 = 0; n0 < 16 && n0 * 128 < total; n0 += 8) {
+  uint4 v[8];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const int qi = et + (n0 + n) * 128;
+    v[n] = qi < total ? __ldg(reinterpret_cast<const uint4*>(U) + qi) : make_uint4(0u, 0u, 0u, 0u);
+  }
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const int qi = et + (n0 + n) * 128;
+    if (qi < total) {
+      const int d = qi / ppr, j0 = 8 * (qi - d * ppr);
+      const int half = d >> 6, piece = (d & 63) >> 3, e = d & 7;
+      const uint32_t w[4] = {v[n].x, v[n].y, v[n].z, v[n].w};
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int row = j0 + jj;                       // rows j0 .. j0+7 share row >> 3 (j0 is a multiple of 8)
+        const uint32_t off = half * (Rn * 128) + (row >> 3) * 1024 + (row & 7) * 128 + ((piece ^ (row & 7)) << 4) + e * 2;
+        *reinterpret_cast<uint16_t*>(dst + off) = (uint16_t)((jj & 1) ? (w[jj >> 1] >> 16) : (w[jj >> 1] & 0xffffu));
+      }
+    }
+  }
+  }
+  fence_proxy_async_smem();                                // generic-proxy writes -> visible to the tensor core's reads
+  __syncwarp();
+  if (lane == 0) mbar_arrive(ready_bar);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmPK, const __grid_constant__ CUtensorMap tmPV, const Args a) {
@@ -219,8 +257,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   uint8_t* ubuf_ptr = base_ptr + kNST * kStageBytes;
   const uint32_t obuf = ubuf + 2 * kUBytes;                     // output staging, one region per epilogue warp
   uint8_t* obuf_ptr = ubuf_ptr + 2 * kUBytes;
-  const uint32_t ctrl = obuf + 4 * kOutBytes;
-  uint8_t* ctrl_ptr = obuf_ptr + 4 * kOutBytes;
+  const uint32_t ctrl = obuf + 8 * kOutBytes;
+  uint8_t* ctrl_ptr = obuf_ptr + 8 * kOutBytes;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (8 + s) * 8; };
   auto acc_full = [&](int i) { return ctrl + (16 + i) * 8; };
@@ -336,152 +374,120 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue warps (2..5)
+    // ------------------------------------------------------------------ epilogue warps (2..9)
     const int q = warp & 3;                                // TMEM lane quarter this warp may read
-    const int et = tid - 64;                               // 0..127
+    const int grp = (warp - 2) >> 2;                       // group 0 takes the even tiles of the CTA, group 1 the odd ones
+    const int et = tid - 64;                               // 0..127 inside group 0, which stages the bases
     int cur_unit = -1, gen = -1;
     int R = 0;
 
-    // Stage the basis of `unit` in buffer gen & 1: element (d, j) of U goes to row j of the K-major operand,
-    // 64-element half d / 64, 16-byte piece ((d % 64) / 8) ^ (j % 8) of the 128-byte row.
-    auto stage_basis = [&](int side, int h, int g) {
-      const int Rn = side ? p.L.r_v : p.L.r_k;
+    auto stage_basis_of = [&](int side, int h, int g) {
       const __nv_bfloat16* Ub = side ? p.L.U_v : p.L.U_k;
-      const __nv_bfloat16* U = Ub + (size_t)h * (side ? p.L.uv_stride : p.L.uk_stride);
-      uint8_t* dst = ubuf_ptr + (g & 1) * kUBytes;
-      // 16-byte pieces (8 columns of one row d of U): all of a thread's loads are issued before the first is used
-      const int ppr = Rn / 8, total = kD * ppr;            // pieces per row; at most 16 pieces per thread
-      uint4 v[16];
-#pragma unroll
-      for (int n = 0; n < 16; ++n) {
-        const int qi = et + n * 128;
-        v[n] = qi < total ? __ldg(reinterpret_cast<const uint4*>(U) + qi) : make_uint4(0u, 0u, 0u, 0u);
-      }
-#pragma unroll
-      for (int n = 0; n < 16; ++n) {
-        const int qi = et + n * 128;
-        if (qi < total) {
-          const int d = qi / ppr, j0 = 8 * (qi - d * ppr);
-          const int half = d >> 6, piece = (d & 63) >> 3, e = d & 7;
-          const uint32_t w[4] = {v[n].x, v[n].y, v[n].z, v[n].w};
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const int row = j0 + jj;                       // rows j0 .. j0+7 share row >> 3 (j0 is a multiple of 8)
-            const uint32_t off = half * (Rn * 128) + (row >> 3) * 1024 + (row & 7) * 128 + ((piece ^ (row & 7)) << 4) + e * 2;
-            *reinterpret_cast<uint16_t*>(dst + off) = (uint16_t)((jj & 1) ? (w[jj >> 1] >> 16) : (w[jj >> 1] & 0xffffu));
-          }
-        }
-      }
-      fence_proxy_async_smem();                            // generic-proxy writes -> visible to the tensor core's reads
-      __syncwarp();
-      if (lane == 0) mbar_arrive(u_ready(g & 1));
+      stage_basis(Ub + (size_t)h * (side ? p.L.uv_stride : p.L.uk_stride), side ? p.L.r_v : p.L.r_k,
+                  ubuf_ptr + (g & 1) * kUBytes, u_ready(g & 1), et, lane);
     };
 
     TileWalker wk;
     wk.init(pref, B, Hkv, a.side0, a.n_side, a.n_chunks, blockIdx.x, gridDim.x);
+    if (grp == 0 && wk.valid()) stage_basis_of(wk.side, wk.h, ++gen);      // the basis of the CTA's first tile
     for (int i = 0; wk.valid(); wk.advance(), ++i) {
+      const bool mine = (i & 1) == grp;
+      if (wk.unit != cur_unit) {
+        cur_unit = wk.unit;
+        R = wk.side ? p.L.r_v : p.L.r_k;
+      }
+      // Group 0 stages the next basis one buffer ahead.  That buffer was last read by the MMAs of the unit before
+      // the current one, which ended at a tile <= i - 1; they are known to be complete once this group has seen
+      // the accumulator of a tile >= that one: its own tile i (then stage after the wait below), else tile i - 1.
+      const int nu = grp == 0 ? wk.next_unit() : -1;
+      const bool stage_next = nu >= 0 && nu != cur_unit;
       const WorkTile t = wk.cur(p.Bt.seq_lens, p.T_max);
-      if (t.unit != cur_unit) {
-        if (gen < 0) stage_basis(t.side, t.h, ++gen);      // first tile of the CTA
-        cur_unit = t.unit;
-        R = t.side ? p.L.r_v : p.L.r_k;
-      }
-      {                                                    // stage the next basis one buffer ahead
-        const int nu = wk.next_unit();
-        if (nu >= 0 && nu != cur_unit) {
-          const int slot = nu / Hkv;
-          stage_basis(slot == 0 ? a.side0 : 1 - a.side0, nu - slot * Hkv, ++gen);
-        }
-      }
       // the page of this warp's 32 tokens: fetched before the wait so its latency hides behind the accumulator's
       const int tok0 = t.t0 + 32 * q;                      // the warp's first token; its 32 tokens share a page
       int page = -1;
-      if (lane == 0 && tok0 < t.len && tok0 / kPage < p.Bt.max_pages)
+      if (mine && lane == 0 && tok0 < t.len && tok0 / kPage < p.Bt.max_pages)
         page = p.Bt.block_table[(size_t)t.b * p.Bt.max_pages + tok0 / kPage];
 
       const int acc = i & 1;
-      mbar_wait(acc_full(acc), (i >> 1) & 1, abort_flag, p.status);
-      tc_fence_after();
-
-      // ---- the warp's 32 rows of the accumulator -> registers (all loads in flight, one wait)
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + acc * 128;
-      uint32_t v[8][16];
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        if (c < R / 16) tmem_ld16(taddr + c * 16, v[c]);
-      tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty(acc));          // this warp has read its quarter of the accumulator
-
-      if (tok0 >= t.len) continue;
-      page = __shfl_sync(0xffffffffu, page, 0);
-      if (page < 0 || page >= p.L.num_pages) {
-        if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
-        continue;
-      }
-      const int row0 = (page * Hkv + t.h) * kPage + (tok0 % kPage);          // pool row of the warp's first token
-      if (tok0 + 32 <= t.len) {
-        // ---- all 32 rows valid: round to bf16 into the swizzled staging boxes, then TMA stores.  A box is 32
+      if (mine) {
+        mbar_wait(acc_full(acc), (i >> 1) & 1, abort_flag, p.status);
+        tc_fence_after();
+        // where the warp's 32 rows go
+        bool valid = tok0 < t.len;
+        page = __shfl_sync(0xffffffffu, page, 0);
+        if (valid && (page < 0 || page >= p.L.num_pages)) {
+          if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
+          valid = false;
+        }
+        const bool full = valid && tok0 + 32 <= t.len;     // else the sequence ends inside these rows
+        const int row0 = (max(page, 0) * Hkv + t.h) * kPage + (tok0 % kPage);  // pool row of the warp's first token
+        // full case: rows are rounded to bf16 into swizzled staging boxes and leave by TMA stores.  A box is 32
         // rows x BW elements (BW = 64, 32 or 16: the largest that divides R), swizzle span = box row.
-        const int lbw = (R % 64 == 0) ? 6 : (R % 32 == 0) ? 5 : 4;       // log2 of the box width
+        const int lbw = (R % 64 == 0) ? 6 : (R % 32 == 0) ? 5 : 4;             // log2 of the box width
         const int BW = 1 << lbw, RB = BW * 2, CPB = BW / 8;
         const uint32_t wbase = obuf + (warp - 2) * kOutBytes;
         uint8_t* wptr = obuf_ptr + (warp - 2) * kOutBytes;
-        if (lane == 0) bulk_wait_read_all();               // the previous tile's stores have left the staging region
-        __syncwarp();
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (c < R / 16) {
-            uint4 o[2];
-            o[0].x = pack_bf16(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]));
-            o[0].y = pack_bf16(__uint_as_float(v[c][2]), __uint_as_float(v[c][3]));
-            o[0].z = pack_bf16(__uint_as_float(v[c][4]), __uint_as_float(v[c][5]));
-            o[0].w = pack_bf16(__uint_as_float(v[c][6]), __uint_as_float(v[c][7]));
-            o[1].x = pack_bf16(__uint_as_float(v[c][8]), __uint_as_float(v[c][9]));
-            o[1].y = pack_bf16(__uint_as_float(v[c][10]), __uint_as_float(v[c][11]));
-            o[1].z = pack_bf16(__uint_as_float(v[c][12]), __uint_as_float(v[c][13]));
-            o[1].w = pack_bf16(__uint_as_float(v[c][14]), __uint_as_float(v[c][15]));
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int col = 16 * c + 8 * e;              // first of the 8 columns in this 16-byte piece
-              const int nb = col >> lbw, cc = (col & (BW - 1)) >> 3;
-              uint32_t off = (uint32_t)(lane * RB + cc * 16);
-              off ^= ((off >> 7) & (uint32_t)(CPB - 1)) << 4;
-              *reinterpret_cast<uint4*>(wptr + ((nb * 32) << (lbw + 1)) + off) = o[e];
-            }
-          }
-        }
-        fence_proxy_async_smem();                          // generic-proxy writes -> visible to the TMA store
-        __syncwarp();
-        if (lane == 0) {
-          const CUtensorMap* tmP = t.side ? &tmPV : &tmPK;
-          for (int nb = 0; nb < (R >> lbw); ++nb) tma_store_2d(tmP, nb * BW, row0, wbase + nb * 32 * RB);
-          bulk_commit_group();
-        }
-      } else {
-        // ---- the sequence ends inside these 32 rows: rows at or beyond its length must stay untouched
-        const int tok = tok0 + lane;
         __nv_bfloat16* pool = t.side ? p.L.v_pool : p.L.k_pool;
-        uint4* dst = reinterpret_cast<uint4*>(pool + ((size_t)row0 + lane) * R);
-        if (tok < t.len) {
+        uint4* dst = reinterpret_cast<uint4*>(pool + ((size_t)row0 + lane) * R);   // partial case: direct stores
+        const bool row_ok = valid && tok0 + lane < t.len;
+        if (full) {
+          if (lane == 0) bulk_wait_read_all();             // the previous tile's stores have left the staging region
+          __syncwarp();
+        }
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + acc * 128;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            if (c < R / 16) {
-              uint4 o0, o1;
-              o0.x = pack_bf16(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]));
-              o0.y = pack_bf16(__uint_as_float(v[c][2]), __uint_as_float(v[c][3]));
-              o0.z = pack_bf16(__uint_as_float(v[c][4]), __uint_as_float(v[c][5]));
-              o0.w = pack_bf16(__uint_as_float(v[c][6]), __uint_as_float(v[c][7]));
-              o1.x = pack_bf16(__uint_as_float(v[c][8]), __uint_as_float(v[c][9]));
-              o1.y = pack_bf16(__uint_as_float(v[c][10]), __uint_as_float(v[c][11]));
-              o1.z = pack_bf16(__uint_as_float(v[c][12]), __uint_as_float(v[c][13]));
-              o1.w = pack_bf16(__uint_as_float(v[c][14]), __uint_as_float(v[c][15]));
-              dst[2 * c] = o0;
-              dst[2 * c + 1] = o1;
+        for (int c0 = 0; c0 < 8; c0 += 4) {                // two batches of up to 64 columns keep the live registers down
+          if (c0 * 16 < R) {
+            uint32_t v[4][16];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if ((c0 + c) * 16 < R) tmem_ld16(taddr + (c0 + c) * 16, v[c]);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if ((c0 + c) * 16 < R) {
+                uint4 o[2];
+                o[0].x = pack_bf16(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]));
+                o[0].y = pack_bf16(__uint_as_float(v[c][2]), __uint_as_float(v[c][3]));
+                o[0].z = pack_bf16(__uint_as_float(v[c][4]), __uint_as_float(v[c][5]));
+                o[0].w = pack_bf16(__uint_as_float(v[c][6]), __uint_as_float(v[c][7]));
+                o[1].x = pack_bf16(__uint_as_float(v[c][8]), __uint_as_float(v[c][9]));
+                o[1].y = pack_bf16(__uint_as_float(v[c][10]), __uint_as_float(v[c][11]));
+                o[1].z = pack_bf16(__uint_as_float(v[c][12]), __uint_as_float(v[c][13]));
+                o[1].w = pack_bf16(__uint_as_float(v[c][14]), __uint_as_float(v[c][15]));
+                if (full) {
+#pragma unroll
+                  for (int e = 0; e < 2; ++e) {
+                    const int col = 16 * (c0 + c) + 8 * e; // first of the 8 columns in this 16-byte piece
+                    const int nb = col >> lbw, cc = (col & (BW - 1)) >> 3;
+                    uint32_t off = (uint32_t)(lane * RB + cc * 16);
+                    off ^= ((off >> 7) & (uint32_t)(CPB - 1)) << 4;
+                    *reinterpret_cast<uint4*>(wptr + ((nb * 32) << (lbw + 1)) + off) = o[e];
+                  }
+                } else if (row_ok) {                       // rows at or beyond the sequence length stay untouched
+                  dst[2 * (c0 + c)] = o[0];
+                  dst[2 * (c0 + c) + 1] = o[1];
+                }
+              }
             }
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty(acc));        // this warp has read its quarter of the accumulator
+        if (full) {
+          fence_proxy_async_smem();                        // generic-proxy writes -> visible to the TMA store
+          __syncwarp();
+          if (lane == 0) {
+            const CUtensorMap* tmP = t.side ? &tmPV : &tmPK;
+            for (int nb = 0; nb < (R >> lbw); ++nb) tma_store_2d(tmP, nb * BW, row0, wbase + nb * 32 * RB);
+            bulk_commit_group();
+          }
+        }
+      }
+      if (stage_next) {
+        const int slot = nu / Hkv;
+        stage_basis_of(slot == 0 ? a.side0 : 1 - a.side0, nu - slot * Hkv, ++gen);
       }
     }
   }
@@ -528,7 +534,7 @@ bool make_pool_store_map(CUtensorMap* tm, const void* pool, int r, const Prefill
 }
 
 int smem_bytes(int nst, int rmax, int B) {
-  return 1024 + nst * kStageBytes + 2 * rmax * 256 + 4 * 32 * rmax * 2 + kCtrlBytes + ((B + 1) * 4 + 127) / 128 * 128;
+  return 1024 + nst * kStageBytes + 2 * rmax * 256 + 8 * 32 * rmax * 2 + kCtrlBytes + ((B + 1) * 4 + 127) / 128 * 128;
 }
 
 }  // namespace
