@@ -35,13 +35,29 @@ import torch
 
 SEED = 0
 CFG2 = dict(B=4, Hq=32, Hkv=8, T=32768, r_k=64, r_v=64)
+# single-layer decode workloads that share the config-2 harness (the headline line is config 2)
+SINGLE_LAYER = {
+    "config2": dict(CFG2, name="config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64"),
+    "config4a": dict(B=1, Hq=32, Hkv=8, T=131072, r_k=48, r_v=64,
+                     name="config4a: one long sequence, B=1 Hq=32 Hkv=8 d=128 T=131072 r_k=48 r_v=64"),
+    "config4b": dict(B=16, Hq=32, Hkv=8, T=16384, r_k=64, r_v=64, ragged=True,
+                     name="config4b: ragged batch, B=16 Hq=32 Hkv=8 d=128 lengths uniform in [1024,16384] r_k=r_v=64"),
+}
 N_CACHES = 4               # rotating layer caches (each 256 MiB of compressed rows)
 METRIC = "decode_attn_effective_hbm_gbs"
 UNIT = "GB/s"
 
 
+def seq_lengths(cfg):
+    from paper_2601_21686_b200 import inputs as I
+    if cfg.get("ragged"):
+        return [int(x) for x in I.ragged_lengths(SEED, cfg["B"])]
+    return [cfg["T"]] * cfg["B"]
+
+
 def step_bytes(cfg) -> int:
-    return cfg["B"] * cfg["Hkv"] * (cfg["T"] + 1) * 2 * (cfg["r_k"] + cfg["r_v"])
+    """Compressed-cache bytes one decode step must read: every cached row of every KV head, new token included."""
+    return sum(n + 1 for n in seq_lengths(cfg)) * cfg["Hkv"] * 2 * (cfg["r_k"] + cfg["r_v"])
 
 
 def measured_peaks():
@@ -115,12 +131,14 @@ class ClockSampler:
 def build_caches(cfg, n_caches, dev, S, I):
     """n_caches independent layer caches, filled by the library's prefill kernel from seeded K, V."""
     B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
-    pg = I.make_paging(SEED, [T] * B, reserve_tokens=1)
+    lens = seq_lengths(cfg)
+    T = max(lens)
+    pg = I.make_paging(SEED, lens, reserve_tokens=1)
     bt = torch.from_numpy(pg.block_table).to(dev)
     lens = torch.from_numpy(pg.seq_lens).to(dev)
     batch = S.Batch(bt, lens)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    layers, prefill_ms = [], []
+    layers, inputs = [], []
     for l in range(n_caches):
         U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
         layer = S.Layer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev),
@@ -128,16 +146,23 @@ def build_caches(cfg, n_caches, dev, S, I):
                         torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.bfloat16, device=dev))
         K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
         V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        S.stief_prefill_compress(layer, batch, K, V, status=status)      # warm-up (also the real fill)
-        torch.cuda.synchronize()
-        e0.record()
-        S.stief_prefill_compress(layer, batch, K, V, status=status)
-        e1.record()
-        torch.cuda.synchronize()
-        prefill_ms.append(e0.elapsed_time(e1))
+        S.stief_prefill_compress(layer, batch, K, V, status=status)      # the real fill (and a warm-up)
         layers.append(layer)
-        del K, V
+        inputs.append((K, V))
+    torch.cuda.synchronize()
+    # timed: the per-layer launches of one prompt back to back (different inputs and pools per layer, each layer's
+    # inputs larger than L2), overlapped the way a 32-layer prefill would launch them
+    reps = 3
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for r in range(reps):
+        for l in range(n_caches):
+            S.stief_prefill_compress(layers[l], batch, inputs[l][0], inputs[l][1], status=status,
+                                     flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if (r or l) else 0)
+    e1.record()
+    torch.cuda.synchronize()
+    prefill_ms = [e0.elapsed_time(e1) / (reps * n_caches)]
+    del inputs
     assert int(status.item()) == 0, f"device status {int(status.item())} while building the cache"
     return layers, batch, status, prefill_ms
 
@@ -163,7 +188,10 @@ def run_ours(args):
         dist.barrier()
     S.lib()
 
-    cfg = dict(CFG2)
+    cfg = dict(SINGLE_LAYER[args.workload])
+    if args.ranks:                                   # a variant of the workload at other ranks (not the headline)
+        cfg["r_k"], cfg["r_v"] = (int(x) for x in args.ranks.split(","))
+        cfg["name"] += f" [ranks overridden: r_k={cfg['r_k']} r_v={cfg['r_v']}]"
     n_caches = args.caches
     B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
     layers, batch, status, prefill_ms = build_caches(cfg, n_caches, dev, S, I)
@@ -269,27 +297,28 @@ def run_ours(args):
         e2e = world * sb * K_steps / (ms_host * 1e-3) / 1e9
         achieved = sb / (kern_avg_ms * 1e-3) / 1e9
         pf_ms = float(np.median(prefill_ms))
-        pf_bytes = B * T * Hkv * (2 * 128 * 2 + 2 * (r_k + r_v))
-        pf_flops = 2.0 * B * T * Hkv * 128 * (r_k + r_v)
+        n_tok = sum(seq_lengths(cfg))
+        pf_bytes = n_tok * Hkv * (2 * 128 * 2 + 2 * (r_k + r_v))
+        pf_flops = 2.0 * n_tok * Hkv * 128 * (r_k + r_v)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 cache, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": "config2: Llama3-8B-shaped single-layer decode, B=4 Hq=32 Hkv=8 d=128 T=32768 r_k=r_v=64, "
-                                   "64-token pages, shuffled block tables; step = append + query projection + split-T attention + combine, one launch",
+            "config": {"workload": cfg["name"] + ", 64-token pages, shuffled block tables; step = append + query projection + "
+                                   "split-T attention + combine, one launch",
                        "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_parts": ns,
                        "launch": ("programmatic dependent launch: each step's kernel may start while the previous step's drains"
                                   if overlap else "serialised launches"),
                        "l2": f"steps rotate over {n_caches} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
                        "parallelism": f"replicas x{world} (independent batches, no collective)"},
-            "tokens_per_s": world * B * K_steps / (ms * 1e-3),
+            "tokens_per_s": world * B * K_steps / (ms * 1e-3), "seq_lens": seq_lengths(cfg) if cfg.get("ragged") else None,
             "frac_of_hbm_peak": value / world / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
             "frac_of_hbm_spec_8000": value / world / 8000.0,
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
                     "tokens_per_s": world * B * K_steps / (ms_host * 1e-3)},
             "gpu_launches": K_steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel<64,64>", "achieved": achieved, "peak": hbm_peak,
+            "roofline": {"bound": "hbm", "kernel": f"decode_persistent_kernel<{r_k},{r_v}>", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": peak_kind, "traffic": args.traffic,
                          "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms,
                          "isolated_launch_ms": kern_isolated_ms, "isolated_min_launch_ms": float(min(kern_ms)),
@@ -299,7 +328,9 @@ def run_ours(args):
                                 "frac_of_hbm_peak": sb * K_steps / (ms_serial * 1e-3) / 1e9 / hbm_peak},
             "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak,
                         "tflops": pf_flops / (pf_ms * 1e-3) / 1e12, "frac_of_bf16_peak": pf_flops / (pf_ms * 1e-3) / 1e12 / tf_peak,
-                        "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache, one layer"},
+                        "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache; per-layer time over back-to-back "
+                                    f"overlapped launches on {n_caches} layers",
+                        "kernel": "prefill_tc_kernel (TMA + tcgen05/TMEM)", "bound": "hbm"},
             "clocks": sampler.summary(t0, time.time()),
         }
         if not args.no_cpu_baseline and world == 1:
@@ -308,6 +339,148 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# the 32-layer workloads: config 3 (decode steps over per-layer ranks) and config 5 (prefill + first decode)
+# ------------------------------------------------------------------------------------------------
+def run_multilayer(args):
+    import paper_2601_21686_b200 as S
+    from paper_2601_21686_b200 import inputs as I
+    from paper_2601_21686_b200 import build as Bld
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("the multi-layer workloads run on one GPU")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Bld.build()
+    S.lib()
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    Hq, Hkv, T, L = 32, 8, 32768, args.layers
+    B = 4 if args.workload == "config3" else 2
+    n_steps = args.steps if args.workload == "config3" else 1
+    prof = I.rank_profile(SEED)[:L]
+    pg = I.make_paging(SEED, [T] * B, reserve_tokens=max(n_steps, 1) + 1)
+    bt = torch.from_numpy(pg.block_table).to(dev)
+    lens = torch.from_numpy(pg.seq_lens).to(dev)
+    batch = S.Batch(bt, lens)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    layers, inputs = [], []
+    for l, (r_k, r_v) in enumerate(prof):
+        U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
+        layers.append(S.Layer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev),
+                              torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.bfloat16, device=dev),
+                              torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.bfloat16, device=dev)))
+        K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
+        V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
+        if args.workload == "config5":
+            inputs.append((K, V))                 # all 32 layers' prompts stay resident (8.6 GB) for the timed prefill
+        else:
+            S.stief_prefill_compress(layers[l], batch, K, V, status=status)
+            del K, V
+    torch.cuda.synchronize()
+    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, Hkv, 128, 0) // 4, dtype=torch.float32, device=dev)
+    S.stief_decode_workspace_init(ws)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    n_in = 4
+    qs = [[I.queries(SEED, l, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for l in range(L)] for i in range(n_in)]
+    kvs = [[I.new_token_kv(SEED, l, B, Hkv, device=dev, step=i) for l in range(L)] for i in range(n_in)]
+    ov = S.STIEF_DECODE_OVERLAP_PREVIOUS
+
+    def decode_step(i):
+        """One token for every sequence: append + attention in every layer, then advance the lengths."""
+        for l in range(L):
+            k_new, v_new = kvs[i % n_in][l]
+            S.stief_decode_step(layers[l], batch, qs[i % n_in][l], k_new, v_new, ws, out, status=status, flags=ov if l else 0)
+        S.stief_advance_seq_lens(lens, 1)
+
+    cache_bytes_per_token = sum(Hkv * 2 * (rk + rv) for rk, rv in prof)      # per cached token, all layers
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    t0 = time.time()
+    line = {"n_gpus": 1, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
+            "dtype": "bf16 cache, fp32 accumulate", "rank_profile": prof, "peak_kind": peak_kind, "hbm_peak_gbs": hbm_peak}
+    if args.workload == "config3":
+        W = 3
+        for i in range(W):
+            decode_step(i)
+        lens.copy_(torch.from_numpy(pg.seq_lens).to(dev))          # the timed steps start from T again
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n_steps):
+            decode_step(W + i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_eager = e0.elapsed_time(e1)
+        # the same step replayed from a CUDA graph (the lengths advance on the device, so one captured step serves
+        # every position): removes the host's per-launch cost, which the small-rank layers cannot hide
+        lens.copy_(torch.from_numpy(pg.seq_lens).to(dev))
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cap_stream):
+            with torch.cuda.graph(graph, stream=cap_stream):
+                decode_step(0)
+        torch.cuda.synchronize()
+        for i in range(W):
+            graph.replay()
+        lens.copy_(torch.from_numpy(pg.seq_lens).to(dev))
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(n_steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        byt = sum(B * (T + s + 1) * cache_bytes_per_token for s in range(n_steps))
+        gbs = byt / (ms * 1e-3) / 1e9
+        line.update({"eager_launches": {"ms_per_step": ms_eager / n_steps, "value": byt / (ms_eager * 1e-3) / 1e9, "unit": UNIT,
+                                        "tokens_per_s": B * n_steps / (ms_eager * 1e-3)},
+                     "launch": "one captured CUDA graph per step (32 decode launches + the length update), replayed"})
+        line.update({"metric": METRIC, "value": gbs, "unit": UNIT, "steps": n_steps, "warmup": W, "ms_per_step": ms / n_steps,
+                     "tokens_per_s": B * n_steps / (ms * 1e-3), "frac_of_hbm_peak": gbs / hbm_peak,
+                     "gpu_launches": n_steps * (L + 1), "bytes_per_step_first": B * (T + 1) * cache_bytes_per_token,
+                     "config": {"workload": f"config3: {L}-layer decode step, per-layer ranks from the seeded profile, B={B} Hq={Hq} "
+                                            f"Hkv={Hkv} d=128 T={T} growing by one token per step; step = for every layer append + "
+                                            "attention (one launch each, overlapped within a step), then advance the lengths",
+                                "global_batch": B, "seq_len": T, "l2": "a step streams 9.9 GB of cache: nothing survives in L2"}})
+    else:
+        pf = S.STIEF_PREFILL_OVERLAP_PREVIOUS
+        for l in range(min(4, L)):                # warm-up on a few layers (they are rewritten below)
+            S.stief_prefill_compress(layers[l], batch, inputs[l][0], inputs[l][1], status=status)
+        decode_step(0)                            # loads every decode kernel variant; its rows are rewritten below
+        lens.copy_(torch.from_numpy(pg.seq_lens).to(dev))
+        torch.cuda.synchronize()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        for l in range(L):
+            S.stief_prefill_compress(layers[l], batch, inputs[l][0], inputs[l][1], status=status, flags=pf if l else 0)
+        e1.record()
+        decode_step(0)
+        e2.record()
+        torch.cuda.synchronize()
+        ms_pf, ms_dec = e0.elapsed_time(e1), e1.elapsed_time(e2)
+        byt = sum(B * T * Hkv * (512 + 2 * (rk + rv)) for rk, rv in prof)
+        flops = sum(2.0 * B * T * Hkv * 128 * (rk + rv) for rk, rv in prof)
+        gbs = byt / (ms_pf * 1e-3) / 1e9
+        line.update({"metric": "prefill_compress_effective_hbm_gbs", "value": gbs, "unit": UNIT, "steps": 1, "warmup": 1,
+                     "ms_per_step": ms_pf, "ms_per_layer": ms_pf / L, "frac_of_hbm_peak": gbs / hbm_peak,
+                     "tflops": flops / (ms_pf * 1e-3) / 1e12, "frac_of_bf16_peak": flops / (ms_pf * 1e-3) / 1e12 / tf_peak,
+                     "prompt_tokens_per_s": B * T / (ms_pf * 1e-3), "gpu_launches": L,
+                     "first_decode_step": {"ms": ms_dec, "gbs": B * (T + 1) * cache_bytes_per_token / (ms_dec * 1e-3) / 1e9},
+                     "config": {"workload": f"config5: prefill compression of a {L}-layer prompt, K,V [B={B},T={T},Hkv={Hkv},128] bf16 per "
+                                            "layer -> paged cache with per-layer ranks (one overlapped launch per layer), then the first decode step",
+                                "global_batch": B, "seq_len": T, "l2": "every layer has its own 268 MB of inputs"}})
+    torch.cuda.synchronize()
+    sampler.stop()
+    line["clocks"] = sampler.summary(t0, time.time())
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -355,7 +528,7 @@ def _threads_used() -> int:
 def cpu_baseline(cfg, seconds_budget=20.0):
     n_seq = 1
     O, I, Kd, Vd, U_k, U_v = _oracle_sample(cfg, n_seq)
-    sb = step_bytes(cfg) * n_seq // cfg["B"]
+    sb = n_seq * (cfg["T"] + 1) * cfg["Hkv"] * 2 * (cfg["r_k"] + cfg["r_v"])
     dts = []
     t_start = time.perf_counter()
     i = 0
@@ -377,7 +550,7 @@ def run_reference(args):
     cfg = dict(CFG2)
     n_seq = 1
     O, I, Kd, Vd, U_k, U_v = _oracle_sample(cfg, n_seq)
-    sb = step_bytes(cfg) * n_seq // cfg["B"]
+    sb = n_seq * (cfg["T"] + 1) * cfg["Hkv"] * 2 * (cfg["r_k"] + cfg["r_v"])
     W, K_steps = max(args.warmup, 1), args.steps
     for i in range(W):
         _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, i)
@@ -403,20 +576,28 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 5000; 128 for config3)")
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4a", "config4b", "config5"],
+                    help="config2 is the headline line; the others are the remaining benchmark configurations")
     ap.add_argument("--num-parts", type=int, default=0, help="CTAs of the persistent decode kernel (0 = one per SM)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ranks", default=None, help="r_k,r_v override for the single-layer workloads, e.g. 48,96")
+    ap.add_argument("--layers", type=int, default=32, help="layers of the multi-layer workloads (config3, config5)")
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="launch every step's kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 128 if args.workload == "config3" else 5000
     if args.impl == "reference":
         run_reference(args)
-    else:
+    elif args.workload in SINGLE_LAYER:
         run_ours(args)
+    else:
+        run_multilayer(args)
 
 
 if __name__ == "__main__":

@@ -24,7 +24,10 @@ cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const C
   }
 }
 
-int decode_box_width(int r) { return (r % 64 == 0) ? 64 : (r % 32 == 0) ? 32 : 16; }
+// Swizzle span (bytes) of the page-tile boxes of rank r, and whether the tile is fetched in its linear view
+// (must agree with Tile<R> in stief_common.cuh)
+int decode_swizzle_span(int r) { return r == 48 ? 32 : r == 96 ? 64 : (r % 64 == 0) ? 128 : 64; }
+bool decode_tile_linear(int r) { return r == 48 || r == 96; }
 
 namespace {
 
@@ -149,12 +152,15 @@ namespace {
 bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
-  const int bw = decode_box_width(r);
-  const cuuint64_t gdim[2] = {(cuuint64_t)r, (cuuint64_t)rows};
-  const cuuint64_t gstride[1] = {(cuuint64_t)r * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)bw, (cuuint32_t)kPage};
+  const int span = decode_swizzle_span(r), bw = span / 2;
+  const bool linear = decode_tile_linear(r);
+  // boxed: the pool as rows of r elements, boxes of 64 rows x bw; linear: the pool as lines of `span` bytes,
+  // one box of 128 r / span lines per (page, head) tile
+  const cuuint64_t gdim[2] = {(cuuint64_t)(linear ? bw : r), (cuuint64_t)(linear ? rows * r * 2 / span : rows)};
+  const cuuint64_t gstride[1] = {(cuuint64_t)(linear ? span : r * 2)};
+  const cuuint32_t box[2] = {(cuuint32_t)bw, (cuuint32_t)(linear ? 128 * r / span : kPage)};
   const cuuint32_t estr[2] = {1, 1};
-  const CUtensorMapSwizzle sw = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  const CUtensorMapSwizzle sw = span == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : span == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   const CUresult rc = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

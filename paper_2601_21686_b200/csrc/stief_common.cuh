@@ -146,25 +146,44 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 // ---------------------------------------------------------------------------------------------
 // swizzled page tiles in shared memory
 // ---------------------------------------------------------------------------------------------
-// A page tile holds 64 cache rows of R bf16.  It is fetched as R/BW boxes of 64 rows x BW elements,
-// BW the largest of 64/32/16 dividing R, each box stored with the TMA swizzle whose span equals the
-// box row (128/64/32 bytes), so that the eight 16-byte row pieces of an 8x8 ldmatrix tile fall in
-// distinct banks.
+// A page tile holds 64 cache rows of R bf16 and is one contiguous block of 128 R bytes in the pool.  It is
+// fetched by TMA with a hardware swizzle chosen so that the eight 16-byte row pieces of an 8x8 ldmatrix tile
+// fall in distinct banks:
+//   R = 32, 64, 128 ("boxed"): boxes of 64 rows x min(R, 64) elements, swizzle span = box row (64 or 128 bytes);
+//                             R = 128 takes two boxes.
+//   R = 48, 96 ("linear"):    the block is viewed as lines of 32 (R = 48) or 64 (R = 96) bytes and fetched as ONE
+//                             box of 192 lines with that swizzle span; shared memory then holds the rows back to
+//                             back (row stride 2 R bytes) with the swizzle applied to the linear offset.  One
+//                             wide request instead of three narrow ones, and still conflict-free.
+// In both forms a step of 8 (or 16) rows leaves the swizzle term of an address unchanged, so the kernels add
+// plain multiples of 8 * RB to a per-lane base.
 template <int R>
 struct Tile {
-  static constexpr int BW = (R % 64 == 0) ? 64 : (R % 32 == 0) ? 32 : 16;   // box width, elements
-  static constexpr int NB = R / BW;                                         // boxes per tile
-  static constexpr int RB = BW * 2;                                         // box row bytes
-  static constexpr int CPB = BW / 8;                                        // 16-byte chunks per box row
-  static constexpr int BOX_BYTES = kPage * RB;
+  static constexpr bool LINEAR = (R == 48 || R == 96);
+  static constexpr int SW = (R == 48) ? 32 : (R == 96) ? 64 : (R % 64 == 0) ? 128 : 64;   // swizzle span, bytes
+  static constexpr int BW = SW / 2;                                         // box width, elements
+  static constexpr int NB = LINEAR ? 1 : (2 * R) / SW;                      // boxes per tile
+  static constexpr int RB = LINEAR ? 2 * R : SW;                            // bytes from one token row to the next
+  static constexpr int CPB = SW / 16;                                       // 16-byte chunks per swizzle span
+  static constexpr int BOX_ROWS = LINEAR ? (128 * R) / SW : kPage;          // rows of the TMA box
+  static constexpr int BOX_BYTES = BOX_ROWS * SW;
   static constexpr int BYTES = kPage * R * 2;
   // byte offset inside the tile of 16-byte chunk c (0 .. R/8-1) of row t
   __device__ static __forceinline__ uint32_t chunk(int t, int c) {
-    const int sub = c / CPB, cc = c % CPB;
-    uint32_t off = static_cast<uint32_t>(t * RB + cc * 16);
-    off ^= ((off >> 7) & (CPB - 1)) << 4;
-    return static_cast<uint32_t>(sub * BOX_BYTES) + off;
+    if constexpr (LINEAR) {
+      uint32_t off = static_cast<uint32_t>(t * RB + c * 16);
+      off ^= ((off >> 7) & (CPB - 1)) << 4;
+      return off;
+    } else {
+      const int sub = c / CPB, cc = c % CPB;
+      uint32_t off = static_cast<uint32_t>(t * RB + cc * 16);
+      off ^= ((off >> 7) & (CPB - 1)) << 4;
+      return static_cast<uint32_t>(sub * BOX_BYTES) + off;
+    }
   }
+  // TMA coordinates of box nb of the tile with index `tile` (= page * Hkv + head)
+  __device__ static __forceinline__ int tma_x(int nb) { return LINEAR ? 0 : nb * BW; }
+  __device__ static __forceinline__ int tma_y(int tile) { return tile * BOX_ROWS; }
 };
 
 // ---------------------------------------------------------------------------------------------

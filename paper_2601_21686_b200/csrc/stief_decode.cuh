@@ -208,13 +208,14 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
             asm volatile("fence.proxy.async.global;" ::: "memory");
           }
           const uint32_t st = ring + slot * C::STAGE_BYTES;
-          const int y = (page * Hkv + h) * kPage;
+          const int tile = page * Hkv + h;
           mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
 #pragma unroll
-          for (int nb = 0; nb < TK::NB; ++nb) tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, nb * TK::BW, y, full_bar(slot));
+          for (int nb = 0; nb < TK::NB; ++nb)
+            tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, TK::tma_x(nb), TK::tma_y(tile), full_bar(slot));
 #pragma unroll
           for (int nb = 0; nb < TV::NB; ++nb)
-            tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, nb * TV::BW, y, full_bar(slot));
+            tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, TV::tma_x(nb), TV::tma_y(tile), full_bar(slot));
         }
         __syncwarp();
       }

@@ -53,7 +53,8 @@ bool encode_bf16_map(CUtensorMap* tm, const void* base, int rank, const unsigned
                      const unsigned long long* strides_bytes, const unsigned* box, CUtensorMapSwizzle swizzle);
 // Full-rank side of the prefill (no basis): the rows are copied to the pool unchanged.  side: 0 = keys, 1 = values.
 cudaError_t launch_prefill_copy(const PrefillArgs& a, int side, cudaStream_t st);
-// Box width (elements) of the TMA tiles the decode kernel expects for rank r.
-int decode_box_width(int r);
+// Shape of the TMA boxes the decode kernel expects for rank r (see Tile<R>).
+int decode_swizzle_span(int r);
+bool decode_tile_linear(int r);
 
 }  // namespace stief
