@@ -75,6 +75,16 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Bounded wait until a shared-memory counter (written by other warps of the CTA after a fence) reaches `target`
+__device__ __forceinline__ void wait_count(volatile int* counter, int target, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t i = 0; i < kWaitSpins; ++i) {
+    if (*counter >= target) return;
+    if ((i & 1023u) == 1023u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  report(status, STIEF_ERR_TIMEOUT);
+}
+
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }

@@ -39,7 +39,7 @@ struct DecodeCfg {
   static constexpr int SPW = (NSTAGE_MAX / NW) > 4 ? 4 : (NSTAGE_MAX / NW);        // private stages per consumer warp
   static constexpr int NS = NW * SPW;
   static constexpr int NT = NW * 32;                     // consumer threads
-  static constexpr int THREADS = NT + 32;                // + 1 producer warp
+  static constexpr int THREADS = 2 * NT;                 // + one producer warp per consumer warp
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
   // scratch after the ring
   static constexpr int CTRL_BYTES = 512;                 // full[NS], empty[NS], append barrier, flags
@@ -138,7 +138,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const uint32_t ctrl = ring + C::RING_BYTES;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (16 + s) * 8; };
-  const uint32_t append_bar = ctrl + 32 * 8;
+  volatile int* append_done = reinterpret_cast<volatile int*>(ctrl_ptr + 32 * 8);   // appending segments whose rows are stored
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8);
   volatile int* last_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
@@ -152,7 +152,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(append_bar, 1);
+    *append_done = 0;
     *abort_flag = 0;
     *last_flag = 0;
     mbar_fence_init();
@@ -170,14 +170,18 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   walk.init(pref, B, upb, pad, c, P, total);
   Segment seg;
 
-  // ------------------------------------------------------------------ producer warp
-  if (warp == NW) {
+  // ------------------------------------------------------------------ producer warps
+  // Producer warp pw feeds consumer warp pw: it issues the TMA loads of every NW-th page into that warp's private
+  // stages.  One issuing thread per CTA could not keep up with small page tiles (a page costs it a few hundred
+  // cycles of waits and descriptor traffic whatever its size), so the issue work is split the way the pages are.
+  if (warp >= NW) {
+    const int pw = warp - NW;
     if (lane == 0) {
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
     }
-    int i = 0;                 // pages issued by this CTA so far (across segments)
-    int n_append = 0;          // segments so far that had to wait for the new token's rows
+    int i_base = 0;            // pages of this CTA before the current segment
+    int n_append = 0;          // appending segments of this CTA so far
     while (walk.next(seg)) {
       const int h = seg.j / QT;
       const int npg = seg.p1 - seg.p0;
@@ -186,10 +190,11 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         const int pos = a.Bt.seq_lens[seg.b];
         wait_append = pos >= 0 && pos / kPage < a.Bt.max_pages;
       }
-      int tbl = 0;
-      for (int k = 0; k < npg; ++k, ++i) {
-        if ((k & 31) == 0) {
-          const int idx = seg.p0 + k + lane;
+      int tbl = 0, win = -1;
+      for (int k = (pw - i_base % NW + NW) % NW; k < npg; k += NW) {
+        if ((k >> 5) != win) {                             // block-table entries of a window of 32 pages, one per lane
+          win = k >> 5;
+          const int idx = seg.p0 + (win << 5) + lane;
           tbl = (idx < seg.p1) ? a.Bt.block_table[(size_t)seg.b * a.Bt.max_pages + idx] : 0;
         }
         int page = __shfl_sync(0xffffffffu, tbl, k & 31);
@@ -197,14 +202,15 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
           if (lane == 0) report(a.status, STIEF_ERR_BOUNDS);
           page = 0;
         }
-        const int cw = i % NW, kw = i / NW;               // consumer warp of this page, its k-th page
-        const int slot = cw * SPW + kw % SPW;
+        const int kw = (i_base + k) / NW;                  // the consumer warp's kw-th page
+        const int slot = pw * SPW + kw % SPW;
         const int use = kw / SPW;
         if (lane == 0) {
           if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
           if (wait_append && k == npg - 1) {
             // the sequence's last page receives the new token's rows from this CTA's consumers first
-            mbar_wait(append_bar, n_append & 1, abort_flag, a.status);
+            wait_count(append_done, n_append + 1, abort_flag, a.status);
+            __threadfence();
             asm volatile("fence.proxy.async.global;" ::: "memory");
           }
           const uint32_t st = ring + slot * C::STAGE_BYTES;
@@ -219,6 +225,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         }
         __syncwarp();
       }
+      i_base += npg;
       if (wait_append) ++n_append;
     }
     return;
@@ -335,7 +342,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       asm volatile("fence.proxy.async.global;" ::: "memory");
     }
     bar1(NT);
-    if (do_append && tid == 0) mbar_arrive(append_bar);               // rows are in the pool: the last page may be fetched
+    if (do_append && tid == 0) *append_done = *append_done + 1;       // rows are in the pool: the last page may be fetched
 
     // A operand of the score MMA: rows 0-7 = bf16(q'), rows 8-15 = bf16(q' - bf16(q'))
     uint32_t qa[RK / 16][4];
