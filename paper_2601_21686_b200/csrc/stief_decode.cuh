@@ -4,18 +4,20 @@
 // over chunks with the back-projection by U_v^T (Eq. 7, Eq. 18).
 //
 // One CTA per SM.  The batch's page tiles are split evenly over the CTAs (stief_partition.cuh); a CTA
-// walks the segments of its range.  A producer warp streams the page tiles K_down[64 x RK],
-// V_down[64 x RV] from HBM into a ring of shared-memory stages with TMA (hardware swizzle, completion
-// on mbarriers) and never stops at segment borders, so the next segment's tiles are already in
-// flight while the consumers finish the current one.  NW consumer warps each take every NW-th page:
-// scores of the group's query heads against the 64 tokens on the tensor cores, online softmax in
-// registers, P V_down accumulated in registers.  At a segment's end the warps merge their running
-// (max, sum, accumulator) and write one chunk-normalised partial; the CTA that delivers a unit's last
-// partial merges all of them and back-projects.
+// walks the segments of its range.  Pages are dealt round-robin to NP page lanes.  Each lane has its own
+// producer warp, which streams the lane's page tiles K_down[64 x RK], V_down[64 x RV] from HBM into the
+// lane's private stages of a shared-memory ring with TMA (hardware swizzle, completion on mbarriers) and
+// never stops at segment borders, so the next segment's tiles are already in flight while the consumers
+// finish the current one.  A lane's pages are consumed by one warp (small tiles) or by two warps that take
+// 32 tokens each (large tiles): scores of the group's query heads against the tokens on the tensor cores,
+// online softmax in registers, P V_down accumulated in registers; every consumer warp is an independent
+// online-softmax stream.  At a segment's end the warps merge their running (max, sum, accumulator) and
+// write one chunk-normalised partial; the CTA that delivers a unit's last partial merges all of them and
+// back-projects.
 //
-// Every consumer warp owns SPW private stages of the ring and walks them in order, so each mbarrier
-// is only ever waited on by one warp, phase after phase (a parity wait can tell two adjacent phases
-// apart but not more).
+// A lane's stages are walked in order and each full-barrier is only waited on by the lane's own consumer
+// warps, phase after phase (a parity wait can tell two adjacent phases apart but not more); the empty-
+// barrier of a stage collects one arrival per consumer warp of the lane before the producer refills it.
 //
 // Precision: q' (already scaled by log2(e)/sqrt(128)) and P are each carried as a pair of bf16 words
 // (value + remainder) occupying rows 0-7 and 8-15 of the 16-row MMA operand, so the products see
@@ -35,11 +37,17 @@ struct DecodeCfg {
   static constexpr int STAGE_BYTES = TK::BYTES + TV::BYTES;
   static constexpr int RING_BUDGET = 192 * 1024;
   static constexpr int NSTAGE_MAX = RING_BUDGET / STAGE_BYTES;
-  static constexpr int NW = NSTAGE_MAX >= 8 ? 4 : (NSTAGE_MAX >= 6 ? 3 : 2);      // consumer warps
-  static constexpr int SPW = (NSTAGE_MAX / NW) > 4 ? 4 : (NSTAGE_MAX / NW);        // private stages per consumer warp
-  static constexpr int NS = NW * SPW;
+  // Pages are dealt round-robin to NP "page lanes"; a lane owns SPW private ring stages, is fed by its own
+  // producer warp and consumed by HALF warps that each take 64 / HALF of the page's tokens (an independent
+  // online-softmax stream each).  Small tiles: 4 lanes x 1 warp.  Tiles above 24 KiB leave room for 6 stages
+  // only, and one warp per page could not keep up with their MMA work: 2 lanes x 2 warps.
+  static constexpr int HALF = NSTAGE_MAX >= 8 ? 1 : 2;
+  static constexpr int NP = NSTAGE_MAX >= 8 ? 4 : 2;
+  static constexpr int NW = NP * HALF;                   // consumer warps
+  static constexpr int SPW = (NSTAGE_MAX / NP) > 4 ? 4 : (NSTAGE_MAX / NP);        // private stages per page lane
+  static constexpr int NS = NP * SPW;
   static constexpr int NT = NW * 32;                     // consumer threads
-  static constexpr int THREADS = 2 * NT;                 // + one producer warp per consumer warp
+  static constexpr int THREADS = NT + NP * 32;           // + one producer warp per page lane
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
   // scratch after the ring
   static constexpr int CTRL_BYTES = 512;                 // full[NS], empty[NS], append barrier, flags
@@ -126,7 +134,9 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   using C = DecodeCfg<RK, RV>;
   using TK = typename C::TK;
   using TV = typename C::TV;
-  constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW, NT = C::NT;
+  constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW, NT = C::NT, NP = C::NP, HALF = C::HALF;
+  constexpr int NJ = 8 / HALF;                           // 8-token score tiles per consumer warp and page
+  constexpr int KK = 4 / HALF;                           // 16-token contraction steps of the mix per warp and page
 
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -150,7 +160,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+      mbar_init(empty_bar(s), HALF);
     }
     *append_done = 0;
     *abort_flag = 0;
@@ -171,7 +181,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   Segment seg;
 
   // ------------------------------------------------------------------ producer warps
-  // Producer warp pw feeds consumer warp pw: it issues the TMA loads of every NW-th page into that warp's private
+  // Producer warp pw feeds page lane pw: it issues the TMA loads of every NP-th page into that lane's private
   // stages.  One issuing thread per CTA could not keep up with small page tiles (a page costs it a few hundred
   // cycles of waits and descriptor traffic whatever its size), so the issue work is split the way the pages are.
   if (warp >= NW) {
@@ -191,7 +201,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         wait_append = pos >= 0 && pos / kPage < a.Bt.max_pages;
       }
       int tbl = 0, win = -1;
-      for (int k = (pw - i_base % NW + NW) % NW; k < npg; k += NW) {
+      for (int k = (pw - i_base % NP + NP) % NP; k < npg; k += NP) {
         if ((k >> 5) != win) {                             // block-table entries of a window of 32 pages, one per lane
           win = k >> 5;
           const int idx = seg.p0 + (win << 5) + lane;
@@ -202,7 +212,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
           if (lane == 0) report(a.status, STIEF_ERR_BOUNDS);
           page = 0;
         }
-        const int kw = (i_base + k) / NW;                  // the consumer warp's kw-th page
+        const int kw = (i_base + k) / NP;                  // the lane's kw-th page
         const int slot = pw * SPW + kw % SPW;
         const int use = kw / SPW;
         if (lane == 0) {
@@ -359,31 +369,38 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 #pragma unroll
     for (int n = 0; n < RV / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
 
-    // first page of this segment that belongs to this warp: global index i = i_base + k, i % NW == warp
-    int k0 = (warp - i_base % NW + NW) % NW;
-    for (int k = k0; k < npg; k += NW) {
-      const int kw = (i_base + k) / NW;
-      const int slot = warp * SPW + kw % SPW;
+    // first page of this segment that belongs to this warp's lane: global index i = i_base + k, i % NP == pl
+    const int pl = warp % NP, hf = warp / NP;
+    const int tb = hf * (kPage / HALF);                    // first token of the page this warp handles
+    int k0 = (pl - i_base % NP + NP) % NP;
+    for (int k = k0; k < npg; k += NP) {
+      const int kw = (i_base + k) / NP;
+      const int slot = pl * SPW + kw % SPW;
       mbar_wait(full_bar(slot), (kw / SPW) & 1, abort_flag, a.status);
       const uint32_t kt = ring + slot * C::STAGE_BYTES;
       const uint32_t vt = kt + TK::BYTES;
       const bool tail = (seg.p0 + k == seg.npages - 1) && (last_valid < kPage);
+      if (HALF > 1 && tail && last_valid <= tb) {          // none of this warp's tokens exists: nothing to add
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(slot));
+        continue;
+      }
 
       // ---- scores of the page: n-tile j covers tokens 8j..8j+7; c0,c1 from bf16(q'), c2,c3 from the remainder
-      float sc[16];
+      float sc[2 * NJ];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < NJ; ++j) {
         float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int q4 = 0; 4 * q4 + 4 <= NCH; ++q4) {
           uint32_t r0, r1, r2, r3;
-          ldsm_x4(kt + koff[q4] + j * 8 * TK::RB, r0, r1, r2, r3);
+          ldsm_x4(kt + koff[q4] + (hf * NJ + j) * 8 * TK::RB, r0, r1, r2, r3);
           mma_bf16(s, qa[2 * q4], r0, r1);
           mma_bf16(s, qa[2 * q4 + 1], r2, r3);
         }
         if constexpr (NCH % 4 == 2) {
           uint32_t r0, r1;
-          ldsm_x2(kt + koff[NCH / 4] + j * 8 * TK::RB, r0, r1);
+          ldsm_x2(kt + koff[NCH / 4] + (hf * NJ + j) * 8 * TK::RB, r0, r1);
           mma_bf16(s, qa[NCH / 2 - 1], r0, r1);
         }
         sc[2 * j] = s[0] + s[2];
@@ -391,15 +408,16 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       }
       if (tail) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int t = 8 * j + 2 * tid4;
+        for (int j = 0; j < NJ; ++j) {
+          const int t = tb + 8 * j + 2 * tid4;
           if (t >= last_valid) sc[2 * j] = -INFINITY;
           if (t + 1 >= last_valid) sc[2 * j + 1] = -INFINITY;
         }
         // rows past the end hold unspecified bits: zero them in V so that 0 * garbage cannot make a NaN
         constexpr int NCV = RV / 8;
-        for (int idx = lane; idx < (kPage - last_valid) * NCV; idx += 32) {
-          const int t = last_valid + idx / NCV, cc = idx % NCV;
+        const int z0 = max(last_valid, tb);                // this warp's rows past the end
+        for (int idx = lane; idx < (tb + kPage / HALF - z0) * NCV; idx += 32) {
+          const int t = z0 + idx / NCV, cc = idx % NCV;
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vt + TV::chunk(t, cc)), "r"(0u) : "memory");
         }
         __syncwarp();
@@ -408,16 +426,16 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       // ---- online softmax (base 2; the scale is folded into q')
       float mx = sc[0];
 #pragma unroll
-      for (int e = 1; e < 16; ++e) mx = fmaxf(mx, sc[e]);
+      for (int e = 1; e < 2 * NJ; ++e) mx = fmaxf(mx, sc[e]);
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
       const float m_new = fmaxf(m, mx);
       const float alpha = fast_exp2(m - m_new);
       m = m_new;
-      uint32_t pa[4][4];
+      uint32_t pa[KK][4];
       float ps = 0.f;
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
+      for (int kk = 0; kk < KK; ++kk) {
         const float p0_ = fast_exp2(sc[4 * kk + 0] - m), p1_ = fast_exp2(sc[4 * kk + 1] - m);
         const float p2_ = fast_exp2(sc[4 * kk + 2] - m), p3_ = fast_exp2(sc[4 * kk + 3] - m);
         ps += (p0_ + p1_) + (p2_ + p3_);
@@ -432,11 +450,11 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
       // ---- mix: o += P V_down (tokens are the contraction index; V tile read transposed)
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
+      for (int kk = 0; kk < KK; ++kk) {
 #pragma unroll
         for (int np = 0; np < RV / 16; ++np) {
           uint32_t r0, r1, r2, r3;
-          ldsm_x4_t(vt + voff[np] + kk * 16 * TV::RB, r0, r1, r2, r3);
+          ldsm_x4_t(vt + voff[np] + (hf * KK + kk) * 16 * TV::RB, r0, r1, r2, r3);
           mma_bf16(o[2 * np], pa[kk], r0, r1);
           mma_bf16(o[2 * np + 1], pa[kk], r2, r3);
         }
