@@ -588,8 +588,12 @@ def main():
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="launch every step's kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
+    # DRAM read + write bytes per launch of decode_persistent_kernel<64,64> on config 2, from the ncu capture
+    # summarised in profiles/decode_persistent_kernel_config2.md (mean of two launches); null for other workloads
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
+    if args.traffic is None and args.workload == "config2" and not args.ranks:
+        args.traffic = 274.05e6
     if args.steps is None:
         args.steps = 128 if args.workload == "config3" else 5000
     if args.impl == "reference":
