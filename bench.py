@@ -172,20 +172,17 @@ def run_ours(args):
     from paper_2601_21686_b200 import inputs as I
     from paper_2601_21686_b200 import build as Bld
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2601_21686_b200 import replicas as R
+    me = R.replica_from_env()
+    world, rank, local_rank = me.world, me.rank, me.local_rank
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    R.init(me, "nccl", dev)
     if rank == 0:
         Bld.build()
-    if world > 1:
-        dist.barrier()
+    R.barrier(me)
     S.lib()
 
     cfg = dict(SINGLE_LAYER[args.workload])
@@ -212,8 +209,7 @@ def run_ours(args):
                             num_parts=ns, status=status, flags=flags)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        R.barrier(me)
         torch.cuda.synchronize()
 
     K_steps, W = args.steps, max(args.warmup, 3)
@@ -284,10 +280,7 @@ def run_ours(args):
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
     # ---- max over ranks
-    times = torch.tensor([ms, ms_host, float(np.mean(kern_ms)), ms_serial], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, ms_host, kern_isolated_ms, ms_serial = (float(x) for x in times.tolist())
+    ms, ms_host, kern_isolated_ms, ms_serial = R.max_over_ranks(me, [ms, ms_host, float(np.mean(kern_ms)), ms_serial], device=dev)
     kern_avg_ms = ms / K_steps          # one launch per step: the timed region divided by its launches
 
     if rank == 0:
@@ -336,9 +329,7 @@ def run_ours(args):
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=20.0)
         print(json.dumps(line))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    R.finish(me)
 
 
 # ------------------------------------------------------------------------------------------------
