@@ -309,6 +309,8 @@ def run_ours(args):
             "frac_of_hbm_spec_8000": value / world / 8000.0,
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
+                    "transfer": "q, k_new, v_new and out are pinned mapped HOST buffers handed to stief_decode_step_host: the kernel "
+                                "reads and writes them across the bus itself; the stream is synchronised after every step",
                     "tokens_per_s": world * B * K_steps / (ms_host * 1e-3)},
             "gpu_launches": K_steps,
             "roofline": {"bound": "hbm", "kernel": f"decode_persistent_kernel<{r_k},{r_v}>", "achieved": achieved, "peak": hbm_peak,

@@ -165,7 +165,10 @@ int stief_decode_step(const stief_layer* layer, const stief_batch* batch, const 
 /* The same step for callers whose activations live in host memory: q_host, k_new_host, v_new_host
  * are copied to `staging` (device, stief_host_staging_bytes) with cudaMemcpyAsync on `stream`, the
  * step runs, and out is copied back to out_host.  Nothing is synchronised: the caller waits on the
- * stream before reading out_host.  Host buffers should be pinned for the copies to be asynchronous. */
+ * stream before reading out_host.  Host buffers should be pinned for the copies to be asynchronous.
+ * When all four host buffers are pinned AND mapped (cudaHostAlloc / cudaHostRegister under unified
+ * addressing) the copies are skipped: the kernel reads q, k_new, v_new from host memory in its prologue
+ * and writes the output rows to out_host itself; `staging` is then unused. */
 size_t stief_host_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 int stief_decode_step_host(const stief_layer* layer, const stief_batch* batch, const uint16_t* q_host,
                            const uint16_t* k_new_host, const uint16_t* v_new_host, void* staging,

@@ -303,21 +303,26 @@ def test_overlapped_prefill_launches_match_serial_ones():
 
 
 def test_host_staged_step():
+    # host buffers pinned and mapped: the kernel reads and writes them directly; pageable buffers: staged copies
     B, Hq, Hkv = 2, 8, 2
     c = U.make_case(60, B, Hq, Hkv, 64, 64, [100, 70], reserve=4)
     Kd, Vd = _prefill_and_check(c)
     k_new, v_new = I.new_token_kv(60, 0, B, Hkv)
-    q = c.q.pin_memory()
-    kh, vh = k_new.pin_memory(), v_new.pin_memory()
-    out_h = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
     staging = torch.empty(S.stief_host_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device="cuda")
     ws = U.workspace_for(c, 2)
-    S.stief_decode_step_host(c.layer, c.batch, q, kh, vh, staging, ws, out_h, num_parts=2, status=c.status)
-    assert _sync_status(c) == 0
     out_d = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device="cuda")
     S.stief_decode_step(c.layer, c.batch, c.q.cuda(), k_new.cuda(), v_new.cuda(), ws, out_d, num_parts=2, status=c.status)
     assert _sync_status(c) == 0
-    assert torch.equal(out_h, out_d.cpu())
+    for pinned in (True, False):
+        mk = (lambda t: t.clone().pin_memory()) if pinned else (lambda t: t.clone())
+        q, kh, vh = mk(c.q), mk(k_new), mk(v_new)
+        out_h = mk(torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16))
+        staging.fill_(0xFF)
+        S.stief_decode_step_host(c.layer, c.batch, q, kh, vh, staging, ws, out_h, num_parts=2, status=c.status)
+        assert _sync_status(c) == 0
+        assert torch.equal(out_h, out_d.cpu())
+        # the pinned route must not have touched the staging buffer, the pageable one must have
+        assert bool((staging == 0xFF).all()) == pinned
 
 
 def test_errors_are_reported_not_trapped():
