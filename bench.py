@@ -296,7 +296,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
             "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 cache, fp32 accumulate", "data": "synthetic",
+            "dtype": "bf16", "dtype_note": "bf16 cache and tensor-core operands, fp32 accumulate", "data": "synthetic",
             "config": {"workload": cfg["name"] + ", 64-token pages, shuffled block tables; step = append + query projection + "
                                    "split-T attention + combine, one launch",
                        "global_batch": B * world, "seq_len": T, "r_k": r_k, "r_v": r_v, "num_parts": ns,
@@ -329,7 +329,7 @@ def run_ours(args):
             "clocks": sampler.summary(t0, time.time()),
         }
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=20.0)
+            line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=10.0)
         print(json.dumps(line))
     R.finish(me)
 
@@ -395,7 +395,7 @@ def run_multilayer(args):
     time.sleep(0.3)
     t0 = time.time()
     line = {"n_gpus": 1, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
-            "dtype": "bf16 cache, fp32 accumulate", "rank_profile": prof, "peak_kind": peak_kind, "hbm_peak_gbs": hbm_peak}
+            "dtype": "bf16", "dtype_note": "bf16 cache and tensor-core operands, fp32 accumulate", "rank_profile": prof, "peak_kind": peak_kind, "hbm_peak_gbs": hbm_peak}
     if args.workload == "config3":
         W = 3
         for i in range(W):
@@ -518,14 +518,14 @@ def _threads_used() -> int:
         return 1
 
 
-def cpu_baseline(cfg, seconds_budget=20.0):
+def cpu_baseline(cfg, seconds_budget=10.0):
     n_seq = 1
     O, I, Kd, Vd, U_k, U_v = _oracle_sample(cfg, n_seq)
     sb = n_seq * (cfg["T"] + 1) * cfg["Hkv"] * 2 * (cfg["r_k"] + cfg["r_v"])
     dts = []
     t_start = time.perf_counter()
     i = 0
-    while i < 3 or (time.perf_counter() - t_start < seconds_budget and i < 20):
+    while i < 3 or (time.perf_counter() - t_start < seconds_budget and i < 150):
         dt, _ = _oracle_step(O, I, cfg, n_seq, Kd, Vd, U_k, U_v, i)
         dts.append(dt)
         i += 1
