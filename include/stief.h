@@ -203,6 +203,51 @@ int stief_decode_attention_static(const stief_layer* layer, const stief_batch* b
                                   int32_t len_add, int32_t num_parts, uint16_t* out, float* out_lse,
                                   int32_t* status, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * 8-bit quantised compressed cache (paper Sec. 4.3: asymmetric integer quantisation of the compressed cache
+ * tensors, group size 64; keys use group-wise parameters shared across batch and sequence positions within a
+ * KV head, values use token-wise group parameters).
+ * A group is 64 consecutive channels of the compressed dimension; a code c in 0..255 stands for
+ * c * scale + zero.  Key parameters are fixed ahead of time (calibration) per KV head and channel group and
+ * given by the caller; a key outside the calibrated range is clamped.  Value parameters are computed from each
+ * row when it is written: zero = min, scale = (max - min) / 255 over the group (scale = 1 when max == min).
+ * The quantiser sees the projection K U_k / V U_v in fp32 (not rounded to bf16 first) and decides in fp32:
+ * code = clamp(rint((x - zero) * (1 / scale))), ties to even.  Ranks must be 64 or 128 and both bases given.
+ * Layout: k_codes, v_codes [num_pages][Hkv][64][r] uint8, r fastest, indexed like the bf16 pools;
+ * k_params [Hkv][r_k / 64][2] fp32 (scale, zero); v_params [num_pages][Hkv][64][r_v / 64][2] fp32 (scale, zero).
+ * Alignment: code pools and v_params 128 bytes, k_params 8 bytes.  Bytes per cached (token, KV head):
+ * r_k + r_v + 8 * (r_v / 64), against 2 (r_k + r_v) for the bf16 cache. */
+typedef struct stief_qlayer {
+  int32_t Hq, Hkv, d;
+  int32_t r_k, r_v;
+  int32_t num_pages;
+  const uint16_t* U_k;
+  int64_t uk_head_stride;
+  const uint16_t* U_v;
+  int64_t uv_head_stride;
+  const float* k_params;
+  uint8_t* k_codes;
+  uint8_t* v_codes;
+  float* v_params;
+} stief_qlayer;
+
+/* Eq. 1 for a whole prompt followed by quantisation; arguments as stief_prefill_compress. */
+int stief_q8_prefill_compress(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* K,
+                              const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
+                              uint32_t flags, int32_t* status, void* stream);
+
+/* One new token per sequence: projects, quantises and stores k_new, v_new at position seq_lens[b]. */
+int stief_q8_append(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* k_new,
+                    const uint16_t* v_new, int32_t* status, void* stream);
+
+/* Decode attention on the quantised cache: ordinary attention (Eq. 18) on the reconstructions (Eq. 7) of the
+ * DEQUANTISED cache, evaluated in the compressed space (the key scale folds into the projected query, the
+ * key zero-point shifts every score of a row by the same amount and so only enters out_lse).  Arguments,
+ * workspace (stief_decode_workspace_bytes with the same r_v) and flags as stief_decode_attention. */
+int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q,
+                              int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
+                              uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+
 /* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
  * stief_decode_step_host call made by this host thread records `start_event` just before and
  * `stop_event` just after its decode kernel on the call's stream (both cudaEvent_t passed as void*),

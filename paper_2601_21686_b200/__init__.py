@@ -39,6 +39,15 @@ class _CLayer(ctypes.Structure):
                 ("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p)]
 
 
+class _CQLayer(ctypes.Structure):
+    _fields_ = [("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("r_k", ctypes.c_int32), ("r_v", ctypes.c_int32), ("num_pages", ctypes.c_int32),
+                ("U_k", ctypes.c_void_p), ("uk_head_stride", ctypes.c_int64),
+                ("U_v", ctypes.c_void_p), ("uv_head_stride", ctypes.c_int64),
+                ("k_params", ctypes.c_void_p), ("k_codes", ctypes.c_void_p), ("v_codes", ctypes.c_void_p),
+                ("v_params", ctypes.c_void_p)]
+
+
 class _CBatch(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
                 ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p)]
@@ -56,7 +65,7 @@ def lib() -> ctypes.CDLL:
                                "(there is no non-CUDA path)")
         L = ctypes.CDLL(LIB_PATH)
         P, I32, I64, SZ, U32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32
-        LP, BP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch)
+        LP, BP, QP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch), ctypes.POINTER(_CQLayer)
         sig = {
             "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, U32, P, P]),
             "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
@@ -71,6 +80,9 @@ def lib() -> ctypes.CDLL:
             "stief_decode_step_host": (ctypes.c_int, [LP, BP, P, P, P, P, P, SZ, I32, P, U32, P, P]),
             "stief_advance_seq_lens": (ctypes.c_int, [P, I32, I32, P]),
             "stief_time_next_decode_kernel": (ctypes.c_int, [P, P]),
+            "stief_q8_prefill_compress": (ctypes.c_int, [QP, BP, P, P, I64, I64, I32, U32, P, P]),
+            "stief_q8_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
+            "stief_q8_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -114,6 +126,34 @@ class Layer:
 
 
 @dataclass
+class QLayer:
+    """One decoder layer's 8-bit quantised compressed cache (device tensors): U_k [Hkv or 1, 128, r_k], U_v
+    [Hkv or 1, 128, r_v] bf16; k_params [Hkv, r_k/64, 2] fp32 (scale, zero; static); k_codes / v_codes
+    [num_pages, Hkv, 64, r] uint8; v_params [num_pages, Hkv, 64, r_v/64, 2] fp32 (scale, zero per token and group)."""
+    Hq: int
+    Hkv: int
+    r_k: int
+    r_v: int
+    U_k: torch.Tensor
+    U_v: torch.Tensor
+    k_params: torch.Tensor
+    k_codes: torch.Tensor
+    v_codes: torch.Tensor
+    v_params: torch.Tensor
+
+    @property
+    def num_pages(self) -> int:
+        return self.k_codes.shape[0]
+
+    def c(self) -> _CQLayer:
+        uk_stride = 0 if self.U_k.shape[0] == 1 else self.U_k.stride(0)
+        uv_stride = 0 if self.U_v.shape[0] == 1 else self.U_v.stride(0)
+        return _CQLayer(self.Hq, self.Hkv, D_HEAD, self.r_k, self.r_v, self.num_pages, _ptr(self.U_k), uk_stride,
+                        _ptr(self.U_v), uv_stride, _ptr(self.k_params), _ptr(self.k_codes), _ptr(self.v_codes),
+                        _ptr(self.v_params))
+
+
+@dataclass
 class Batch:
     """Paging state: block_table [B, max_pages_per_seq] int32, seq_lens [B] int32 (device tensors)."""
     block_table: torch.Tensor
@@ -144,6 +184,31 @@ def stief_prefill_compress(layer: Layer, batch: Batch, K: torch.Tensor, V: torch
     _check(lib().stief_prefill_compress(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
                                         K.shape[1] if T_max is None else T_max, flags, _ptr(status), _stream()),
            "stief_prefill_compress")
+
+
+def stief_q8_prefill_compress(layer: QLayer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
+                              status: Optional[torch.Tensor] = None, flags: int = 0):
+    """K, V [B, T, Hkv, 128] bf16 -> 8-bit quantised paged compressed cache."""
+    assert K.stride(3) == 1 and K.stride(2) == D_HEAD and V.stride() == K.stride()
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_q8_prefill_compress(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
+                                           K.shape[1] if T_max is None else T_max, flags, _ptr(status), _stream()),
+           "stief_q8_prefill_compress")
+
+
+def stief_q8_append(layer: QLayer, batch: Batch, k_new: torch.Tensor, v_new: torch.Tensor, status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_q8_append(ctypes.byref(cl), ctypes.byref(cb), _ptr(k_new), _ptr(v_new), _ptr(status), _stream()),
+           "stief_q8_append")
+
+
+def stief_q8_decode_attention(layer: QLayer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, out: torch.Tensor,
+                              num_parts: int = 0, out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
+                              status: Optional[torch.Tensor] = None, flags: int = 0):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_q8_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
+                                           flags, _ptr(status), _stream()), "stief_q8_decode_attention")
 
 
 def stief_append(layer: Layer, batch: Batch, k_new: torch.Tensor, v_new: torch.Tensor, status: Optional[torch.Tensor] = None):

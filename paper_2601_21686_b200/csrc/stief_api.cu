@@ -2,8 +2,7 @@
 // No allocation, no synchronisation; everything is enqueued on the caller's stream.
 #include <cstring>
 
-#include "stief_kernels.h"
-#include "stief_partition.cuh"
+#include "stief_host_util.h"
 
 namespace stief {
 
@@ -31,9 +30,9 @@ bool decode_tile_linear(int r) { return r == 48 || r == 96; }
 
 namespace {
 
+using namespace host;
+
 bool rank_ok(int r) { return r == 32 || r == 48 || r == 64 || r == 96 || r == 128; }
-bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
-size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int check_layer(const stief_layer* l) {
   if (!l) return STIEF_ERR_INVALID_ARG;
@@ -48,11 +47,6 @@ int check_layer(const stief_layer* l) {
   if ((long long)l->num_pages * l->Hkv * kPage >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
   return STIEF_OK;
 }
-int check_batch(const stief_batch* b) {
-  if (!b || b->B <= 0 || b->max_pages_per_seq <= 0 || !b->block_table || !b->seq_lens) return STIEF_ERR_INVALID_ARG;
-  if (b->B > kMaxBatch) return STIEF_ERR_INVALID_ARG;
-  return STIEF_OK;
-}
 
 LayerDev to_dev(const stief_layer* l) {
   LayerDev d;
@@ -62,54 +56,8 @@ LayerDev to_dev(const stief_layer* l) {
   d.k_pool = reinterpret_cast<__nv_bfloat16*>(l->k_pool); d.v_pool = reinterpret_cast<__nv_bfloat16*>(l->v_pool);
   return d;
 }
-BatchDev to_dev(const stief_batch* b) {
-  BatchDev d;
-  d.B = b->B; d.max_pages = b->max_pages_per_seq; d.block_table = b->block_table; d.seq_lens = b->seq_lens;
-  return d;
-}
 
-int sm_count() {
-  static int cached[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
-    cudaGetLastError();
-    return 148;
-  }
-  if (cached[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
-      cudaGetLastError();
-      n = 148;
-    }
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
 
-int resolve_parts(int num_parts) { return num_parts > 0 ? num_parts : sm_count(); }
-int query_tiles(int Hq, int Hkv) { return (Hq / Hkv + kGroupTile - 1) / kGroupTile; }
-
-struct Workspace {
-  int* counters;
-  float* partial_o;
-  float* partial_lse;
-  size_t bytes;
-};
-Workspace carve(void* base, int B, int Hq, int Hkv, int r_v, int n_cta) {
-  Workspace w;
-  const size_t n_units = (size_t)B * Hkv * query_tiles(Hq, Hkv);
-  const size_t slots = n_units + (size_t)n_cta;
-  size_t off = 0;
-  uint8_t* p = static_cast<uint8_t*>(base);
-  w.counters = reinterpret_cast<int*>(p + off);
-  off += align_up(n_units * 4, 128);
-  w.partial_o = reinterpret_cast<float*>(p + off);
-  off += align_up(slots * kGroupTile * r_v * 4, 128);
-  w.partial_lse = reinterpret_cast<float*>(p + off);
-  off += align_up(slots * kGroupTile * 4, 128);
-  w.bytes = off;
-  return w;
-}
 
 // ---- tensor maps ----------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -211,7 +159,7 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   dl.overlap_previous = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0;
   DecodeArgs& a = dl.args;
   a.L = to_dev(layer);
-  a.Bt = to_dev(batch);
+  a.Bt = host::to_dev(batch);
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
@@ -251,7 +199,7 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
     return STIEF_ERR_INVALID_ARG;
   if (batch->B > 1 && stride_b == 0) return STIEF_ERR_INVALID_ARG;
   PrefillArgs a;
-  a.L = to_dev(layer); a.Bt = to_dev(batch);
+  a.L = to_dev(layer); a.Bt = host::to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);
   a.stride_b = stride_b; a.stride_t = stride_t; a.T_max = T_max; a.status = status;
   a.overlap_previous = (flags & STIEF_PREFILL_OVERLAP_PREVIOUS) != 0;
@@ -266,7 +214,7 @@ int stief_append(const stief_layer* layer, const stief_batch* batch, const uint1
   if (rc) return rc;
   if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return STIEF_ERR_INVALID_ARG;
   AppendArgs a;
-  a.L = to_dev(layer); a.Bt = to_dev(batch);
+  a.L = to_dev(layer); a.Bt = host::to_dev(batch);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
   a.status = status;
@@ -305,7 +253,7 @@ int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int3
   const int n_cta = resolve_parts(num_parts);
   const Workspace w = carve(const_cast<void*>(workspace), batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
   CombineArgs ca;
-  ca.L = to_dev(layer); ca.Bt = to_dev(batch);
+  ca.L = to_dev(layer); ca.Bt = host::to_dev(batch);
   ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
   ca.n_cta = n_cta; ca.QT = query_tiles(layer->Hq, layer->Hkv); ca.len_add = len_add;
   ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;

@@ -149,7 +149,7 @@ constexpr int kCombineScratchFloats = kGroupTile * kD + kSegChunk * kGroupTile +
 template <int RV>
 __device__ __forceinline__ void combine_unit(const LayerDev& L, int b, int h, int qt, int slot0, int nseg, const float* partial_o,
                                              const float* partial_lse, __nv_bfloat16* out, float* out_lse, float* od, float* wsm,
-                                             int tid, int nt) {
+                                             int tid, int nt, const float* lse_shift = nullptr) {
   constexpr int NV = RV / 4;                               // float4 pieces per row
   constexpr int IPT = 3;                                   // pieces per thread: 8 * NV <= 256 <= 3 * 96
   const int G = L.G;
@@ -260,7 +260,9 @@ __device__ __forceinline__ void combine_unit(const LayerDev& L, int b, int h, in
       *reinterpret_cast<float4*>(od + r * kD + 4 * j4) = make_float4(num[i].x * inv, num[i].y * inv, num[i].z * inv, num[i].w * inv);
     }
   }
-  if (tid < ng && out_lse) out_lse[head0 + tid] = Drow[tid] > 0.f ? Mrow[tid] + __logf(Drow[tid]) : -INFINITY;
+  // lse_shift: a per-row constant that was left out of every score of the unit (it cancels in the softmax)
+  if (tid < ng && out_lse)
+    out_lse[head0 + tid] = Drow[tid] > 0.f ? Mrow[tid] + __logf(Drow[tid]) + (lse_shift ? lse_shift[tid] : 0.f) : -INFINITY;
   bar1(nt);
   for (int dd = tid; dd < kD; dd += nt) {
     float acc[kGroupTile];

@@ -45,6 +45,12 @@ struct Args {
   int n_chunks;              // chunks per unit's tile list (see TileWalker)
   int nst;                   // ring stages
   int rmax;                  // larger of the ranks that are projected
+  // 8-bit quantised cache (Q8 kernel only): code pools [pages][Hkv][64][r] uint8, value parameters
+  // [pages][Hkv][64][r_v/64][2] fp32 (scale, zero), static key parameters [Hkv][r_k/64][2] fp32
+  uint8_t* k_codes;
+  uint8_t* v_codes;
+  float* v_params;
+  const float* k_params;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -242,6 +248,9 @@ __device__ __forceinline__ void stage_basis(const __nv_bfloat16* __restrict__ U,
   if (lane == 0) mbar_arrive(ready_bar);
 }
 
+// Q8 = false: bf16 cache.  Q8 = true: the epilogue quantises each 64-channel group of a row to 8-bit codes
+// (asymmetric; static key parameters, token-wise value parameters) instead of rounding it to bf16.
+template <bool Q8>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmPK, const __grid_constant__ CUtensorMap tmPV, const Args a) {
@@ -419,7 +428,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
           if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
           valid = false;
         }
-        const bool full = valid && tok0 + 32 <= t.len;     // else the sequence ends inside these rows
+        const bool full = !Q8 && valid && tok0 + 32 <= t.len;   // else the sequence ends inside these rows (or codes are stored)
         const int row0 = (max(page, 0) * Hkv + t.h) * kPage + (tok0 % kPage);  // pool row of the warp's first token
         // full case: rows are rounded to bf16 into swizzled staging boxes and leave by TMA stores.  A box is 32
         // rows x BW elements (BW = 64, 32 or 16: the largest that divides R), swizzle span = box row.
@@ -443,6 +452,48 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int c = 0; c < 4; ++c)
               if ((c0 + c) * 16 < R) tmem_ld16(taddr + (c0 + c) * 16, v[c]);
             tmem_ld_wait();
+            if constexpr (Q8) {
+              // columns 16 c0 .. 16 c0 + 63 are one quantisation group of this thread's row
+              if (row_ok) {
+                const int g = c0 >> 2, ng = R >> 6;
+                float sc, zp;
+                if (t.side == 0) {
+                  const float2 kp = *reinterpret_cast<const float2*>(a.k_params + ((size_t)t.h * ng + g) * 2);
+                  sc = kp.x;
+                  zp = kp.y;
+                } else {
+                  float mn = __uint_as_float(v[0][0]), mx = mn;
+#pragma unroll
+                  for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                      mn = fminf(mn, __uint_as_float(v[c][e]));
+                      mx = fmaxf(mx, __uint_as_float(v[c][e]));
+                    }
+                  sc = mx > mn ? __fdiv_rn(mx - mn, 255.f) : 1.f;
+                  zp = mn;
+                  *reinterpret_cast<float2*>(a.v_params + (((size_t)row0 + lane) * ng + g) * 2) = make_float2(sc, zp);
+                }
+                const float inv = __fdiv_rn(1.f, sc);
+                uint8_t* qdst = (t.side ? a.v_codes : a.k_codes) + ((size_t)row0 + lane) * R + 64 * g;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  uint32_t w[4];
+#pragma unroll
+                  for (int e4 = 0; e4 < 4; ++e4) {
+                    uint32_t word = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][4 * e4 + e]), zp), inv);
+                      const uint32_t code = (uint32_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+                      word |= code << (8 * e);
+                    }
+                    w[e4] = word;
+                  }
+                  *reinterpret_cast<uint4*>(qdst + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+              }
+            } else {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               if ((c0 + c) * 16 < R) {
@@ -469,6 +520,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   dst[2 * (c0 + c) + 1] = o[1];
                 }
               }
+            }
             }
           }
         }
@@ -539,32 +591,26 @@ int smem_bytes(int nst, int rmax, int B) {
 
 }  // namespace
 
-cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
-  const bool proj_k = a.L.U_k != nullptr, proj_v = a.L.U_v != nullptr;
-  if (!proj_k) {
-    cudaError_t e = launch_prefill_copy(a, 0, st);
-    if (e != cudaSuccess) return e;
-  }
-  if (!proj_v) {
-    cudaError_t e = launch_prefill_copy(a, 1, st);
-    if (e != cudaSuccess) return e;
-  }
-  if (!proj_k && !proj_v) return cudaSuccess;
+namespace {
 
+template <bool Q8>
+cudaError_t launch_prefill_tc(const PrefillArgs& a, const Args* q8, cudaStream_t st) {
+  const bool proj_k = a.L.U_k != nullptr, proj_v = a.L.U_v != nullptr;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   CUtensorMap tmK, tmV;
   if (!make_input_map(&tmK, proj_k ? a.K : a.V, a) || !make_input_map(&tmV, proj_v ? a.V : a.K, a)) return cudaErrorInvalidValue;
-  CUtensorMap tmPK, tmPV;
-  if (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a))
+  CUtensorMap tmPK = tmK, tmPV = tmV;                     // the quantising kernel stores without TMA: placeholders
+  if (!Q8 && (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a)))
     return cudaErrorInvalidValue;
-  Args args;
+  Args args = {};
+  if (q8) args = *q8;
   args.p = a;
   args.n_side = (proj_k ? 1 : 0) + (proj_v ? 1 : 0);
   args.side0 = proj_k ? 0 : 1;
@@ -603,7 +649,33 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.overlap_previous ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, tmK, tmV, tmPK, tmPV, args);
+  return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<Q8>, tmK, tmV, tmPK, tmPV, args);
+}
+
+}  // namespace
+
+cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
+  const bool proj_k = a.L.U_k != nullptr, proj_v = a.L.U_v != nullptr;
+  if (!proj_k) {
+    cudaError_t e = launch_prefill_copy(a, 0, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (!proj_v) {
+    cudaError_t e = launch_prefill_copy(a, 1, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (!proj_k && !proj_v) return cudaSuccess;
+  return launch_prefill_tc<false>(a, nullptr, st);
+}
+
+cudaError_t launch_prefill_q8(const PrefillArgs& a, uint8_t* k_codes, uint8_t* v_codes, float* v_params, const float* k_params,
+                              cudaStream_t st) {
+  Args q8 = {};
+  q8.k_codes = k_codes;
+  q8.v_codes = v_codes;
+  q8.v_params = v_params;
+  q8.k_params = k_params;
+  return launch_prefill_tc<true>(a, &q8, st);
 }
 
 }  // namespace stief

@@ -1,0 +1,202 @@
+"""GPU parity of the 8-bit quantised compressed cache against its oracle (oracle/stief_quant_oracle.py).
+
+A quantised code is an integer decided by floating point, so both sides decide in the same precision (fp32, the
+kernel's); what still differs is the fp32 accumulation order of the projection the quantiser sees.  A cache element
+therefore passes if its dequantised value is within one quantisation step of the oracle's (and the parameters agree to
+fp32 rounding of the row's extremes); the share of codes that differ at all is bounded.  The decode kernel is checked
+twice: tightly on the oracle's OWN codes uploaded to the device, and end to end (GPU prefill + append + decode) with
+the spec output tolerances (max-abs 1e-2, relative L2 5e-3)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2601_21686_b200 as S
+from oracle import stief_oracle as O
+from oracle import stief_quant_oracle as Q
+from paper_2601_21686_b200 import inputs as I
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+class QCase:
+    def __init__(self, seed, B, Hq, Hkv, r_k, r_v, seq_lens, reserve=2, shared_key_basis=False):
+        self.B, self.Hq, self.Hkv, self.r_k, self.r_v = B, Hq, Hkv, r_k, r_v
+        self.seq_lens = np.asarray(seq_lens, dtype=np.int32)
+        T = max(int(self.seq_lens.max()), 1)
+        self.K = I.lowrank_keys(seed, 0, B, T, Hkv)
+        self.V = I.gaussian_kv(seed, I.TAG_V, 0, B, T, Hkv)
+        self.q = I.queries(seed, 0, B, Hq)
+        self.U_k, self.U_v = I.stiefel_bases(seed, 0, Hkv, r_k, r_v, shared_key_basis=shared_key_basis)
+        self.pg = I.make_paging(seed, self.seq_lens, reserve_tokens=reserve, extra_pages=1)
+        Uk, Uv = U.f64(self.U_k), U.f64(self.U_v)
+        Kf, Vf = U.f64(self.K), U.f64(self.V)
+        # oracle side: fp32 projections, static key parameters calibrated per head on all rows of the batch
+        self.Kd = [[Q.project_f32(Kf[b, :n, h], O.basis_of(Uk, h)) for h in range(Hkv)] for b, n in enumerate(self.seq_lens)]
+        self.Vd = [[Q.project_f32(Vf[b, :n, h], O.basis_of(Uv, h)) for h in range(Hkv)] for b, n in enumerate(self.seq_lens)]
+        kp = []
+        for h in range(Hkv):
+            allrows = np.concatenate([self.Kd[b][h] for b in range(B) if self.seq_lens[b] > 0], 0)
+            s, z = Q.key_params_from_calibration(allrows * np.float32(1.25), 8)     # some headroom for appended rows
+            kp.append(np.stack([s, z], -1))
+        self.k_params = np.stack(kp).astype(np.float32)                              # [Hkv, ngk, 2]
+        P = self.pg.num_pages
+        fill = lambda shape, v, dt: torch.full(shape, v, dtype=dt, device=DEV)
+        self.layer = S.QLayer(Hq, Hkv, r_k, r_v, self.U_k.to(DEV), self.U_v.to(DEV), torch.from_numpy(self.k_params).to(DEV),
+                              fill((P, Hkv, 64, r_k), 0xAB, torch.uint8), fill((P, Hkv, 64, r_v), 0xCD, torch.uint8),
+                              fill((P, Hkv, 64, r_v // 64, 2), float("nan"), torch.float32))
+        bt = np.where(self.pg.block_table < 0, 0, self.pg.block_table).astype(np.int32)
+        self.batch = S.Batch(torch.from_numpy(bt).to(DEV), torch.from_numpy(self.seq_lens.copy()).to(DEV))
+        self.status = torch.zeros(1, dtype=torch.int32, device=DEV)
+
+    def oracle_cache(self, b, h, extra_k=None, extra_v=None):
+        Kd, Vd = self.Kd[b][h], self.Vd[b][h]
+        if extra_k is not None:
+            Kd, Vd = np.concatenate([Kd, extra_k], 0), np.concatenate([Vd, extra_v], 0)
+        ks, kz = self.k_params[h, :, 0], self.k_params[h, :, 1]
+        Kc = Q.quantize_keys(Kd, ks, kz, 8)
+        Vc, vs, vz = Q.quantize_values(Vd, 8)
+        return Kd, Vd, Kc, ks, kz, Vc, vs, vz
+
+    def gather(self, t, b, n):
+        """[n, Hkv, ...] rows of sequence b gathered from a device pool through the block table."""
+        p = t.cpu()
+        idx = torch.arange(n)
+        pages = torch.from_numpy(self.pg.block_table[b].astype(np.int64))[idx // 64]
+        return p[pages, :, idx % 64]
+
+
+def _check_cache(c: QCase):
+    mism = tot = 0
+    for b in range(c.B):
+        n = int(c.seq_lens[b])
+        if n == 0:
+            continue
+        gk = c.gather(c.layer.k_codes, b, n).numpy().astype(np.int32)
+        gv = c.gather(c.layer.v_codes, b, n).numpy().astype(np.int32)
+        gp = c.gather(c.layer.v_params, b, n).numpy()
+        for h in range(c.Hkv):
+            Kd, Vd, Kc, ks, kz, Vc, vs, vz = c.oracle_cache(b, h)
+            # keys: static parameters are inputs, so the codes may differ by one where the projection sits on a rounding edge
+            assert np.abs(gk[:, h] - Kc).max() <= 1
+            mism += int((gk[:, h] != Kc).sum()) + int((gv[:, h] != Vc).sum())
+            tot += Kc.size + Vc.size
+            # values: parameters from the row's own extremes (fp32 accumulation differences only)
+            assert np.allclose(gp[:, h, :, 0], vs, rtol=2e-4, atol=1e-7) and np.allclose(gp[:, h, :, 1], vz, rtol=1e-4, atol=2e-5)
+            deq_gpu = Q.dequant_values(gv[:, h], gp[:, h, :, 0], gp[:, h, :, 1])
+            deq_ref = Q.dequant_values(Vc, vs, vz)
+            step = np.repeat(vs, 64, axis=1)[:, :c.r_v]
+            assert np.all(np.abs(deq_gpu - deq_ref) <= 1.02 * step + 1e-5)
+            assert np.all(np.abs(deq_gpu - Vd) <= 0.52 * step + 2e-5)           # and each is a valid rounding of its row
+    assert mism <= max(4, 2e-3 * tot), f"{mism} of {tot} codes differ from the oracle's"
+
+
+def _untouched(c: QCase):
+    used = np.zeros((c.pg.num_pages, 64), dtype=bool)
+    for b in range(c.B):
+        for t in range(int(c.seq_lens[b])):
+            used[c.pg.block_table[b, t // 64], t % 64] = True
+    m = ~used[:, None, :].repeat(c.Hkv, 1)
+    assert np.all(c.layer.k_codes.cpu().numpy()[m] == 0xAB) and np.all(c.layer.v_codes.cpu().numpy()[m] == 0xCD)
+    assert np.all(np.isnan(c.layer.v_params.cpu().numpy()[m]))
+
+
+def _oracle_out(c: QCase, q, caches):
+    G = c.Hq // c.Hkv
+    out = np.zeros((c.B, c.Hq, 128))
+    lse = np.full((c.B, c.Hq), -np.inf)
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    qf = U.f64(q)
+    for b in range(c.B):
+        for g in range(c.Hq):
+            h = g // G
+            _, _, Kc, ks, kz, Vc, vs, vz = caches[b][h]
+            out[b, g], lse[b, g] = Q.attend_quantized_path_b(qf[b, g], Kc, ks, kz, Vc, vs, vz, O.basis_of(Uk, h), O.basis_of(Uv, h))
+    return out, lse
+
+
+def _workspace(c: QCase, parts):
+    ws = torch.full((S.stief_decode_workspace_bytes(c.B, c.Hq, c.Hkv, c.r_v, parts) // 4,), float("nan"), dtype=torch.float32, device=DEV)
+    S.stief_decode_workspace_init(ws)
+    return ws
+
+
+def _upload(c: QCase, caches):
+    kc, vc, vp = c.layer.k_codes.cpu(), c.layer.v_codes.cpu(), c.layer.v_params.cpu()
+    for b in range(c.B):
+        for h in range(c.Hkv):
+            _, _, Kc, ks, kz, Vc, vs, vz = caches[b][h]
+            for t in range(Kc.shape[0]):
+                pgi = int(c.pg.block_table[b, t // 64])
+                kc[pgi, h, t % 64] = torch.from_numpy(Kc[t].astype(np.uint8))
+                vc[pgi, h, t % 64] = torch.from_numpy(Vc[t].astype(np.uint8))
+                vp[pgi, h, t % 64, :, 0] = torch.from_numpy(vs[t])
+                vp[pgi, h, t % 64, :, 1] = torch.from_numpy(vz[t])
+    c.layer.k_codes.copy_(kc); c.layer.v_codes.copy_(vc); c.layer.v_params.copy_(vp)
+
+
+@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 64), (64, 128), (128, 128)])
+def test_q8_prefill_matches_the_oracles_quantiser(r_k, r_v):
+    c = QCase(200 + r_k + r_v, 3, 8, 2, r_k, r_v, [200, 64, 129])
+    S.stief_q8_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    _check_cache(c)
+    _untouched(c)
+
+
+@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 64), (64, 128), (128, 128)])
+def test_q8_decode_on_the_oracles_own_codes_is_tight(r_k, r_v):
+    c = QCase(300 + r_k + r_v, 2, 8, 2, r_k, r_v, [333, 70])
+    caches = [[c.oracle_cache(b, h) for h in range(c.Hkv)] for b in range(c.B)]
+    _upload(c, caches)
+    ref, ref_lse = _oracle_out(c, c.q, caches)
+    for parts in (1, 3, 0):
+        out = torch.full((c.B, c.Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+        lse = torch.full((c.B, c.Hq), float("nan"), dtype=torch.float32, device=DEV)
+        S.stief_q8_decode_attention(c.layer, c.batch, c.q.cuda(), _workspace(c, parts), out, parts, lse, status=c.status)
+        torch.cuda.synchronize()
+        assert int(c.status.item()) == 0
+        U.check_out(out, ref, max_abs=6e-3, rel_l2=3e-3)
+        assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 2e-3
+
+
+def test_q8_prefill_append_decode_end_to_end():
+    B, Hq, Hkv = 3, 16, 4
+    c = QCase(400, B, Hq, Hkv, 64, 64, [700, 63, 128], reserve=4)
+    S.stief_q8_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    k_new, v_new = I.new_token_kv(400, 0, B, Hkv)
+    S.stief_q8_append(c.layer, c.batch, k_new.cuda(), v_new.cuda(), status=c.status)
+    ws = _workspace(c, 0)
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    S.stief_q8_decode_attention(c.layer, c.batch, c.q.cuda(), ws, out, 0, lse, len_add=1, status=c.status)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    kn, vn = U.f64(k_new), U.f64(v_new)
+    caches = [[c.oracle_cache(b, h, Q.project_f32(kn[b, h][None], O.basis_of(Uk, h)), Q.project_f32(vn[b, h][None], O.basis_of(Uv, h)))
+               for h in range(Hkv)] for b in range(B)]
+    # the appended rows: codes within one of the oracle's, parameters from the row's extremes
+    for b in range(B):
+        n = int(c.seq_lens[b]) + 1
+        gk = c.gather(c.layer.k_codes, b, n).numpy().astype(np.int32)
+        gv = c.gather(c.layer.v_codes, b, n).numpy().astype(np.int32)
+        gp = c.gather(c.layer.v_params, b, n).numpy()
+        for h in range(Hkv):
+            _, _, Kc, ks, kz, Vc, vs, vz = caches[b][h]
+            assert np.abs(gk[-1, h] - Kc[-1]).max() <= 1 and np.abs(gv[-1, h] - Vc[-1]).max() <= 1
+            assert np.allclose(gp[-1, h, :, 0], vs[-1], rtol=2e-4) and np.allclose(gp[-1, h, :, 1], vz[-1], rtol=1e-4, atol=2e-5)
+    ref, ref_lse = _oracle_out(c, c.q, caches)
+    U.check_out(out, ref)
+    assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 5e-3
+
+
+def test_q8_rejects_unsupported_ranks_on_the_host():
+    c = QCase(500, 1, 4, 1, 64, 64, [100])
+    bad = S.QLayer(4, 1, 48, 64, c.layer.U_k, c.layer.U_v, c.layer.k_params, c.layer.k_codes, c.layer.v_codes, c.layer.v_params)
+    out = torch.empty(1, 4, 128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(S.StiefError) as e:
+        S.stief_q8_decode_attention(bad, c.batch, c.q.cuda(), _workspace(c, 0), out)
+    assert e.value.code == S.STIEF_ERR_UNSUPPORTED
