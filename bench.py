@@ -335,6 +335,96 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# config 2 on the 8-bit quantised cache (a measurement case, not the headline line)
+# ------------------------------------------------------------------------------------------------
+def run_q8(args):
+    import paper_2601_21686_b200 as S
+    from paper_2601_21686_b200 import inputs as I
+    from paper_2601_21686_b200 import build as Bld
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Bld.build()
+    S.lib()
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    cfg = dict(SINGLE_LAYER["config2"])
+    if args.ranks:
+        cfg["r_k"], cfg["r_v"] = (int(x) for x in args.ranks.split(","))
+    B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
+    n_caches = args.caches
+    pg = I.make_paging(SEED, [T] * B, reserve_tokens=1)
+    batch = S.Batch(torch.from_numpy(pg.block_table).to(dev), torch.from_numpy(pg.seq_lens).to(dev))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    layers, inputs = [], []
+    for l in range(n_caches):
+        U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
+        K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
+        V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
+        # static key parameters: calibrated on this prompt's own projected keys (min / max per head and 64-channel group)
+        Kd = torch.einsum("bthd,hdr->bthr", K.float(), U_k.to(dev).float())
+        mn = Kd.reshape(B * T, Hkv, r_k // 64, 64).amin(dim=(0, 3))
+        mx = Kd.reshape(B * T, Hkv, r_k // 64, 64).amax(dim=(0, 3))
+        kpar = torch.stack([(mx - mn) * 1.25 / 255.0, mn * 1.25], -1).contiguous()
+        del Kd
+        layers.append(S.QLayer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev), kpar,
+                               torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.uint8, device=dev),
+                               torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.uint8, device=dev),
+                               torch.zeros(pg.num_pages, Hkv, 64, r_v // 64, 2, dtype=torch.float32, device=dev)))
+        S.stief_q8_prefill_compress(layers[l], batch, K, V, status=status)
+        inputs.append((K, V))
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 3
+    e0.record()
+    for r in range(reps):
+        for l in range(n_caches):
+            S.stief_q8_prefill_compress(layers[l], batch, inputs[l][0], inputs[l][1], status=status,
+                                        flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if (r or l) else 0)
+    e1.record()
+    torch.cuda.synchronize()
+    pf_ms = e0.elapsed_time(e1) / (reps * n_caches)
+    del inputs
+    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, Hkv, r_v, 0) // 4, dtype=torch.float32, device=dev)
+    S.stief_decode_workspace_init(ws)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    n_in = 8
+    qs = [I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for i in range(n_in)]
+    kvs = [I.new_token_kv(SEED, 0, B, Hkv, device=dev, step=i) for i in range(n_in)]
+
+    def step(i):
+        S.stief_q8_append(layers[i % n_caches], batch, kvs[i % n_in][0], kvs[i % n_in][1], status=status)
+        S.stief_q8_decode_attention(layers[i % n_caches], batch, qs[i % n_in], ws, out, 0, len_add=1, status=status)
+
+    K_steps, W = min(args.steps, 2000), max(args.warmup, 3)
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(K_steps):
+        step(W + i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    per_unit = r_k + r_v + 8 * (r_v // 64)
+    sb = B * Hkv * (T + 1) * per_unit
+    gbs = sb * K_steps / (ms * 1e-3) / 1e9
+    pf_bytes = B * T * Hkv * (2 * 128 * 2 + per_unit)
+    print(json.dumps({
+        "metric": "q8_decode_attn_effective_hbm_gbs", "value": gbs, "unit": UNIT, "n_gpus": 1, "steps": K_steps, "warmup": W,
+        "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "dtype_note": "8-bit codes expanded to bf16 tensor-core operands, fp32 accumulate", "data": "synthetic",
+        "config": {"workload": cfg["name"] + f" on the 8-bit quantised cache ({per_unit} bytes per token and KV head instead of {2 * (r_k + r_v)}); "
+                               "step = append launch + attention launch", "l2": f"steps rotate over {n_caches} layer caches"},
+        "tokens_per_s": B * K_steps / (ms * 1e-3), "frac_of_hbm_peak": gbs / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
+        "bytes_per_step": sb, "gpu_launches": 2 * K_steps,
+        "same_step_in_bf16_cache_bytes_gbs": B * Hkv * (T + 1) * 2 * (r_k + r_v) * K_steps / (ms * 1e-3) / 1e9,
+        "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak}}))
+
+
+# ------------------------------------------------------------------------------------------------
 # the 32-layer workloads: config 3 (decode steps over per-layer ranks) and config 5 (prefill + first decode)
 # ------------------------------------------------------------------------------------------------
 def run_multilayer(args):
@@ -576,6 +666,7 @@ def main():
                     help="config2 is the headline line; the others are the remaining benchmark configurations")
     ap.add_argument("--num-parts", type=int, default=0, help="CTAs of the persistent decode kernel (0 = one per SM)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--q8", action="store_true", help="config 2 on the 8-bit quantised cache (measurement case)")
     ap.add_argument("--ranks", default=None, help="r_k,r_v override for the single-layer workloads, e.g. 48,96")
     ap.add_argument("--layers", type=int, default=32, help="layers of the multi-layer workloads (config3, config5)")
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
@@ -591,6 +682,8 @@ def main():
         args.steps = 128 if args.workload == "config3" else 5000
     if args.impl == "reference":
         run_reference(args)
+    elif args.q8:
+        run_q8(args)
     elif args.workload in SINGLE_LAYER:
         run_ours(args)
     else:
