@@ -370,7 +370,7 @@ def run_q8(args):
         del Kd
         layers.append(S.QLayer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev), kpar,
                                torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.uint8, device=dev),
-                               torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.uint8, device=dev),
+                               torch.zeros(pg.num_pages, Hkv, r_v, 64, dtype=torch.uint8, device=dev),
                                torch.zeros(pg.num_pages, Hkv, 64, r_v // 64, 2, dtype=torch.float32, device=dev)))
         S.stief_q8_prefill_compress(layers[l], batch, K, V, status=status)
         inputs.append((K, V))

@@ -213,7 +213,10 @@ int stief_decode_attention_static(const stief_layer* layer, const stief_batch* b
  * row when it is written: zero = min, scale = (max - min) / 255 over the group (scale = 1 when max == min).
  * The quantiser sees the projection K U_k / V U_v in fp32 (not rounded to bf16 first) and decides in fp32:
  * code = clamp(rint((x - zero) * (1 / scale))), ties to even.  Ranks must be 64 or 128 and both bases given.
- * Layout: k_codes, v_codes [num_pages][Hkv][64][r] uint8, r fastest, indexed like the bf16 pools;
+ * Layout: k_codes [num_pages][Hkv][64][r_k] uint8, r fastest, indexed like the bf16 pools; v_codes
+ * [num_pages][Hkv][r_v][64] uint8, CHANNEL-major inside a page, and token t of the page sits at position
+ * (t & ~15) + 4*((t & 7) >> 1) + (t & 1) + 2*((t >> 3) & 1) of its channel rows (the order in which the
+ * tensor-core mix consumes tokens: raw codes are its operands, nothing is expanded in shared memory);
  * k_params [Hkv][r_k / 64][2] fp32 (scale, zero); v_params [num_pages][Hkv][64][r_v / 64][2] fp32 (scale, zero).
  * Alignment: code pools and v_params 128 bytes, k_params 8 bytes.  Bytes per cached (token, KV head):
  * r_k + r_v + 8 * (r_v / 64), against 2 (r_k + r_v) for the bf16 cache. */

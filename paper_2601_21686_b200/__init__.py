@@ -128,8 +128,8 @@ class Layer:
 @dataclass
 class QLayer:
     """One decoder layer's 8-bit quantised compressed cache (device tensors): U_k [Hkv or 1, 128, r_k], U_v
-    [Hkv or 1, 128, r_v] bf16; k_params [Hkv, r_k/64, 2] fp32 (scale, zero; static); k_codes / v_codes
-    [num_pages, Hkv, 64, r] uint8; v_params [num_pages, Hkv, 64, r_v/64, 2] fp32 (scale, zero per token and group)."""
+    [Hkv or 1, 128, r_v] bf16; k_params [Hkv, r_k/64, 2] fp32 (scale, zero; static); k_codes [num_pages, Hkv, 64, r_k] uint8;
+    v_codes [num_pages, Hkv, r_v, 64] uint8 (channel-major pages with permuted token positions, see stief.h); v_params [num_pages, Hkv, 64, r_v/64, 2] fp32 (scale, zero per token and group)."""
     Hq: int
     Hkv: int
     r_k: int

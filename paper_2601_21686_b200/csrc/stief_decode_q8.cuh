@@ -1,18 +1,25 @@
 // Decode attention over the 8-bit quantised compressed cache (paper Sec. 4.3): the persistent split-T kernel of
-// stief_decode.cuh with a different way of getting a page's operands into shared memory.  The cache holds
-// K codes [64 x RK] and V codes [64 x RV] (uint8) per (page, head) plus the value rows' (scale, zero) pairs; the
-// three contiguous blocks of a page are fetched with 1-D bulk async copies into the lane's ring stage.  The
-// consuming warp then expands them once into bf16 operand tiles in a private scratch area (swizzled like the bf16
-// kernel's TMA tiles) -- key codes as they are (integers up to 255 are exact in bf16; the key scale is folded into
-// the projected query and the key zero-point only shifts a row's scores by a constant, so it enters out_lse alone),
-// value codes dequantised as code * scale + zero -- frees the stage at once, and runs the same tensor-core score /
-// online-softmax / mix code as the bf16 kernel on the scratch tiles.  Partition, prologue (query projection, no
-// fused append here), segment merge and last-arriver combine are the bf16 kernel's.
+// stief_decode.cuh with the page operands kept as integer codes all the way into the tensor cores.
 //
-// This first version spends more issue slots on the expansion than the bf16 kernel spends on a whole page, so it
-// is bound by that, not by HBM: what it buys is cache capacity (136 instead of 256 bytes per token and head at rank
-// 64/64).  The faster route (integer tensor-core MMAs on the raw codes with value pages stored channel-major) is
-// described in the design notes.
+// The cache holds, per (page, head): K codes [64 tokens][RK] uint8 (token-major), V codes [RV channels][64
+// positions] uint8 (channel-major, see below) and the value rows' (scale, zero) pairs.  K and V tiles are fetched by
+// TMA box loads with a hardware swizzle (ldmatrix then reads them without bank conflicts), the parameters by a 1-D
+// bulk copy.  Both contractions run on mma.sync.m16n8k32 (s8 x u8 -> s32) with the raw codes as the B operand:
+//   scores: A = q' (key scale folded in) as a per-row 16-bit fixed point split into two signed 8-bit digits, which
+//           occupy rows 0-7 and 8-15 of the 16-row operand; the integer sums are recombined as 256 hi + lo and
+//           scaled back per row.  The key zero-point shifts all scores of a row equally: it only enters out_lse.
+//   mix:    A = p_t * scale_t,g per value group g, again as two digits of a per-row, per-page fixed point; the value
+//           zero-points add sum_t p_t zero_t,g to every channel of the group (kept as a running scalar per group).
+// No code is ever expanded to floating point in shared memory.
+//
+// Why value pages are channel-major and their 64 token positions permuted: the B fragment of the mix needs four
+// consecutive TOKENS of one channel in a register, which is what ldmatrix delivers from channel-major rows; and the
+// A fragment wants, for the thread (gid, tid4), the probabilities of k-slots 4 tid4 .. 4 tid4 + 3 of each 16-slot
+// chunk, while the score accumulators leave that thread with tokens 2 tid4, 2 tid4 + 1 of each 8-token tile.  So
+// within every 16 tokens, token u sits at position 4 (u mod 8 / 2) + (u mod 2) + 2 (u / 8): the thread's own
+// probabilities are then exactly its A fragment and no lane ever exchanges data (v_position() below).
+//
+// Four page lanes, each with its own producer warp and two consumer warps that take 32 tokens of a page each.
 #pragma once
 
 #include "stief_decode.cuh"
@@ -38,39 +45,65 @@ struct DecodeQ8Args {
   int32_t* status;
 };
 
+// position of token t (0..63) inside a value page's channel rows
+__host__ __device__ __forceinline__ int v_position(int t) {
+  const int u = t & 15;
+  return (t & ~15) + 4 * ((u & 7) >> 1) + (u & 1) + 2 * (u >> 3);
+}
+
 template <int RK, int RV>
 struct DecodeQ8Cfg {
-  using TK = Tile<RK>;
-  using TV = Tile<RV>;
+  using TK = Tile<RK / 2>;               // 64 rows of RK bytes have the geometry of 64 rows of RK/2 bf16
+  using TV = Tile<32>;                   // channel rows of 64 bytes (64-byte swizzle), RV of them
   static constexpr int NGV = RV / 64;
   static constexpr int K_BYTES = kPage * RK, V_BYTES = kPage * RV, P_BYTES = kPage * NGV * 8;
-  static constexpr int STAGE_BYTES = K_BYTES + V_BYTES + P_BYTES;        // all multiples of 16
-  static constexpr int SCRATCH_BYTES = TK::BYTES + TV::BYTES;            // one lane's bf16 operand tiles
-  static constexpr int HALF = 1;
+  static constexpr int TX_BYTES = K_BYTES + V_BYTES + P_BYTES;           // bytes one page brings into a stage
+  static constexpr int STAGE_BYTES = (TX_BYTES + 1023) / 1024 * 1024;    // stages keep the key tile's swizzle alignment
+  static constexpr int HALF = 2;
+  static constexpr int NP = 4;
+  static constexpr int NW = NP * HALF;
+  static constexpr int NT = NW * 32;
+  static constexpr int THREADS = NT + NP * 32;
   static constexpr int CTRL_BYTES = 512;
   static constexpr int PREF_BYTES = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
   static constexpr int QP_BYTES = kGroupTile * kD * 4;
   static constexpr int ROWS_BYTES = 10 * kD * 4;
-  static constexpr int MISC4 = CTRL_BYTES + PREF_BYTES + QP_BYTES + ROWS_BYTES + 4 * 9 * kD * 4;
-  // four page lanes when their scratch tiles leave room for at least two stages each, else two
-  static constexpr int NP = (232448 - 1024 - MISC4 - 4 * SCRATCH_BYTES >= 4 * 2 * STAGE_BYTES) ? 4 : 2;
-  static constexpr int NW = NP * HALF;
-  static constexpr int NT = NW * 32;
-  static constexpr int THREADS = NT + NP * 32;
   static constexpr int RED_BYTES = NW * 9 * kD * 4;
-  static constexpr int UNION_BYTES = (ROWS_BYTES + RED_BYTES) > 24576 ? (ROWS_BYTES + RED_BYTES) : 24576;
+  static constexpr int UNION_BYTES = ROWS_BYTES + RED_BYTES;
   static constexpr int MISC = CTRL_BYTES + PREF_BYTES + QP_BYTES + UNION_BYTES;
-  static constexpr int RING_BUDGET = 232448 - 1024 - MISC - NP * SCRATCH_BYTES;
+  static constexpr int RING_BUDGET = 232448 - 1024 - MISC;
   static constexpr int SPW = (RING_BUDGET / (NP * STAGE_BYTES)) > 4 ? 4 : (RING_BUDGET / (NP * STAGE_BYTES));
   static constexpr int NS = NP * SPW;
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
-  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + NP * SCRATCH_BYTES + MISC;
+  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + MISC;
   static_assert(RK % 64 == 0 && RV % 64 == 0 && RK <= 128 && RV <= 128, "quantisation groups are 64 channels");
+  static_assert(TK::NB == 1 && TK::BYTES == K_BYTES, "key tile is one swizzled box");
+  static_assert(STAGE_BYTES % 1024 == 0 && K_BYTES % 1024 == 0, "tiles keep their swizzle alignment");
   static_assert(SPW >= 2 && NS <= 16, "ring shape");
   static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= UNION_BYTES, "merge scratch must fit");
   static_assert(kCombineScratchFloats * 4 <= UNION_BYTES, "combine scratch must fit");
   static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KiB shared memory of an SM");
 };
+
+// D += A(16x32, row, s8) * B(32x8, col, u8), s32 accumulate
+__device__ __forceinline__ void mma_s8u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Two signed 8-bit digits of a 16-bit fixed-point value a in [-32640, 32639]: a = 256 hi + lo, both in [-128, 127]
+__device__ __forceinline__ void digits(float x, float inv_delta, int& hi, int& lo) {
+  int v = __float2int_rn(x * inv_delta);
+  v = max(-32640, min(32639, v));
+  hi = (v + 128) >> 8;
+  lo = v - (hi << 8);
+}
+__device__ __forceinline__ uint32_t pack4(int b0, int b1, int b2, int b3) {
+  return (uint32_t)(b0 & 0xff) | ((uint32_t)(b1 & 0xff) << 8) | ((uint32_t)(b2 & 0xff) << 16) | ((uint32_t)(b3 & 0xff) << 24);
+}
+constexpr float kFixedMax = 32639.f;
 
 // 1-D bulk async copy global -> shared (both 16-byte aligned, size a multiple of 16), completion in bytes on an mbarrier
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -82,13 +115,13 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 
 template <int RK, int RV>
 __global__ void __launch_bounds__(DecodeQ8Cfg<RK, RV>::THREADS, 1)
-decode_q8_kernel(const DecodeQ8Args a) {
+decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeQ8Args a) {
   using C = DecodeQ8Cfg<RK, RV>;
   using TK = typename C::TK;
   using TV = typename C::TV;
   constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW, NT = C::NT, NP = C::NP, HALF = C::HALF;
-  constexpr int NJ = 8 / HALF;                           // 8-token score tiles per consumer warp and page
-  constexpr int KK = 4 / HALF;                           // 16-token contraction steps of the mix per warp and page
+  constexpr int NJ = 4;                                  // 8-token score tiles per consumer warp and page (32 tokens)
+  constexpr int NGV = C::NGV;
 
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -96,14 +129,14 @@ decode_q8_kernel(const DecodeQ8Args a) {
 
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
-  const uint32_t scratch = ring + C::RING_BYTES;                        // NP lanes x (K tile, V tile) in bf16
-  uint8_t* ctrl_ptr = ring_ptr + C::RING_BYTES + NP * C::SCRATCH_BYTES;
-  const uint32_t ctrl = scratch + NP * C::SCRATCH_BYTES;
+  uint8_t* ctrl_ptr = ring_ptr + C::RING_BYTES;
+  const uint32_t ctrl = ring + C::RING_BYTES;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (16 + s) * 8; };
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8);
   volatile int* last_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);
   float* lse_shift = reinterpret_cast<float*>(ctrl_ptr + 34 * 8);      // [8]: q' . key zero-point / sqrt(128) of the unit's rows
+  float* q_delta = reinterpret_cast<float*>(ctrl_ptr + 38 * 8);        // [8]: fixed-point step of the unit's scaled query rows
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -137,6 +170,10 @@ decode_q8_kernel(const DecodeQ8Args a) {
   // cycles of waits and descriptor traffic whatever its size), so the issue work is split the way the pages are.
   if (warp >= NW) {
     const int pw = warp - NW;
+    if (lane == 0) {
+      tma_prefetch_desc(&tmK);
+      tma_prefetch_desc(&tmV);
+    }
     int i_base = 0;            // pages of this CTA before the current segment
     while (walk.next(seg)) {
       const int h = seg.j / QT;
@@ -160,9 +197,9 @@ decode_q8_kernel(const DecodeQ8Args a) {
           if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
           const uint32_t st = ring + slot * C::STAGE_BYTES;
           const size_t tile = (size_t)page * Hkv + h;
-          mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
-          bulk_load_1d(st, a.k_codes + tile * C::K_BYTES, C::K_BYTES, full_bar(slot));
-          bulk_load_1d(st + C::K_BYTES, a.v_codes + tile * C::V_BYTES, C::V_BYTES, full_bar(slot));
+          mbar_arrive_expect_tx(full_bar(slot), C::TX_BYTES);
+          tma_load_2d(st, &tmK, 0, (int)tile * kPage, full_bar(slot));                  // 64 token rows of RK bytes
+          tma_load_2d(st + C::K_BYTES, &tmV, 0, (int)tile * RV, full_bar(slot));        // RV channel rows of 64 bytes
           bulk_load_1d(st + C::K_BYTES + C::V_BYTES, a.v_params + tile * (C::P_BYTES / 4), C::P_BYTES, full_bar(slot));
         }
         __syncwarp();
@@ -176,18 +213,14 @@ decode_q8_kernel(const DecodeQ8Args a) {
   const int gid = lane >> 2, tid4 = lane & 3, l7 = lane & 7;
   const float qscale = kLog2e * 0.08838834764831845f;     // log2(e) / sqrt(128)
 
-  // per-lane pieces of the ldmatrix addresses (the swizzle term depends on the lane only)
-  constexpr int NCH = RK / 8;
-  uint32_t koff[(NCH + 3) / 4];
+  // per-lane pieces of the ldmatrix addresses (the swizzle term depends on the lane only).  A key ldmatrix.x4
+  // covers 8 tokens x 64 channels (four 16-byte chunks); a value ldmatrix.x4 covers two 8-channel tiles x the
+  // warp's 32 positions (two chunks each).
+  const int pl = warp % NP, hf = warp / NP;               // page lane; which 32 tokens of a page this warp takes
+  uint32_t koff[RK / 64];
 #pragma unroll
-  for (int q4 = 0; q4 < (NCH + 3) / 4; ++q4) {
-    const int cc = (4 * q4 + 4 <= NCH) ? 4 * q4 + (lane >> 3) : 4 * q4 + ((lane >> 3) & 1);
-    koff[q4] = TK::chunk(l7, cc);
-  }
-  uint32_t voff[RV / 16];
-#pragma unroll
-  for (int np = 0; np < RV / 16; ++np) voff[np] = TV::chunk(l7 + ((lane >> 3) & 1) * 8, 2 * np + (lane >> 4));
-
+  for (int ks = 0; ks < RK / 64; ++ks) koff[ks] = TK::chunk(l7, 4 * ks + (lane >> 3));
+  const uint32_t voff = TV::chunk(l7 + 8 * (lane >> 4), 2 * hf + ((lane >> 3) & 1));
   int i_base = 0;              // pages of this CTA before the current segment
 
   while (walk.next(seg)) {
@@ -242,112 +275,90 @@ decode_q8_kernel(const DecodeQ8Args a) {
       lse_shift[tid] = sh * 0.08838834764831845f;          // / sqrt(128)
     }
     bar1(NT);
+    if (tid < 8) {                                         // fixed-point step of each scaled query row
+      float mx = 0.f;
+      for (int j = 0; j < RK; ++j) mx = fmaxf(mx, fabsf(qp[tid * RK + j]));
+      q_delta[tid] = mx > 0.f ? mx / kFixedMax : 1.f;
+    }
+    bar1(NT);
 
-    // A operand of the score MMA: rows 0-7 = bf16(q'), rows 8-15 = bf16(q' - bf16(q'))
-    uint32_t qa[RK / 16][4];
+    // A operand of the score MMA: rows 0-7 = high digits of the scaled query rows, rows 8-15 = low digits
+    const float dq = q_delta[gid];
+    uint32_t qa[RK / 32][4];
+    {
+      const float inv = 1.f / dq;
 #pragma unroll
-    for (int ks = 0; ks < RK / 16; ++ks) {
-      const float2 x = *reinterpret_cast<const float2*>(qp + gid * RK + 16 * ks + 2 * tid4);
-      const float2 y = *reinterpret_cast<const float2*>(qp + gid * RK + 16 * ks + 8 + 2 * tid4);
-      split_bf16(x.x, x.y, qa[ks][0], qa[ks][1]);
-      split_bf16(y.x, y.y, qa[ks][2], qa[ks][3]);
+      for (int ks = 0; ks < RK / 32; ++ks) {
+        int hi[8], lo[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          digits(qp[gid * RK + 32 * ks + 4 * tid4 + e], inv, hi[e], lo[e]);
+          digits(qp[gid * RK + 32 * ks + 16 + 4 * tid4 + e], inv, hi[4 + e], lo[4 + e]);
+        }
+        qa[ks][0] = pack4(hi[0], hi[1], hi[2], hi[3]);
+        qa[ks][1] = pack4(lo[0], lo[1], lo[2], lo[3]);
+        qa[ks][2] = pack4(hi[4], hi[5], hi[6], hi[7]);
+        qa[ks][3] = pack4(lo[4], lo[5], lo[6], lo[7]);
+      }
     }
 
     float m = -INFINITY, l = 0.f;
-    float o[RV / 8][4];
+    float o[RV / 8][2];                                    // row gid, channels 8 n + 2 tid4, + 1
+    float zc[NGV];                                         // sum_t p_t zero_t,g over this thread's tokens
 #pragma unroll
-    for (int n = 0; n < RV / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    for (int n = 0; n < RV / 8; ++n) o[n][0] = o[n][1] = 0.f;
+#pragma unroll
+    for (int g = 0; g < NGV; ++g) zc[g] = 0.f;
 
     // first page of this segment that belongs to this warp's lane: global index i = i_base + k, i % NP == pl
-    const int pl = warp % NP, hf = warp / NP;
-    const int tb = hf * (kPage / HALF);                    // first token of the page this warp handles
+    const int tb = 32 * hf;                                // first token of the page this warp handles
     int k0 = (pl - i_base % NP + NP) % NP;
     for (int k = k0; k < npg; k += NP) {
       const int kw = (i_base + k) / NP;
       const int slot = pl * SPW + kw % SPW;
       mbar_wait(full_bar(slot), (kw / SPW) & 1, abort_flag, a.status);
+      const uint32_t kt = ring + slot * C::STAGE_BYTES;
+      const uint32_t vt = kt + C::K_BYTES;
+      const uint32_t pt = vt + C::V_BYTES;
       const bool tail = (seg.p0 + k == seg.npages - 1) && (last_valid < kPage);
-      // ---- expand the page's codes into this lane's bf16 operand tiles, then give the stage back
-      const uint32_t st = ring + slot * C::STAGE_BYTES;
-      const uint32_t kt = scratch + pl * C::SCRATCH_BYTES;
-      const uint32_t vt = kt + TK::BYTES;
-      __syncwarp();                                        // the previous page's ldmatrix reads of the tiles are done
-      {
-        constexpr int KP = RK / 16;                        // 16-byte pieces (16 codes) per key row
-#pragma unroll 4
-        for (int idx = lane; idx < kPage * KP; idx += 32) {
-          const int t = idx / KP, pc = idx % KP;
-          uint32_t w0, w1, w2, w3;
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(st + idx * 16));
-          const uint32_t w[4] = {w0, w1, w2, w3};
-          uint32_t o[8];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {                    // integers up to 255 are exact in bf16
-            o[2 * e] = pack_bf16((float)(w[e] & 0xffu), (float)((w[e] >> 8) & 0xffu));
-            o[2 * e + 1] = pack_bf16((float)((w[e] >> 16) & 0xffu), (float)(w[e] >> 24));
-          }
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(kt + TK::chunk(t, 2 * pc)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(kt + TK::chunk(t, 2 * pc + 1)), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-        }
-        constexpr int VP = RV / 16;
-        const uint32_t vs = st + C::K_BYTES, ps = vs + C::V_BYTES;
-#pragma unroll 4
-        for (int idx = lane; idx < kPage * VP; idx += 32) {
-          const int t = idx / VP, pc = idx % VP;
-          uint32_t w0, w1, w2, w3;
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(vs + idx * 16));
-          float sc, zp;                                    // the row's parameters of the group this piece lies in
-          asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(sc), "=f"(zp) : "r"(ps + (t * C::NGV + (pc >> 2)) * 8));
-          const uint32_t w[4] = {w0, w1, w2, w3};
-          uint32_t o[8];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            o[2 * e] = pack_bf16(fmaf((float)(w[e] & 0xffu), sc, zp), fmaf((float)((w[e] >> 8) & 0xffu), sc, zp));
-            o[2 * e + 1] = pack_bf16(fmaf((float)((w[e] >> 16) & 0xffu), sc, zp), fmaf((float)(w[e] >> 24), sc, zp));
-          }
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(vt + TV::chunk(t, 2 * pc)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(vt + TV::chunk(t, 2 * pc + 1)), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-        }
+      if (tail && last_valid <= tb) {                      // none of this warp's tokens exists: nothing to add
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(slot));
+        continue;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_bar(slot));         // the stage's bytes have been read: it may be refilled
 
-      // ---- scores of the page: n-tile j covers tokens 8j..8j+7; c0,c1 from bf16(q'), c2,c3 from the remainder
+      // ---- scores of the warp's 32 tokens: tile j covers tokens tb + 8j .. + 7; integer sums of both digits
       float sc[2 * NJ];
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        int s4[4] = {0, 0, 0, 0};
 #pragma unroll
-        for (int q4 = 0; 4 * q4 + 4 <= NCH; ++q4) {
+        for (int ks = 0; ks < RK / 64; ++ks) {
           uint32_t r0, r1, r2, r3;
-          ldsm_x4(kt + koff[q4] + (hf * NJ + j) * 8 * TK::RB, r0, r1, r2, r3);
-          mma_bf16(s, qa[2 * q4], r0, r1);
-          mma_bf16(s, qa[2 * q4 + 1], r2, r3);
+          ldsm_x4(kt + koff[ks] + (tb + 8 * j) * TK::RB, r0, r1, r2, r3);
+          mma_s8u8(s4, qa[2 * ks], r0, r1);
+          mma_s8u8(s4, qa[2 * ks + 1], r2, r3);
         }
-        if constexpr (NCH % 4 == 2) {
-          uint32_t r0, r1;
-          ldsm_x2(kt + koff[NCH / 4] + (hf * NJ + j) * 8 * TK::RB, r0, r1);
-          mma_bf16(s, qa[NCH / 2 - 1], r0, r1);
-        }
-        sc[2 * j] = s[0] + s[2];
-        sc[2 * j + 1] = s[1] + s[3];
+        sc[2 * j] = dq * (float)(256 * s4[0] + s4[2]);
+        sc[2 * j + 1] = dq * (float)(256 * s4[1] + s4[3]);
       }
-      if (tail) {
+      // value parameters of this thread's 8 tokens (token of tile j, element e: tb + 8j + 2 tid4 + e)
+      float vs[NGV][2 * NJ], vz[NGV][2 * NJ];
 #pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-          const int t = tb + 8 * j + 2 * tid4;
-          if (t >= last_valid) sc[2 * j] = -INFINITY;
-          if (t + 1 >= last_valid) sc[2 * j + 1] = -INFINITY;
+      for (int j = 0; j < NJ; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int t = tb + 8 * j + 2 * tid4 + e;
+          const bool ok = !tail || t < last_valid;
+          if (!ok) sc[2 * j + e] = -INFINITY;
+#pragma unroll
+          for (int g = 0; g < NGV; ++g) {
+            float x, y;
+            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(x), "=f"(y) : "r"(pt + (t * NGV + g) * 8));
+            vs[g][2 * j + e] = ok ? x : 0.f;               // rows past the end hold unspecified bits
+            vz[g][2 * j + e] = ok ? y : 0.f;
+          }
         }
-        // rows past the end hold unspecified bits: zero them in V so that 0 * garbage cannot make a NaN
-        constexpr int NCV = RV / 8;
-        const int z0 = max(last_valid, tb);                // this warp's rows past the end
-        for (int idx = lane; idx < (tb + kPage / HALF - z0) * NCV; idx += 32) {
-          const int t = z0 + idx / NCV, cc = idx % NCV;
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vt + TV::chunk(t, cc)), "r"(0u) : "memory");
-        }
-        __syncwarp();
-      }
 
       // ---- online softmax (base 2; the scale is folded into q')
       float mx = sc[0];
@@ -358,34 +369,57 @@ decode_q8_kernel(const DecodeQ8Args a) {
       const float m_new = fmaxf(m, mx);
       const float alpha = fast_exp2(m - m_new);
       m = m_new;
-      uint32_t pa[KK][4];
+      float pr[2 * NJ];
       float ps = 0.f;
 #pragma unroll
-      for (int kk = 0; kk < KK; ++kk) {
-        const float p0_ = fast_exp2(sc[4 * kk + 0] - m), p1_ = fast_exp2(sc[4 * kk + 1] - m);
-        const float p2_ = fast_exp2(sc[4 * kk + 2] - m), p3_ = fast_exp2(sc[4 * kk + 3] - m);
-        ps += (p0_ + p1_) + (p2_ + p3_);
-        split_bf16(p0_, p1_, pa[kk][0], pa[kk][1]);
-        split_bf16(p2_, p3_, pa[kk][2], pa[kk][3]);
+      for (int e = 0; e < 2 * NJ; ++e) {
+        pr[e] = fast_exp2(sc[e] - m);
+        ps += pr[e];
       }
       l = l * alpha + ps;
 #pragma unroll
       for (int n = 0; n < RV / 8; ++n) {
-        o[n][0] *= alpha; o[n][1] *= alpha; o[n][2] *= alpha; o[n][3] *= alpha;
+        o[n][0] *= alpha;
+        o[n][1] *= alpha;
       }
 
-      // ---- mix: o += P V_down (tokens are the contraction index; V tile read transposed)
+      // ---- mix: per value group, p_t * scale_t,g as two digits of a per-row fixed point against the raw codes
 #pragma unroll
-      for (int kk = 0; kk < KK; ++kk) {
+      for (int g = 0; g < NGV; ++g) {
+        float w[2 * NJ], wmax = 0.f, zsum = 0.f;
 #pragma unroll
-        for (int np = 0; np < RV / 16; ++np) {
+        for (int e = 0; e < 2 * NJ; ++e) {
+          w[e] = pr[e] * vs[g][e];
+          wmax = fmaxf(wmax, w[e]);
+          zsum = fmaf(pr[e], vz[g][e], zsum);
+        }
+        zc[g] = zc[g] * alpha + zsum;
+        wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, 1));
+        wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, 2));
+        const float dp = wmax > 0.f ? wmax / kFixedMax : 1.f;
+        const float inv = 1.f / dp;
+        int hi[8], lo[8];
+#pragma unroll
+        for (int e = 0; e < 2 * NJ; ++e) digits(w[e], inv, hi[e], lo[e]);
+        // k-slots 4 tid4 .. + 3 of the first 16 positions hold tiles 0 and 1, of the second 16 tiles 2 and 3
+        const uint32_t pa[4] = {pack4(hi[0], hi[1], hi[2], hi[3]), pack4(lo[0], lo[1], lo[2], lo[3]),
+                                pack4(hi[4], hi[5], hi[6], hi[7]), pack4(lo[4], lo[5], lo[6], lo[7])};
+#pragma unroll
+        for (int n2 = 0; n2 < 4; ++n2) {                   // two 8-channel tiles per ldmatrix: 64 channels per group
+          const int n = 8 * g + 2 * n2;
           uint32_t r0, r1, r2, r3;
-          ldsm_x4_t(vt + voff[np] + (hf * KK + kk) * 16 * TV::RB, r0, r1, r2, r3);
-          mma_bf16(o[2 * np], pa[kk], r0, r1);
-          mma_bf16(o[2 * np + 1], pa[kk], r2, r3);
+          ldsm_x4(vt + voff + n * 8 * TV::RB, r0, r1, r2, r3);
+          int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
+          mma_s8u8(c0, pa, r0, r1);
+          mma_s8u8(c1, pa, r2, r3);
+          o[n][0] = fmaf(dp, (float)(256 * c0[0] + c0[2]), o[n][0]);
+          o[n][1] = fmaf(dp, (float)(256 * c0[1] + c0[3]), o[n][1]);
+          o[n + 1][0] = fmaf(dp, (float)(256 * c1[0] + c1[2]), o[n + 1][0]);
+          o[n + 1][1] = fmaf(dp, (float)(256 * c1[1] + c1[3]), o[n + 1][1]);
         }
       }
-
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar(slot));
     }
     i_base += npg;
 
@@ -396,8 +430,13 @@ decode_q8_kernel(const DecodeQ8Args a) {
     float* wm = wo + NW * 8 * RV;        // [NW][8]
     float* wl = wm + NW * 8;             // [NW][8]
 #pragma unroll
+    for (int g = 0; g < NGV; ++g) {                        // the group's zero-point term, summed over the row's four threads
+      zc[g] += __shfl_xor_sync(0xffffffffu, zc[g], 1);
+      zc[g] += __shfl_xor_sync(0xffffffffu, zc[g], 2);
+    }
+#pragma unroll
     for (int n = 0; n < RV / 8; ++n) {
-      *reinterpret_cast<float2*>(wo + (warp * 8 + gid) * RV + 8 * n + 2 * tid4) = make_float2(o[n][0] + o[n][2], o[n][1] + o[n][3]);
+      *reinterpret_cast<float2*>(wo + (warp * 8 + gid) * RV + 8 * n + 2 * tid4) = make_float2(o[n][0] + zc[n / 8], o[n][1] + zc[n / 8]);
     }
     if (tid4 == 0) {
       wm[warp * 8 + gid] = m;

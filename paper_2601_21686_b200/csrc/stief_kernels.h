@@ -54,6 +54,9 @@ cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const C
 // given swizzle.  Returns false when the driver entry point is missing or refuses the arguments.
 bool encode_bf16_map(CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
                      const unsigned long long* strides_bytes, const unsigned* box, CUtensorMapSwizzle swizzle);
+// The same for a tensor of bytes.
+bool encode_u8_map(CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
+                   const unsigned long long* strides_bytes, const unsigned* box, CUtensorMapSwizzle swizzle);
 // Full-rank side of the prefill (no basis): the rows are copied to the pool unchanged.  side: 0 = keys, 1 = values.
 cudaError_t launch_prefill_copy(const PrefillArgs& a, int side, cudaStream_t st);
 // Shape of the TMA boxes the decode kernel expects for rank r (see Tile<R>).

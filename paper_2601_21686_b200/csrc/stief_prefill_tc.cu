@@ -53,6 +53,12 @@ struct Args {
   const float* k_params;
 };
 
+// position of token t (0..63) inside a quantised value page's channel rows (see stief_decode_q8.cuh)
+__device__ __forceinline__ int q8_v_position(int t) {
+  const int u = t & 15;
+  return (t & ~15) + 4 * ((u & 7) >> 1) + (u & 1) + 2 * (u >> 3);
+}
+
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
   asm volatile(
@@ -475,7 +481,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   *reinterpret_cast<float2*>(a.v_params + (((size_t)row0 + lane) * ng + g) * 2) = make_float2(sc, zp);
                 }
                 const float inv = __fdiv_rn(1.f, sc);
-                uint8_t* qdst = (t.side ? a.v_codes : a.k_codes) + ((size_t)row0 + lane) * R + 64 * g;
+                if (t.side) {
+                  // value codes are stored channel-major with the page's 64 positions permuted (v_position): the
+                  // 32 lanes of the warp write 32 bytes of one channel row
+                  const int tp = (row0 % kPage) + lane;                               // token within its page
+                  uint8_t* vrow = a.v_codes + ((size_t)(row0 / kPage) * R + 64 * g) * kPage + q8_v_position(tp);
+#pragma unroll
+                  for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                      const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][e]), zp), inv);
+                      vrow[(size_t)(16 * c + e) * kPage] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+                    }
+                } else {
+                uint8_t* qdst = a.k_codes + ((size_t)row0 + lane) * R + 64 * g;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                   uint32_t w[4];
@@ -491,6 +510,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     w[e4] = word;
                   }
                   *reinterpret_cast<uint4*>(qdst + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
                 }
               }
             } else {

@@ -79,7 +79,10 @@ append_q8_kernel(const AppendQ8Args a) {
   }
   if (j < R) {
     const float y = __fmul_rn(__fsub_rn(acc, zp), __fdiv_rn(1.f, sc));
-    (side ? a.v_codes : a.k_codes)[row * R + j] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+    const uint8_t code = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+    const size_t tile = (size_t)page * a.L.Hkv + h;
+    if (side == 0) a.k_codes[row * R + j] = code;                                             // [token][channel]
+    else a.v_codes[(tile * R + j) * kPage + v_position(pos % kPage)] = code;                  // [channel][position]
   }
 }
 
@@ -108,7 +111,21 @@ static cudaError_t launch_decode_q8(const DecodeQ8Args& a, int n_cta, bool overl
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = overlap_previous ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kern, a);
+  // key codes: [tiles * 64 token rows][RK bytes], one box per tile; value codes: [tiles * RV channel rows][64 bytes]
+  const unsigned long long tiles = (unsigned long long)a.L.num_pages * a.L.Hkv;
+  CUtensorMap tmK, tmV;
+  {
+    const unsigned long long dims[2] = {(unsigned long long)RK, tiles * kPage}, strides[1] = {(unsigned long long)RK};
+    const unsigned box[2] = {(unsigned)RK, (unsigned)kPage};
+    if (!encode_u8_map(&tmK, a.k_codes, 2, dims, strides, box, RK == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
+      return cudaErrorInvalidValue;
+  }
+  {
+    const unsigned long long dims[2] = {(unsigned long long)kPage, tiles * RV}, strides[1] = {(unsigned long long)kPage};
+    const unsigned box[2] = {(unsigned)kPage, (unsigned)RV};
+    if (!encode_u8_map(&tmV, a.v_codes, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B)) return cudaErrorInvalidValue;
+  }
+  return cudaLaunchKernelEx(&cfg, kern, tmK, tmV, a);
 }
 
 namespace {

@@ -20,6 +20,18 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+def vpos(t):
+    """Position of token t (0..63 within its page) inside a value page's channel rows: the documented layout."""
+    t = np.asarray(t)
+    return (t & ~15) + 4 * ((t & 7) >> 1) + (t & 1) + 2 * ((t >> 3) & 1)
+
+
+def test_value_positions_are_a_permutation_of_each_16_tokens():
+    p = vpos(np.arange(64))
+    assert sorted(p.tolist()) == list(range(64)) and np.all(p // 16 == np.arange(64) // 16)
+    assert p[:16].tolist() == [0, 1, 4, 5, 8, 9, 12, 13, 2, 3, 6, 7, 10, 11, 14, 15]
+
+
 class QCase:
     def __init__(self, seed, B, Hq, Hkv, r_k, r_v, seq_lens, reserve=2, shared_key_basis=False):
         self.B, self.Hq, self.Hkv, self.r_k, self.r_v = B, Hq, Hkv, r_k, r_v
@@ -44,7 +56,7 @@ class QCase:
         P = self.pg.num_pages
         fill = lambda shape, v, dt: torch.full(shape, v, dtype=dt, device=DEV)
         self.layer = S.QLayer(Hq, Hkv, r_k, r_v, self.U_k.to(DEV), self.U_v.to(DEV), torch.from_numpy(self.k_params).to(DEV),
-                              fill((P, Hkv, 64, r_k), 0xAB, torch.uint8), fill((P, Hkv, 64, r_v), 0xCD, torch.uint8),
+                              fill((P, Hkv, 64, r_k), 0xAB, torch.uint8), fill((P, Hkv, r_v, 64), 0xCD, torch.uint8),
                               fill((P, Hkv, 64, r_v // 64, 2), float("nan"), torch.float32))
         bt = np.where(self.pg.block_table < 0, 0, self.pg.block_table).astype(np.int32)
         self.batch = S.Batch(torch.from_numpy(bt).to(DEV), torch.from_numpy(self.seq_lens.copy()).to(DEV))
@@ -60,11 +72,18 @@ class QCase:
         return Kd, Vd, Kc, ks, kz, Vc, vs, vz
 
     def gather(self, t, b, n):
-        """[n, Hkv, ...] rows of sequence b gathered from a device pool through the block table."""
+        """[n, Hkv, ...] rows of sequence b gathered from a token-major device pool through the block table."""
         p = t.cpu()
         idx = torch.arange(n)
         pages = torch.from_numpy(self.pg.block_table[b].astype(np.int64))[idx // 64]
         return p[pages, :, idx % 64]
+
+    def gather_v(self, b, n):
+        """[n, Hkv, r_v] value codes of sequence b: pages are [Hkv][r_v channels][64 positions]."""
+        p = self.layer.v_codes.cpu()
+        idx = torch.arange(n)
+        pages = torch.from_numpy(self.pg.block_table[b].astype(np.int64))[idx // 64]
+        return p[pages, :, :, torch.from_numpy(vpos(idx.numpy() % 64))]
 
 
 def _check_cache(c: QCase):
@@ -74,7 +93,7 @@ def _check_cache(c: QCase):
         if n == 0:
             continue
         gk = c.gather(c.layer.k_codes, b, n).numpy().astype(np.int32)
-        gv = c.gather(c.layer.v_codes, b, n).numpy().astype(np.int32)
+        gv = c.gather_v(b, n).numpy().astype(np.int32)
         gp = c.gather(c.layer.v_params, b, n).numpy()
         for h in range(c.Hkv):
             Kd, Vd, Kc, ks, kz, Vc, vs, vz = c.oracle_cache(b, h)
@@ -98,8 +117,14 @@ def _untouched(c: QCase):
         for t in range(int(c.seq_lens[b])):
             used[c.pg.block_table[b, t // 64], t % 64] = True
     m = ~used[:, None, :].repeat(c.Hkv, 1)
-    assert np.all(c.layer.k_codes.cpu().numpy()[m] == 0xAB) and np.all(c.layer.v_codes.cpu().numpy()[m] == 0xCD)
+    assert np.all(c.layer.k_codes.cpu().numpy()[m] == 0xAB)
     assert np.all(np.isnan(c.layer.v_params.cpu().numpy()[m]))
+    used_pos = np.zeros_like(used)
+    for pgi in range(used.shape[0]):
+        used_pos[pgi, vpos(np.nonzero(used[pgi])[0])] = True
+    vc = c.layer.v_codes.cpu().numpy()                                      # [P, Hkv, r_v, 64]
+    mv = ~used_pos[:, None, None, :].repeat(c.Hkv, 1).repeat(c.r_v, 2)
+    assert np.all(vc[mv] == 0xCD)
 
 
 def _oracle_out(c: QCase, q, caches):
@@ -130,7 +155,7 @@ def _upload(c: QCase, caches):
             for t in range(Kc.shape[0]):
                 pgi = int(c.pg.block_table[b, t // 64])
                 kc[pgi, h, t % 64] = torch.from_numpy(Kc[t].astype(np.uint8))
-                vc[pgi, h, t % 64] = torch.from_numpy(Vc[t].astype(np.uint8))
+                vc[pgi, h, :, int(vpos(t % 64))] = torch.from_numpy(Vc[t].astype(np.uint8))
                 vp[pgi, h, t % 64, :, 0] = torch.from_numpy(vs[t])
                 vp[pgi, h, t % 64, :, 1] = torch.from_numpy(vz[t])
     c.layer.k_codes.copy_(kc); c.layer.v_codes.copy_(vc); c.layer.v_params.copy_(vp)
@@ -182,7 +207,7 @@ def test_q8_prefill_append_decode_end_to_end():
     for b in range(B):
         n = int(c.seq_lens[b]) + 1
         gk = c.gather(c.layer.k_codes, b, n).numpy().astype(np.int32)
-        gv = c.gather(c.layer.v_codes, b, n).numpy().astype(np.int32)
+        gv = c.gather_v(b, n).numpy().astype(np.int32)
         gp = c.gather(c.layer.v_params, b, n).numpy()
         for h in range(Hkv):
             _, _, Kc, ks, kz, Vc, vs, vz = caches[b][h]
