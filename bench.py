@@ -393,9 +393,11 @@ def run_q8(args):
     qs = [I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for i in range(n_in)]
     kvs = [I.new_token_kv(SEED, 0, B, Hkv, device=dev, step=i) for i in range(n_in)]
 
+    overlap = S.STIEF_DECODE_OVERLAP_PREVIOUS if (args.overlap and n_caches >= 2) else 0
+
     def step(i):
-        S.stief_q8_append(layers[i % n_caches], batch, kvs[i % n_in][0], kvs[i % n_in][1], status=status)
-        S.stief_q8_decode_attention(layers[i % n_caches], batch, qs[i % n_in], ws, out, 0, len_add=1, status=status)
+        S.stief_q8_decode_step(layers[i % n_caches], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
+                               status=status, flags=overlap)
 
     K_steps, W = min(args.steps, 2000), max(args.warmup, 3)
     for i in range(W):
@@ -417,9 +419,10 @@ def run_q8(args):
         "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
         "dtype_note": "8-bit codes expanded to bf16 tensor-core operands, fp32 accumulate", "data": "synthetic",
         "config": {"workload": cfg["name"] + f" on the 8-bit quantised cache ({per_unit} bytes per token and KV head instead of {2 * (r_k + r_v)}); "
-                               "step = append launch + attention launch", "l2": f"steps rotate over {n_caches} layer caches"},
+                               "step = append + query projection + split-T attention + combine, one launch"
+                               + (", overlapped launches" if overlap else ""), "l2": f"steps rotate over {n_caches} layer caches"},
         "tokens_per_s": B * K_steps / (ms * 1e-3), "frac_of_hbm_peak": gbs / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
-        "bytes_per_step": sb, "gpu_launches": 2 * K_steps,
+        "bytes_per_step": sb, "gpu_launches": K_steps,
         "same_step_in_bf16_cache_bytes_gbs": B * Hkv * (T + 1) * 2 * (r_k + r_v) * K_steps / (ms * 1e-3) / 1e9,
         "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak}}))
 

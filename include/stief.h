@@ -251,6 +251,13 @@ int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batc
                               int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
                               uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
 
+/* One decode step of one layer on the quantised cache in one launch: project, quantise and store (k_new, v_new)
+ * at position seq_lens[b], then attend over seq_lens[b] + 1 tokens.  Same result as stief_q8_append followed by
+ * stief_q8_decode_attention with len_add = 1. */
+int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+                         const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts,
+                         uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+
 /* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
  * stief_decode_step_host call made by this host thread records `start_event` just before and
  * `stop_event` just after its decode kernel on the call's stream (both cudaEvent_t passed as void*),

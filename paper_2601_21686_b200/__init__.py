@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
             "stief_q8_prefill_compress": (ctypes.c_int, [QP, BP, P, P, I64, I64, I32, U32, P, P]),
             "stief_q8_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
             "stief_q8_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
+            "stief_q8_decode_step": (ctypes.c_int, [QP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -209,6 +210,15 @@ def stief_q8_decode_attention(layer: QLayer, batch: Batch, q: torch.Tensor, work
     _check(lib().stief_q8_decode_attention(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
                                            flags, _ptr(status), _stream()), "stief_q8_decode_attention")
+
+
+def stief_q8_decode_step(layer: QLayer, batch: Batch, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                         workspace: torch.Tensor, out: torch.Tensor, num_parts: int = 0, out_lse: Optional[torch.Tensor] = None,
+                         status: Optional[torch.Tensor] = None, flags: int = 0):
+    cl, cb = layer.c(), batch.c()
+    _check(lib().stief_q8_decode_step(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
+                                      flags, _ptr(status), _stream()), "stief_q8_decode_step")
 
 
 def stief_append(layer: Layer, batch: Batch, k_new: torch.Tensor, v_new: torch.Tensor, status: Optional[torch.Tensor] = None):

@@ -30,11 +30,13 @@ namespace stief {
 struct DecodeQ8Args {
   LayerDev L;                    // bases and shape (the bf16 pool pointers are unused)
   BatchDev Bt;
-  const uint8_t* k_codes;        // [pages][Hkv][64][RK]
-  const uint8_t* v_codes;        // [pages][Hkv][64][RV]
-  const float* v_params;         // [pages][Hkv][64][RV/64][2] (scale, zero)
+  uint8_t* k_codes;              // [pages][Hkv][64][RK]
+  uint8_t* v_codes;              // [pages][Hkv][RV][64 positions]
+  float* v_params;               // [pages][Hkv][64][RV/64][2] (scale, zero)
   const float* k_params;         // [Hkv][RK/64][2] (scale, zero)
   const __nv_bfloat16* q;        // [B][Hq][128]
+  const __nv_bfloat16* k_new;    // [B][Hkv][128] or NULL: project, quantise and store at position seq_lens[b] first
+  const __nv_bfloat16* v_new;
   float* partial_o;
   float* partial_lse;
   int* counters;
@@ -137,6 +139,7 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   volatile int* last_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);
   float* lse_shift = reinterpret_cast<float*>(ctrl_ptr + 34 * 8);      // [8]: q' . key zero-point / sqrt(128) of the unit's rows
   float* q_delta = reinterpret_cast<float*>(ctrl_ptr + 38 * 8);        // [8]: fixed-point step of the unit's scaled query rows
+  volatile int* append_done = reinterpret_cast<volatile int*>(ctrl_ptr + 32 * 8);   // appending segments whose rows are stored
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -150,6 +153,7 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     *abort_flag = 0;
     *last_flag = 0;
+    *append_done = 0;
     mbar_fence_init();
   }
   const int pad = seg_pad_pages(RK, RV);
@@ -159,6 +163,8 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int upb = Hkv * QT;
   const int total = pref[B] * upb;
   const int P = pages_per_cta(total, n_cta);
+
+  const bool appending = a.k_new != nullptr;
 
   SegmentWalker walk;
   walk.init(pref, B, upb, pad, c, P, total);
@@ -175,9 +181,15 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       tma_prefetch_desc(&tmV);
     }
     int i_base = 0;            // pages of this CTA before the current segment
+    int n_append = 0;          // appending segments of this CTA so far
     while (walk.next(seg)) {
       const int h = seg.j / QT;
       const int npg = seg.p1 - seg.p0;
+      bool wait_append = false;
+      if (appending && seg.p1 == seg.npages) {
+        const int pos = a.Bt.seq_lens[seg.b];
+        wait_append = pos >= 0 && pos / kPage < a.Bt.max_pages;
+      }
       int tbl = 0, win = -1;
       for (int k = (pw - i_base % NP + NP) % NP; k < npg; k += NP) {
         if ((k >> 5) != win) {                             // block-table entries of a window of 32 pages, one per lane
@@ -195,6 +207,12 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int use = kw / SPW;
         if (lane == 0) {
           if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
+          if (wait_append && k == npg - 1) {
+            // the sequence's last page receives the new token's codes from this CTA's consumers first
+            wait_count(append_done, n_append + 1, abort_flag, a.status);
+            __threadfence();
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+          }
           const uint32_t st = ring + slot * C::STAGE_BYTES;
           const size_t tile = (size_t)page * Hkv + h;
           mbar_arrive_expect_tx(full_bar(slot), C::TX_BYTES);
@@ -205,6 +223,7 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         __syncwarp();
       }
       i_base += npg;
+      if (wait_append) ++n_append;
     }
     return;
   }
@@ -231,28 +250,50 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int len_raw = a.Bt.seq_lens[b] + a.len_add;
     const int len = min(max(len_raw, 0), seg.npages * kPage);
     const int last_valid = len - (seg.npages - 1) * kPage;          // tokens in the sequence's last page (1..64)
+    const bool has_final = seg.p1 == seg.npages;
+    bool do_append = false;
+    int new_page = -1, new_pos = 0;
+    if (appending && has_final) {
+      const int pos = a.Bt.seq_lens[b];
+      if (pos >= 0 && pos / kPage < a.Bt.max_pages) {
+        do_append = true;                                            // the producer waits for our signal
+        new_pos = pos % kPage;
+        new_page = a.Bt.block_table[(size_t)b * a.Bt.max_pages + pos / kPage];
+        if (new_page < 0 || new_page >= a.L.num_pages) new_page = -1;     // bad page: signal, but store nothing
+      }
+    }
     // ---- prologue: q' = q U_k for the unit's queries.  The key scale of each 64-channel group is folded into
     // q' (scores are then taken against the raw codes); the key zero-point shifts all scores of a row by
     // q' . zero, which cancels in the softmax and across segments and is added to out_lse at the very end.
-    float* rows = un;                    // [9][128] fp32 (row 8 unused here)
+    float* rows = un;                    // [9][128] fp32: the queries, row 8 = the new key
+    float* vrow = un + 9 * kD;           // [128]: the new value, later its projection
     float* red = un + 10 * kD;           // [NW][9][128]
     const __nv_bfloat16* Uk = a.L.U_k + (size_t)h * a.L.uk_stride;
-    const uint32_t row_mask = (1u << ng) - 1u;
+    const __nv_bfloat16* Uv = a.L.U_v + (size_t)h * a.L.uv_stride;
+    const uint32_t row_mask = ((1u << ng) - 1u) | (do_append ? 0x100u : 0u);
     {
       BasisSlice<NW, RK> sk;
       sk.load(Uk, warp, lane);
-      constexpr int NPC = (8 * 16 + NT - 1) / NT;
+      constexpr int NPC = (9 * 16 + NT - 1) / NT;
       uint4 pc[NPC];
 #pragma unroll
       for (int i = 0; i < NPC; ++i) {
         const int idx = tid + i * NT, r = idx / 16, c = idx % 16;
         pc[i] = make_uint4(0u, 0u, 0u, 0u);
         if (r < ng) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (head0 + r) * kD) + c);
+        else if (r == 8 && do_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * kD) + c);
+      }
+      uint4 pv = make_uint4(0u, 0u, 0u, 0u);
+      if (do_append && tid < 16) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * kD) + tid);
+      if (do_append && tid < 16) {
+        const uint32_t w[4] = {pv.x, pv.y, pv.z, pv.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(vrow + tid * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
       }
 #pragma unroll
       for (int i = 0; i < NPC; ++i) {
         const int idx = tid + i * NT;
-        if (idx < 8 * 16) {
+        if (idx < 9 * 16) {
           const uint32_t w[4] = {pc[i].x, pc[i].y, pc[i].z, pc[i].w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(rows + idx * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
@@ -261,12 +302,20 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       bar1(NT);
       sk.contract(rows, row_mask, red, warp, lane);
     }
+    BasisSlice<NW, RV> sv;
+    if (do_append) sv.load(Uv, warp, lane);                // in flight while the key side is reduced
     bar1(NT);
     const float* kpar = a.k_params + (size_t)h * (RK / 64) * 2;
-    for (int idx = tid; idx < 8 * RK; idx += NT) {
+    for (int idx = tid; idx < 9 * RK; idx += NT) {
       const int r = idx / RK, j = idx % RK;
       const float x = ((row_mask >> r) & 1u) ? warp_shares<NW>(red, r, j) : 0.f;
-      qp[r * RK + j] = x * qscale * __ldg(kpar + 2 * (j >> 6));
+      if (r < 8) {
+        qp[r * RK + j] = x * qscale * __ldg(kpar + 2 * (j >> 6));
+      } else if (do_append && new_page >= 0) {             // the new key's code under the head's static parameters
+        const float sc = __ldg(kpar + 2 * (j >> 6)), zp = __ldg(kpar + 2 * (j >> 6) + 1);
+        const float y = __fmul_rn(__fsub_rn(x, zp), __fdiv_rn(1.f, sc));
+        a.k_codes[(((size_t)new_page * Hkv + h) * kPage + new_pos) * RK + j] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+      }
     }
     if (tid < 8) {
       float sh = 0.f;
@@ -281,6 +330,34 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       q_delta[tid] = mx > 0.f ? mx / kFixedMax : 1.f;
     }
     bar1(NT);
+    if (do_append) {
+      // the new value row: project (the row sits where row 0 is expected), then token-wise group parameters and codes
+      sv.contract(vrow, 1u, red, warp, lane);
+      bar1(NT);
+      for (int j = tid; j < RV; j += NT) vrow[j] = warp_shares<NW>(red, 0, j);
+      bar1(NT);
+      if (new_page >= 0) {
+        for (int j = tid; j < RV; j += NT) {
+          const int g = j >> 6;
+          float mn = vrow[64 * g], mxv = mn;
+          for (int e = 1; e < 64; ++e) {
+            mn = fminf(mn, vrow[64 * g + e]);
+            mxv = fmaxf(mxv, vrow[64 * g + e]);
+          }
+          const float sc = mxv > mn ? __fdiv_rn(mxv - mn, 255.f) : 1.f;
+          const float y = __fmul_rn(__fsub_rn(vrow[j], mn), __fdiv_rn(1.f, sc));
+          const size_t tile = (size_t)new_page * Hkv + h;
+          a.v_codes[(tile * RV + j) * kPage + v_position(new_pos)] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+          if ((j & 63) == 0) *reinterpret_cast<float2*>(a.v_params + ((tile * kPage + new_pos) * NGV + g) * 2) = make_float2(sc, mn);
+        }
+      } else if (tid == 0) {
+        report(a.status, STIEF_ERR_BOUNDS);
+      }
+      __threadfence();
+      asm volatile("fence.proxy.async.global;" ::: "memory");
+      bar1(NT);
+      if (tid == 0) *append_done = *append_done + 1;       // codes are in the pools: the last page may be fetched
+    }
 
     // A operand of the score MMA: rows 0-7 = high digits of the scaled query rows, rows 8-15 = low digits
     const float dq = q_delta[gid];

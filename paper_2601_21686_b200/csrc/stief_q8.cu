@@ -205,10 +205,11 @@ int stief_q8_append(const stief_qlayer* layer, const stief_batch* batch, const u
   return cudaGetLastError() == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
-int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, int32_t len_add,
-                              void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
-                              uint32_t flags, int32_t* status, void* stream) {
+static int run_q8_decode(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+                         const uint16_t* v_new, int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
+                         uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream) {
   if (flags & ~STIEF_DECODE_OVERLAP_PREVIOUS) return STIEF_ERR_INVALID_ARG;
+  if (k_new && (!v_new || !host::aligned(k_new, 16) || !host::aligned(v_new, 16) || len_add != 1)) return STIEF_ERR_INVALID_ARG;
   int rc = check_qlayer(layer);
   if (rc) return rc;
   rc = host::check_batch(batch);
@@ -227,6 +228,8 @@ int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batc
   a.Bt = host::to_dev(batch);
   a.k_codes = layer->k_codes; a.v_codes = layer->v_codes; a.v_params = layer->v_params; a.k_params = layer->k_params;
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
+  a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
   a.partial_o = w.partial_o; a.partial_lse = w.partial_lse; a.counters = w.counters;
   a.out = reinterpret_cast<__nv_bfloat16*>(out);
   a.out_lse = out_lse;
@@ -241,6 +244,20 @@ int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batc
   else if (layer->r_v == 64) e = launch_decode_q8<128, 64>(a, n_cta, ov, st);
   else e = launch_decode_q8<128, 128>(a, n_cta, ov, st);
   return e == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
+int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, int32_t len_add,
+                              void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out, float* out_lse,
+                              uint32_t flags, int32_t* status, void* stream) {
+  return run_q8_decode(layer, batch, q, nullptr, nullptr, len_add, workspace, workspace_bytes, num_parts, out, out_lse, flags, status,
+                       stream);
+}
+
+int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+                         const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts, uint16_t* out,
+                         float* out_lse, uint32_t flags, int32_t* status, void* stream) {
+  if (!k_new || !v_new) return STIEF_ERR_INVALID_ARG;
+  return run_q8_decode(layer, batch, q, k_new, v_new, 1, workspace, workspace_bytes, num_parts, out, out_lse, flags, status, stream);
 }
 
 }  // extern "C"

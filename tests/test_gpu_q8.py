@@ -218,6 +218,43 @@ def test_q8_prefill_append_decode_end_to_end():
     assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 5e-3
 
 
+@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 128)])
+def test_q8_fused_step_equals_append_then_attention_also_with_overlapped_launches(r_k, r_v):
+    B, Hq, Hkv = 2, 8, 2
+    cs = [QCase(600 + l, B, Hq, Hkv, r_k, r_v, [450, 127], reserve=4) for l in range(2)]
+    for c in cs:
+        S.stief_q8_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    torch.cuda.synchronize()
+    snap = [(c.layer.k_codes.clone(), c.layer.v_codes.clone(), c.layer.v_params.clone()) for c in cs]
+    ws = _workspace(cs[0], 0)
+    kvs = [tuple(t.cuda() for t in I.new_token_kv(600, l, B, Hkv)) for l in range(2)]
+    res = {}
+    for mode in ("separate", "fused", "fused_overlapped"):
+        for c, (kc, vc, vp) in zip(cs, snap):
+            c.layer.k_codes.copy_(kc); c.layer.v_codes.copy_(vc); c.layer.v_params.copy_(vp)
+        outs = [torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV) for _ in range(4)]
+        for i in range(4):                               # layers alternate, so consecutive kernels touch different pools
+            c, (kn, vn) = cs[i % 2], kvs[i % 2]
+            if mode == "separate":
+                S.stief_q8_append(c.layer, c.batch, kn, vn, status=c.status)
+                S.stief_q8_decode_attention(c.layer, c.batch, c.q.cuda(), ws, outs[i], 0, len_add=1, status=c.status)
+            else:
+                S.stief_q8_decode_step(c.layer, c.batch, c.q.cuda(), kn, vn, ws, outs[i], status=c.status,
+                                       flags=S.STIEF_DECODE_OVERLAP_PREVIOUS if (mode == "fused_overlapped" and i) else 0)
+        torch.cuda.synchronize()
+        assert all(int(c.status.item()) == 0 for c in cs)
+        res[mode] = ([o.clone() for o in outs], [(c.layer.k_codes.clone(), c.layer.v_codes.clone(), c.layer.v_params.clone()) for c in cs])
+    for mode in ("fused", "fused_overlapped"):
+        for a, b in zip(res["separate"][0], res[mode][0]):
+            U.check_out(a, b.double().cpu().numpy(), max_abs=4e-3, rel_l2=2e-3)     # projection order differs in the last bits
+        for (k0, v0, p0), (k1, v1, p1) in zip(res["separate"][1], res[mode][1]):
+            assert (k0.int() - k1.int()).abs().max() <= 1 and (v0.int() - v1.int()).abs().max() <= 1
+            m = ~torch.isnan(p0)
+            assert torch.equal(torch.isnan(p0), torch.isnan(p1)) and torch.allclose(p0[m], p1[m], rtol=2e-4, atol=2e-5)
+    for a, b in zip(res["fused"][0], res["fused_overlapped"][0]):
+        assert torch.equal(a, b)
+
+
 def test_q8_rejects_unsupported_ranks_on_the_host():
     c = QCase(500, 1, 4, 1, 64, 64, [100])
     bad = S.QLayer(4, 1, 48, 64, c.layer.U_k, c.layer.U_v, c.layer.k_params, c.layer.k_codes, c.layer.v_codes, c.layer.v_params)
