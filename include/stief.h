@@ -56,8 +56,13 @@ enum stief_status {
  * U_k: [Hkv][128][r_k] bf16 row-major (r fastest) with head stride uk_head_stride elements; stride 0
  * means one key basis shared by all heads of the layer (the paper's head-sharing scheme, Sec. 3.3).
  * U_v: [Hkv][128][r_v], per-head value bases (stride 128*r_v) or shared (stride 0).
- * A NULL basis keeps that side full rank (Algorithm 2 lets a layer keep keys or values
- * uncompressed): the rank must then be 128 and rows are stored / used unprojected.
+ * A NULL basis means the library does not project that side: its rows arrive with r elements and are
+ * stored and used as they are.  With r = 128 that is a layer that keeps keys or values full rank
+ * (Algorithm 2); with r < 128 the projection has been folded into the model's linear layers (Sec. 3.3,
+ * "Overheads": W_K U_k and W_Q U_k produce compressed keys and queries, W_V U_v compressed values, and
+ * U_v^T W_O consumes the compressed attention output).  For a key side without basis q, k_new and K have
+ * r_k elements per head; for a value side without basis v_new and V have r_v elements per head and the
+ * outputs `out` are [B][Hq][r_v]: no back-projection is applied.
  * The same U buffers serve compression, query projection and back-projection.
  * Alignment: pools and bases 128 bytes. */
 typedef struct stief_layer {
@@ -81,9 +86,9 @@ typedef struct stief_batch {
 } stief_batch;
 
 /* Eq. 1 for a whole prompt: for every b, t < seq_lens[b], h: K_down[t,h,:] = rnd_bf16(K[b,t,h,:] U_k[h])
- * and the same for V, accumulated in fp32, stored to the paged pools.  K, V are bf16 with element
- * strides stride_b (between sequences) and stride_t (between tokens); heads are contiguous blocks of
- * 128 elements; rows must be 16-byte aligned.  T_max bounds seq_lens (it sizes the launch; tokens
+ * and the same for V, accumulated in fp32, stored to the paged pools.  K and V are bf16 with element
+ * strides stride_b / v_stride_b (between sequences) and stride_t / v_stride_t (between tokens); heads are
+ * contiguous blocks of 128 elements (r elements on a side without basis); rows must be 16-byte aligned.  T_max bounds seq_lens (it sizes the launch; tokens
  * beyond seq_lens[b] are never stored; the input rows of a sequence's last 128-token tile are read up
  * to T_max).
  * flags: 0, or STIEF_PREFILL_OVERLAP_PREVIOUS: the kernel may start (and write its pools) before the kernel
@@ -93,8 +98,8 @@ typedef struct stief_batch {
  * different layers satisfy that.  The kernel still completes only after its predecessor has. */
 #define STIEF_PREFILL_OVERLAP_PREVIOUS 1u
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K,
-                           const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
-                           uint32_t flags, int32_t* status, void* stream);
+                           const uint16_t* V, int64_t stride_b, int64_t stride_t, int64_t v_stride_b,
+                           int64_t v_stride_t, int32_t T_max, uint32_t flags, int32_t* status, void* stream);
 
 /* Eq. 1 for one new token per sequence: projects k_new, v_new [B][Hkv][128] and stores the rows at
  * position seq_lens[b] (the page block_table[b][seq_lens[b]/64] must already be assigned).  The

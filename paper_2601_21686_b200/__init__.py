@@ -67,7 +67,7 @@ def lib() -> ctypes.CDLL:
         P, I32, I64, SZ, U32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32
         LP, BP, QP = ctypes.POINTER(_CLayer), ctypes.POINTER(_CBatch), ctypes.POINTER(_CQLayer)
         sig = {
-            "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I32, U32, P, P]),
+            "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I64, I64, I32, U32, P, P]),
             "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
             "stief_decode_num_parts": (I32, []),
             "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
@@ -179,11 +179,14 @@ def stief_version() -> int:
 
 def stief_prefill_compress(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
                            status: Optional[torch.Tensor] = None, flags: int = 0):
-    """K, V [B, T, Hkv, 128] bf16 (strides over b and t free, heads and d contiguous) -> paged compressed cache."""
-    assert K.stride(3) == 1 and K.stride(2) == D_HEAD and V.stride() == K.stride()
+    """K, V [B, T, Hkv, 128] bf16 (strides over b and t free, heads and d contiguous) -> paged compressed cache.
+    A side without basis takes rows of r elements: [B, T, Hkv, r]."""
+    assert K.stride(3) == 1 and K.stride(2) == K.shape[3] and V.stride(3) == 1 and V.stride(2) == V.shape[3]
+    assert K.shape[3] == (D_HEAD if layer.U_k is not None else layer.r_k) and V.shape[3] == (D_HEAD if layer.U_v is not None else layer.r_v)
     cl, cb = layer.c(), batch.c()
     _check(lib().stief_prefill_compress(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
-                                        K.shape[1] if T_max is None else T_max, flags, _ptr(status), _stream()),
+                                        V.stride(0), V.stride(1), K.shape[1] if T_max is None else T_max, flags, _ptr(status),
+                                        _stream()),
            "stief_prefill_compress")
 
 

@@ -41,7 +41,6 @@ int check_layer(const stief_layer* l) {
   if (!rank_ok(l->r_k) || !rank_ok(l->r_v)) return STIEF_ERR_UNSUPPORTED;
   if (!l->k_pool || !l->v_pool || !aligned(l->k_pool, 128) || !aligned(l->v_pool, 128)) return STIEF_ERR_INVALID_ARG;
   if ((l->U_k && !aligned(l->U_k, 128)) || (l->U_v && !aligned(l->U_v, 128))) return STIEF_ERR_INVALID_ARG;
-  if ((!l->U_k && l->r_k != kD) || (!l->U_v && l->r_v != kD)) return STIEF_ERR_INVALID_ARG;
   if (l->uk_head_stride < 0 || l->uv_head_stride < 0) return STIEF_ERR_INVALID_ARG;
   if ((l->uk_head_stride % 64) != 0 || (l->uv_head_stride % 64) != 0) return STIEF_ERR_INVALID_ARG;   // keeps every head's basis 128-byte aligned
   if ((long long)l->num_pages * l->Hkv * kPage >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
@@ -205,20 +204,24 @@ using namespace stief;
 extern "C" {
 
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K, const uint16_t* V,
-                           int64_t stride_b, int64_t stride_t, int32_t T_max, uint32_t flags, int32_t* status, void* stream) {
+                           int64_t stride_b, int64_t stride_t, int64_t v_stride_b, int64_t v_stride_t, int32_t T_max,
+                           uint32_t flags, int32_t* status, void* stream) {
   if (flags & ~STIEF_PREFILL_OVERLAP_PREVIOUS) return STIEF_ERR_INVALID_ARG;
   int rc = check_layer(layer);
   if (rc) return rc;
   rc = check_batch(batch);
   if (rc) return rc;
   if (!K || !V || !aligned(K, 16) || !aligned(V, 16)) return STIEF_ERR_INVALID_ARG;
-  if (T_max <= 0 || stride_t < (int64_t)layer->Hkv * kD || stride_b < 0 || (stride_t % 8) != 0 || (stride_b % 8) != 0)
+  const int64_t dk = layer->U_k ? kD : layer->r_k, dv = layer->U_v ? kD : layer->r_v;      // elements per input row of each side
+  if (T_max <= 0 || stride_t < layer->Hkv * dk || stride_b < 0 || (stride_t % 8) != 0 || (stride_b % 8) != 0)
     return STIEF_ERR_INVALID_ARG;
-  if (batch->B > 1 && stride_b == 0) return STIEF_ERR_INVALID_ARG;
+  if (v_stride_t < layer->Hkv * dv || v_stride_b < 0 || (v_stride_t % 8) != 0 || (v_stride_b % 8) != 0) return STIEF_ERR_INVALID_ARG;
+  if (batch->B > 1 && (stride_b == 0 || v_stride_b == 0)) return STIEF_ERR_INVALID_ARG;
   PrefillArgs a;
   a.L = to_dev(layer); a.Bt = host::to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K); a.V = reinterpret_cast<const __nv_bfloat16*>(V);
-  a.stride_b = stride_b; a.stride_t = stride_t; a.T_max = T_max; a.status = status;
+  a.stride_b = stride_b; a.stride_t = stride_t; a.v_stride_b = v_stride_b; a.v_stride_t = v_stride_t;
+  a.T_max = T_max; a.status = status;
   a.overlap_previous = (flags & STIEF_PREFILL_OVERLAP_PREVIOUS) != 0;
   return launch_prefill(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }

@@ -291,6 +291,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     const __nv_bfloat16* Uk = a.L.U_k ? a.L.U_k + (size_t)h * a.L.uk_stride : nullptr;
     const __nv_bfloat16* Uv = a.L.U_v ? a.L.U_v + (size_t)h * a.L.uv_stride : nullptr;
     const uint32_t row_mask = ((1u << ng) - 1u) | (do_append ? 0x100u : 0u);
+    // a side without a basis is handled in its own dimension: its q / k (or v) rows arrive with r elements
+    const int dk = Uk ? kD : RK, dv = Uv ? kD : RV;
     {
       BasisSlice<NW, RK> sk;
       if (Uk) sk.load(Uk, warp, lane);
@@ -301,11 +303,13 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       for (int i = 0; i < NPC; ++i) {
         const int idx = tid + i * NT, r = idx / 16, c = idx % 16;
         pc[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (r < ng) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (head0 + r) * kD) + c);
-        else if (r == 8 && do_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * kD) + c);
+        if (8 * c < dk) {
+          if (r < ng) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (head0 + r) * dk) + c);
+          else if (r == 8 && do_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * dk) + c);
+        }
       }
       uint4 pv = make_uint4(0u, 0u, 0u, 0u);
-      if (do_append && tid < 16) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * kD) + tid);
+      if (do_append && tid < 16 && 8 * tid < dv) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * dv) + tid);
 #pragma unroll
       for (int i = 0; i < NPC; ++i) {
         const int idx = tid + i * NT;
@@ -536,7 +540,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       const int h = j / QT, qt = j % QT;
       const int ng = min(kGroupTile, G - qt * kGroupTile);
       const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
-      for (int idx = tid; idx < ng * kD; idx += NT) a.out[head0 * kD + idx] = __float2bfloat16_rn(0.f);
+      const int d_out = a.L.U_v ? kD : RV;
+      for (int idx = tid; idx < ng * d_out; idx += NT) a.out[head0 * d_out + idx] = __float2bfloat16_rn(0.f);
       if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
     }
   }

@@ -28,7 +28,8 @@ struct PrefillArgs {
   BatchDev Bt;
   const __nv_bfloat16* K;
   const __nv_bfloat16* V;
-  long long stride_b, stride_t;
+  long long stride_b, stride_t;       // element strides of K between sequences / tokens
+  long long v_stride_b, v_stride_t;   // the same for V
   int T_max;
   int32_t* status;
   bool overlap_previous;        // launch with programmatic stream serialization

@@ -264,7 +264,8 @@ __device__ __forceinline__ void combine_unit(const LayerDev& L, int b, int h, in
   if (tid < ng && out_lse)
     out_lse[head0 + tid] = Drow[tid] > 0.f ? Mrow[tid] + __logf(Drow[tid]) + (lse_shift ? lse_shift[tid] : 0.f) : -INFINITY;
   bar1(nt);
-  for (int dd = tid; dd < kD; dd += nt) {
+  const int d_out = Uv ? kD : RV;                           // without a value basis the output stays in the compressed space
+  for (int dd = tid; dd < d_out; dd += nt) {
     float acc[kGroupTile];
 #pragma unroll
     for (int r = 0; r < kGroupTile; ++r) acc[r] = 0.f;
@@ -292,7 +293,7 @@ __device__ __forceinline__ void combine_unit(const LayerDev& L, int b, int h, in
     }
 #pragma unroll
     for (int r = 0; r < kGroupTile; ++r)
-      if (r < ng) out[(head0 + r) * kD + dd] = __float2bfloat16_rn(acc[r]);
+      if (r < ng) out[(head0 + r) * d_out + dd] = __float2bfloat16_rn(acc[r]);
   }
   bar1(nt);
 }

@@ -9,11 +9,13 @@ constexpr int kPfThreads = 128;
 constexpr int kPfTokens = 512;        // tokens per CTA
 
 // rows kept full rank (no basis): the cache stores the bf16 rows unchanged
-__device__ void prefill_copy(const __nv_bfloat16* X, __nv_bfloat16* pool, const PrefillArgs& a, int b, int h, int len) {
+__device__ void prefill_copy(const __nv_bfloat16* X, __nv_bfloat16* pool, const PrefillArgs& a, int b, int h, int len, int R,
+                             long long stride_b, long long stride_t) {
   const int t0 = blockIdx.x * kPfTokens;
-  const __nv_bfloat16* Xb = X + (size_t)b * a.stride_b + (size_t)h * kD;
-  for (int idx = threadIdx.x; idx < kPfTokens * 16; idx += kPfThreads) {
-    const int t = t0 + idx / 16, c = idx % 16;
+  const int cpr = R / 8;                                   // 16-byte pieces per row of R elements
+  const __nv_bfloat16* Xb = X + (size_t)b * stride_b + (size_t)h * R;
+  for (int idx = threadIdx.x; idx < kPfTokens * cpr; idx += kPfThreads) {
+    const int t = t0 + idx / cpr, c = idx % cpr;
     if (t >= len) break;
     const int pi = t / kPage;
     const int page = (pi < a.Bt.max_pages) ? a.Bt.block_table[(size_t)b * a.Bt.max_pages + pi] : -1;
@@ -22,7 +24,7 @@ __device__ void prefill_copy(const __nv_bfloat16* X, __nv_bfloat16* pool, const 
       continue;
     }
     const size_t row = ((size_t)page * a.L.Hkv + h) * kPage + (t % kPage);
-    reinterpret_cast<uint4*>(pool + row * kD)[c] = __ldg(reinterpret_cast<const uint4*>(Xb + (size_t)t * a.stride_t) + c);
+    reinterpret_cast<uint4*>(pool + row * R)[c] = __ldg(reinterpret_cast<const uint4*>(Xb + (size_t)t * stride_t) + c);
   }
 }
 
@@ -32,7 +34,8 @@ prefill_copy_kernel(const PrefillArgs a, const int side) {
   int len = a.Bt.seq_lens[b];
   if (len > a.T_max) len = a.T_max;
   if ((int)blockIdx.x * kPfTokens >= len) return;
-  prefill_copy(side ? a.V : a.K, side ? a.L.v_pool : a.L.k_pool, a, b, h, len);
+  if (side) prefill_copy(a.V, a.L.v_pool, a, b, h, len, a.L.r_v, a.v_stride_b, a.v_stride_t);
+  else prefill_copy(a.K, a.L.k_pool, a, b, h, len, a.L.r_k, a.stride_b, a.stride_t);
 }
 
 cudaError_t launch_prefill_copy(const PrefillArgs& a, int side, cudaStream_t st) {

@@ -586,11 +586,12 @@ int sm_count_of_current_device() {
 }
 
 // [B][T_max][Hkv][128] bf16 with element strides (stride_b, stride_t, 128, 1), boxes of 128 tokens x 64 elements
-bool make_input_map(CUtensorMap* tm, const void* X, const PrefillArgs& a) {
-  const unsigned long long sb = a.stride_b > 0 ? (unsigned long long)a.stride_b : (unsigned long long)a.stride_t * a.T_max;
+bool make_input_map(CUtensorMap* tm, const void* X, const PrefillArgs& a, bool value_side) {
+  const long long stride_b = value_side ? a.v_stride_b : a.stride_b, stride_t = value_side ? a.v_stride_t : a.stride_t;
+  const unsigned long long sb = stride_b > 0 ? (unsigned long long)stride_b : (unsigned long long)stride_t * a.T_max;
   const unsigned long long dims[4] = {(unsigned long long)kD, (unsigned long long)a.L.Hkv, (unsigned long long)a.T_max,
                                       (unsigned long long)a.Bt.B};
-  const unsigned long long strides[3] = {(unsigned long long)kD * 2, (unsigned long long)a.stride_t * 2, sb * 2};
+  const unsigned long long strides[3] = {(unsigned long long)kD * 2, (unsigned long long)stride_t * 2, sb * 2};
   const unsigned box[4] = {64, 1, (unsigned)kTileM, 1};
   return encode_bf16_map(tm, X, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
@@ -625,7 +626,8 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, const Args* q8, cudaStream_t
     configured[dev] = true;
   }
   CUtensorMap tmK, tmV;
-  if (!make_input_map(&tmK, proj_k ? a.K : a.V, a) || !make_input_map(&tmV, proj_v ? a.V : a.K, a)) return cudaErrorInvalidValue;
+  if (!make_input_map(&tmK, proj_k ? a.K : a.V, a, !proj_k) || !make_input_map(&tmV, proj_v ? a.V : a.K, a, proj_v))
+    return cudaErrorInvalidValue;
   CUtensorMap tmPK = tmK, tmPV = tmV;                     // the quantising kernel stores without TMA: placeholders
   if (!Q8 && (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a)))
     return cudaErrorInvalidValue;

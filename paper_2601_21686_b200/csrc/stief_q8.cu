@@ -179,7 +179,8 @@ int stief_q8_prefill_compress(const stief_qlayer* layer, const stief_batch* batc
   a.Bt = host::to_dev(batch);
   a.K = reinterpret_cast<const __nv_bfloat16*>(K);
   a.V = reinterpret_cast<const __nv_bfloat16*>(V);
-  a.stride_b = stride_b; a.stride_t = stride_t; a.T_max = T_max; a.status = status;
+  a.stride_b = stride_b; a.stride_t = stride_t; a.v_stride_b = stride_b; a.v_stride_t = stride_t;
+  a.T_max = T_max; a.status = status;
   a.overlap_previous = (flags & STIEF_PREFILL_OVERLAP_PREVIOUS) != 0;
   return launch_prefill_q8(a, layer->k_codes, layer->v_codes, layer->v_params, layer->k_params, static_cast<cudaStream_t>(stream)) ==
                  cudaSuccess

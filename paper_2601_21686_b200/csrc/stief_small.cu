@@ -57,12 +57,13 @@ append_kernel(const AppendArgs a) {
     return;
   }
   const size_t row = ((size_t)page * a.L.Hkv + h) * kPage + (pos % kPage);
-  const __nv_bfloat16* src = (which ? a.v_new : a.k_new) + ((size_t)b * a.L.Hkv + h) * kD;
   const __nv_bfloat16* Ub = which ? a.L.U_v : a.L.U_k;
   const __nv_bfloat16* U = Ub ? Ub + (size_t)h * (which ? a.L.uv_stride : a.L.uk_stride) : nullptr;
   const int R = which ? a.L.r_v : a.L.r_k;
+  const int d_in = U ? kD : R;                             // a side without a basis arrives in its own dimension
+  const __nv_bfloat16* src = (which ? a.v_new : a.k_new) + ((size_t)b * a.L.Hkv + h) * d_in;
   __nv_bfloat16* dst = (which ? a.L.v_pool : a.L.k_pool) + row * R;
-  if (threadIdx.x < kD) x[threadIdx.x] = __bfloat162float(src[threadIdx.x]);
+  if (threadIdx.x < d_in) x[threadIdx.x] = __bfloat162float(src[threadIdx.x]);
   __syncthreads();
   const float* res = x;                                    // no basis: the row is stored as it is
   if (U) {

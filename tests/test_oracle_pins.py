@@ -339,6 +339,22 @@ def test_paper_sizing_example_and_cache_ratio():
 
 # ---------------------------------------------------------------- planted mistakes must be caught
 
+def test_folding_the_projections_into_the_linear_layers_changes_nothing():
+    # Sec. 3.3 "Overheads": with q' = q P_K handed over by a folded W_Q and the output left in the compressed space for a
+    # folded P_V^T W_O, the attention is the same function: out = out_down P_V^T, lse unchanged
+    n, r_k, r_v = 90, 48, 96
+    Uk = I.stiefel_basis_f64(21, I.TAG_UK, 0, 0, r_k)
+    Uv = I.stiefel_basis_f64(21, I.TAG_UV, 0, 0, r_v)
+    K = I.normal_f64(I.stream_key(21, I.TAG_K), n * 128).numpy().reshape(n, 128)
+    V = I.normal_f64(I.stream_key(21, I.TAG_V), n * 128).numpy().reshape(n, 128)
+    q = I.normal_f64(I.stream_key(21, I.TAG_Q), 128).numpy()
+    Kd, Vd = O.compress(K, Uk, storage=False), O.compress(V, Uv, storage=False)
+    out, lse = O.attend_path_b(q, Kd, Vd, Uk, Uv)
+    out_down, lse_f = O.attend_path_b(q @ Uk, Kd, Vd, None, None)
+    assert out_down.shape == (r_v,) and abs(lse - lse_f) < 1e-12
+    assert np.abs(out_down @ Uv.T - out).max() < 1e-12
+
+
 def test_planted_mistakes_fail_the_pins():
     """Sanity of the pins themselves: a wrong softmax scale or a wrong query-head -> KV-head map is
     detected by the reconstructed-KV library check (the mistakes are planted here, on the CPU)."""
