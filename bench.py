@@ -680,7 +680,7 @@ def main():
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
     if args.traffic is None and args.workload == "config2" and not args.ranks:
-        args.traffic = 274.05e6
+        args.traffic = 271.70e6
     if args.steps is None:
         args.steps = 128 if args.workload == "config3" else 5000
     if args.impl == "reference":
