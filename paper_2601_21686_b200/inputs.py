@@ -212,3 +212,30 @@ def make_paging(seed: int, seq_lens, reserve_tokens: int = 0, extra_pages: int =
 
 def ragged_lengths(seed: int, B: int, lo: int = 1024, hi: int = 16384) -> np.ndarray:
     return randint(stream_key(seed, TAG_LENS), B, lo, hi).astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------
+# error surfaces for the rank selector (inputs only: the selector's arithmetic is not here)
+# --------------------------------------------------------------------------------------
+
+TAG_SURFACE = 13
+
+
+def error_surfaces(seed: int, n_layers: int, cand_k=RANK_SET, cand_v=RANK_SET, d: int = D_HEAD) -> np.ndarray:
+    """Synthetic layer-output error tables [L][len(cand_k)][len(cand_v)] (fp64) with the qualitative shape the paper
+    reports for its measured ones: zero at the full-rank pair, growing as either rank drops, values costlier to
+    compress than keys, early and late layers more sensitive than the middle ones, plus seeded per-entry jitter."""
+    u = uniform_bits53(stream_key(seed, TAG_SURFACE), torch.arange(n_layers * (2 + len(cand_k) * len(cand_v)), dtype=torch.int64)).numpy()
+    out = np.zeros((n_layers, len(cand_k), len(cand_v)))
+    pos = 0
+    for l in range(n_layers):
+        x = l / max(n_layers - 1, 1)
+        bowl = 0.35 + 1.2 * (2.0 * x - 1.0) ** 2 + (0.6 if x > 0.8 else 0.0)
+        a_k = bowl * (0.6 + 0.8 * u[pos]); a_v = 1.8 * bowl * (0.6 + 0.8 * u[pos + 1]); pos += 2
+        for i, rk in enumerate(cand_k):
+            for j, rv in enumerate(cand_v):
+                lost_k, lost_v = 1.0 - rk / d, 1.0 - rv / d
+                base = a_k * lost_k ** 1.5 + a_v * lost_v ** 1.5 + 0.5 * a_k * a_v * lost_k * lost_v
+                out[l, i, j] = 0.0 if (rk == d and rv == d) else base * (0.9 + 0.2 * u[pos])
+                pos += 1
+    return out
