@@ -447,7 +447,11 @@ def run_multilayer(args):
     Hq, Hkv, T, L = 32, 8, 32768, args.layers
     B = 4 if args.workload == "config3" else 2
     n_steps = args.steps if args.workload == "config3" else 1
-    prof = I.rank_profile(SEED)[:L]
+    if args.rho is not None:
+        # ranks from the library's own selector (Algorithm 2) on synthetic error surfaces of the shape the paper reports
+        prof, _ = S.stief_select_ranks(L, I.RANK_SET, I.RANK_SET, args.rho, surfaces=I.error_surfaces(SEED, L))
+    else:
+        prof = I.rank_profile(SEED)[:L]
     pg = I.make_paging(SEED, [T] * B, reserve_tokens=max(n_steps, 1) + 1)
     bt = torch.from_numpy(pg.block_table).to(dev)
     lens = torch.from_numpy(pg.seq_lens).to(dev)
@@ -677,6 +681,7 @@ def main():
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
     # DRAM read + write bytes per launch of decode_persistent_kernel<64,64> on config 2, from the ncu capture
     # summarised in profiles/decode_persistent_kernel_config2.md (mean of two launches); null for other workloads
+    ap.add_argument("--rho", type=float, default=None, help="multi-layer workloads: take the per-layer ranks from stief_select_ranks at this cache ratio instead of the seeded random profile")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
     if args.traffic is None and args.workload == "config2" and not args.ranks:

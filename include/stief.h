@@ -46,7 +46,8 @@ enum stief_status {
   STIEF_ERR_WORKSPACE = 3,    /* workspace too small for the requested number of splits                */
   STIEF_ERR_CUDA = 4,         /* a CUDA runtime/driver call failed (cudaGetLastError is left readable) */
   STIEF_ERR_BOUNDS = 5,       /* device-side: page id or position out of range (status word only)      */
-  STIEF_ERR_TIMEOUT = 6       /* device-side: a bounded wait on an async copy ran out (status word)    */
+  STIEF_ERR_TIMEOUT = 6,      /* device-side: a bounded wait on an async copy ran out (status word)    */
+  STIEF_ERR_INFEASIBLE = 7    /* rank selection: no candidate pair fits the budget at some layer       */
 };
 
 #define STIEF_PAGE 64
@@ -269,6 +270,35 @@ int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, co
  * so the kernel can be timed alone inside a longer step.  One-shot: cleared by that call.  Passing NULLs
  * cancels a pending request. */
 int stief_time_next_decode_kernel(void* start_event, void* stop_event);
+
+/* ---- rank selection (host only) --------------------------------------------------------------------------
+ * Sequential budgeted rank selection, Algorithm 2 of the paper (Sec. 3.4, Eq. 15-17; cost c = (r_K + r_V) / (2 d_h),
+ * Eq. 23): turns a target cache ratio rho into the per-layer (r_k, r_v) that stief_layer descriptors carry.  The
+ * budget starts at L * rho; before layer l (0-based) the per-layer budget is what is left divided by the L - l layers
+ * still to choose (the divisor of Algorithm 2); the candidate pair of least error whose cost does not exceed it is
+ * taken and its cost subtracted.  Feasibility is decided in exact integer arithmetic on the bits of rho, so a pair
+ * whose cost equals the budget is always accepted.  Ties in the error go to the cheaper pair, then to the smaller key
+ * rank.
+ *
+ * All pointers are HOST pointers; nothing is launched and no CUDA call is made.
+ *   cand_k[n_k], cand_v[n_v]  candidate ranks, each in 1 .. d_h, in any order (d_h itself = keep that side full rank)
+ *   rho                       target ratio, 1/1024 <= rho <= 1
+ *   the error tables come from exactly one of
+ *     surfaces  [L][n_k][n_v] doubles, all known up front, or
+ *     surface   a callback asked for layer l's table only after layers 0 .. l-1 are chosen (the paper evaluates each
+ *               surface on activations that passed through the compressed prefix): it receives ctx, l, the r_k / r_v
+ *               arrays (entries 0 .. l-1 valid) and writes n_k * n_v doubles row-major into delta; non-zero return
+ *               aborts the selection.
+ *   r_k[L], r_v[L]            outputs, owned by the caller
+ *   spent                     optional: total cost sum_l c(r_k[l], r_v[l]) (never above L * rho)
+ *   failed_layer              optional: -1, or the layer at which the call gave up
+ * Returns STIEF_OK; STIEF_ERR_INVALID_ARG (bad sizes, both or neither table source, NaN in a table, callback
+ * failure); STIEF_ERR_INFEASIBLE when no pair fits at some layer (happens exactly when rho is below the cheapest
+ * candidate pair's cost, and then at layer 0). */
+typedef int (*stief_surface_fn)(void* ctx, int32_t layer, const int32_t* r_k_chosen, const int32_t* r_v_chosen, double* delta);
+int stief_select_ranks(int32_t L, int32_t d_h, const int32_t* cand_k, int32_t n_k, const int32_t* cand_v, int32_t n_v,
+                       double rho, const double* surfaces, stief_surface_fn surface, void* ctx, int32_t* r_k,
+                       int32_t* r_v, double* spent, int32_t* failed_layer);
 
 const char* stief_status_string(int status);
 int stief_version(void);

@@ -10,7 +10,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
-from typing import Optional
+from typing import Optional, Sequence
 
 import torch
 
@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libstief.so")
 
 STIEF_OK, STIEF_ERR_INVALID_ARG, STIEF_ERR_UNSUPPORTED, STIEF_ERR_WORKSPACE = 0, 1, 2, 3
-STIEF_ERR_CUDA, STIEF_ERR_BOUNDS, STIEF_ERR_TIMEOUT = 4, 5, 6
+STIEF_ERR_CUDA, STIEF_ERR_BOUNDS, STIEF_ERR_TIMEOUT, STIEF_ERR_INFEASIBLE = 4, 5, 6, 7
 PAGE = 64
 D_HEAD = 128
 STIEF_DECODE_OVERLAP_PREVIOUS = 1
@@ -53,6 +53,9 @@ class _CBatch(ctypes.Structure):
                 ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p)]
 
 
+_SURFACE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
+                               ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double))
+
 _lib_handle = None
 
 
@@ -84,6 +87,7 @@ def lib() -> ctypes.CDLL:
             "stief_q8_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
             "stief_q8_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
             "stief_q8_decode_step": (ctypes.c_int, [QP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
+            "stief_select_ranks": (ctypes.c_int, [I32, I32, P, I32, P, I32, ctypes.c_double, P, _SURFACE_FN, P, P, P, P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -313,3 +317,40 @@ def stief_time_next_decode_kernel(start_event: Optional[torch.cuda.Event], stop_
         if not ev.cuda_event:                 # torch creates the handle lazily, on first record
             ev.record()
     _check(lib().stief_time_next_decode_kernel(start_event.cuda_event, stop_event.cuda_event), "stief_time_next_decode_kernel")
+
+
+def stief_select_ranks(L: int, cand_k: Sequence[int], cand_v: Sequence[int], rho: float, surfaces=None, surface=None,
+                       d_h: int = D_HEAD):
+    """Sequential budgeted rank selection (Algorithm 2) on the host.  ``surfaces``: array-like [L][n_k][n_v] of layer
+    errors, or ``surface(l, chosen)`` -> table [n_k][n_v], called once per layer with the list of (r_k, r_v) already
+    chosen.  Returns (ranks, spent): L pairs and their total cost."""
+    import numpy as np
+    ck = (ctypes.c_int32 * len(cand_k))(*cand_k)
+    cv = (ctypes.c_int32 * len(cand_v))(*cand_v)
+    rk, rv = (ctypes.c_int32 * max(L, 1))(), (ctypes.c_int32 * max(L, 1))()
+    spent, failed = ctypes.c_double(0.0), ctypes.c_int32(-1)
+    tab, cb, raised = None, _SURFACE_FN(), []
+    if surfaces is not None:
+        tab = np.ascontiguousarray(surfaces, dtype=np.float64)
+        if tab.shape != (L, len(cand_k), len(cand_v)):
+            raise ValueError("surfaces must be [L][len(cand_k)][len(cand_v)]")
+    if surface is not None:
+        def _cb(_ctx, l, prk, prv, delta):
+            try:
+                t = np.asarray(surface(l, [(prk[i], prv[i]) for i in range(l)]), dtype=np.float64)
+                if t.shape != (len(cand_k), len(cand_v)):
+                    raise ValueError("surface() must return [len(cand_k)][len(cand_v)]")
+                for n, x in enumerate(t.ravel()):
+                    delta[n] = x
+                return 0
+            except Exception as e:      # an exception must not unwind through the C frame
+                raised.append(e)
+                return 1
+        cb = _SURFACE_FN(_cb)
+    rc = lib().stief_select_ranks(L, d_h, ck, len(cand_k), cv, len(cand_v), float(rho),
+                                  None if tab is None else tab.ctypes.data, cb, None, rk, rv,
+                                  ctypes.byref(spent), ctypes.byref(failed))
+    if raised:
+        raise raised[0]
+    _check(rc, f"stief_select_ranks (layer {failed.value})" if failed.value >= 0 else "stief_select_ranks")
+    return [(rk[l], rv[l]) for l in range(L)], spent.value

@@ -352,10 +352,11 @@ const char* stief_status_string(int status) {
     case STIEF_ERR_CUDA: return "CUDA call failed";
     case STIEF_ERR_BOUNDS: return "page id or position out of range (device)";
     case STIEF_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case STIEF_ERR_INFEASIBLE: return "no candidate rank pair fits the budget";
     default: return "unknown status";
   }
 }
 
-int stief_version(void) { return 200; }
+int stief_version(void) { return 210; }
 
 }  // extern "C"

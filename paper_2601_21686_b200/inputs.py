@@ -234,7 +234,7 @@ def error_surfaces(seed: int, n_layers: int, cand_k=RANK_SET, cand_v=RANK_SET, d
         a_k = bowl * (0.6 + 0.8 * u[pos]); a_v = 1.8 * bowl * (0.6 + 0.8 * u[pos + 1]); pos += 2
         for i, rk in enumerate(cand_k):
             for j, rv in enumerate(cand_v):
-                lost_k, lost_v = 1.0 - rk / d, 1.0 - rv / d
+                lost_k, lost_v = max(0.0, 1.0 - rk / d), max(0.0, 1.0 - rv / d)
                 base = a_k * lost_k ** 1.5 + a_v * lost_v ** 1.5 + 0.5 * a_k * a_v * lost_k * lost_v
                 out[l, i, j] = 0.0 if (rk == d and rv == d) else base * (0.9 + 0.2 * u[pos])
                 pos += 1
