@@ -139,6 +139,22 @@ def attend_path_b(q: np.ndarray, K_down: np.ndarray, V_down: np.ndarray, U_k, U_
     return out, lse
 
 
+def attend_rows_causal(Q: np.ndarray, K_down: np.ndarray, V_down: np.ndarray, U_k, U_v, q_start: int, path: str = "b",
+                       d_h: int = D_HEAD):
+    """Several query rows of one head against one cache (App. A.1: during prefilling Q has one row per prefix token;
+    Eq. 18 per row).  Row i sits at absolute position q_start + i and, the layer being a decoder layer, attends the
+    cached positions 0 .. q_start + i only (its own key/value row is in the cache).  Each row is the single-row
+    definition applied to that prefix.  Returns (out [n_q, d_out], lse [n_q])."""
+    fn = attend_path_a if path == "a" else attend_path_b
+    outs, lses = [], []
+    for i in range(Q.shape[0]):
+        n = q_start + i + 1
+        o, l = fn(Q[i], K_down[:n], V_down[:n], U_k, U_v, d_h)
+        outs.append(o)
+        lses.append(l)
+    return np.stack(outs), np.array(lses)
+
+
 def attend_compressed_partial(q, K_down, V_down, U_k, d_h: int = D_HEAD):
     """One T-chunk of Path B without the back-projection: (o_down [r_v] normalised within the chunk, lse)."""
     K_down = np.asarray(K_down, dtype=np.float64)

@@ -355,6 +355,49 @@ def test_folding_the_projections_into_the_linear_layers_changes_nothing():
     assert np.abs(out_down @ Uv.T - out).max() < 1e-12
 
 
+def test_causal_rows_against_library_attention():
+    # full rank, the whole sequence as queries: the textbook causal attention of a decoder, here torch's own routine
+    # in fp64; then a chunk of queries at an offset, with the mask written out (True = may attend)
+    import torch
+    n, d = 70, 128
+    K = I.normal_f64(I.stream_key(31, I.TAG_K), n * d).numpy().reshape(n, d)
+    V = I.normal_f64(I.stream_key(31, I.TAG_V), n * d).numpy().reshape(n, d)
+    Q = I.normal_f64(I.stream_key(31, I.TAG_Q), n * d).numpy().reshape(n, d)
+    tq, tk, tv = (torch.from_numpy(x)[None, None] for x in (Q, K, V))
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)[0, 0].numpy()
+    for path in ("a", "b"):
+        got, lse = O.attend_rows_causal(Q, K, V, None, None, 0, path=path)
+        assert np.abs(got - want).max() < 1e-12
+    assert abs(lse[0] - (K[0] @ Q[0]) / np.sqrt(d)) < 1e-12                  # one visible position: lse = its score
+    start, nq = 41, 29
+    mask = torch.arange(n)[None, :] <= (start + torch.arange(nq))[:, None]
+    want = torch.nn.functional.scaled_dot_product_attention(tq[:, :, start:], tk, tv, attn_mask=mask)[0, 0].numpy()
+    got, _ = O.attend_rows_causal(Q[start:], K, V, None, None, start)
+    assert got.shape == (nq, d) and np.abs(got - want).max() < 1e-12
+
+
+def test_causal_rows_with_bases_and_causality():
+    n, r_k, r_v, start = 90, 48, 96, 60
+    Uk = I.stiefel_basis_f64(32, I.TAG_UK, 0, 0, r_k)
+    Uv = I.stiefel_basis_f64(32, I.TAG_UV, 0, 0, r_v)
+    K = I.normal_f64(I.stream_key(32, I.TAG_K), n * 128).numpy().reshape(n, 128)
+    V = I.normal_f64(I.stream_key(32, I.TAG_V), n * 128).numpy().reshape(n, 128)
+    Q = I.normal_f64(I.stream_key(32, I.TAG_Q), (n - start) * 128).numpy().reshape(n - start, 128)
+    Kd, Vd = O.compress(K, Uk), O.compress(V, Uv)
+    a, la = O.attend_rows_causal(Q, Kd, Vd, Uk, Uv, start, path="a")
+    b, lb = O.attend_rows_causal(Q, Kd, Vd, Uk, Uv, start, path="b")
+    assert np.abs(a - b).max() < 1e-12 and np.abs(la - lb).max() < 1e-12
+    # the last row is plain decode attention over the whole cache
+    o, l = O.attend_path_b(Q[-1], Kd, Vd, Uk, Uv)
+    assert np.array_equal(o, b[-1]) and l == lb[-1]
+    # a cache row at position p influences rows at positions >= p and no earlier one
+    p = start + 10
+    Kd2 = Kd.copy(); Kd2[p] += 1.0
+    c, _ = O.attend_rows_causal(Q, Kd2, Vd, Uk, Uv, start)
+    changed = np.abs(c - b).max(axis=1) > 0
+    assert not changed[:10].any() and changed[10:].all()
+
+
 def test_planted_mistakes_fail_the_pins():
     """Sanity of the pins themselves: a wrong softmax scale or a wrong query-head -> KV-head map is
     detected by the reconstructed-KV library check (the mistakes are planted here, on the CPU)."""
