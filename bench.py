@@ -428,6 +428,84 @@ def run_q8(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# a chunk of causal queries over the compressed cache (chunked prefill): a measurement case, not the headline line
+# ------------------------------------------------------------------------------------------------
+def run_mq(args):
+    import paper_2601_21686_b200 as S
+    from paper_2601_21686_b200 import inputs as I
+    from paper_2601_21686_b200 import build as Bld
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Bld.build()
+    S.lib()
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    cfg = dict(SINGLE_LAYER["config2"])
+    if args.ranks:
+        cfg["r_k"], cfg["r_v"] = (int(x) for x in args.ranks.split(","))
+    B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
+    n_q = args.n_q
+    pg = I.make_paging(SEED, [T] * B, reserve_tokens=1)
+    batch = S.Batch(torch.from_numpy(pg.block_table).to(dev), torch.from_numpy(pg.seq_lens).to(dev))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n_caches = max(1, min(args.caches, 2))
+    layers = []
+    for l in range(n_caches):
+        U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
+        layer = S.Layer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev),
+                        torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.bfloat16, device=dev),
+                        torch.zeros(pg.num_pages, Hkv, 64, r_v, dtype=torch.bfloat16, device=dev))
+        K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
+        V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
+        S.stief_prefill_compress(layer, batch, K, V, status=status)
+        del K, V
+        layers.append(layer)
+    qs = [I.normal_bf16(I.stream_key(SEED, I.TAG_Q, 100 + i), (B, n_q, Hq, 128), device=dev) for i in range(2)]
+    out = torch.empty(B, n_q, Hq, 128, dtype=torch.bfloat16, device=dev)
+    torch.cuda.synchronize()
+
+    def step(i):
+        S.stief_mq_attention(layers[i % n_caches], batch, qs[i % 2], out, status=status)
+
+    K_steps, W = min(args.steps, 50), max(min(args.warmup, 5), 3)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for i in range(K_steps):
+        step(W + i)
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1) / K_steps
+    sampler.stop()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    visible = sum(T - n_q + i + 1 for i in range(n_q))                     # cached positions each query row attends, summed
+    flops = B * Hq * (2 * visible * (r_k + r_v) + n_q * 2 * 128 * (r_k + r_v))
+    tflops = flops / (ms * 1e-3) / 1e12
+    cache_bytes = B * Hkv * T * 2 * (r_k + r_v)
+    print(json.dumps({
+        "metric": "mq_attention_tflops", "value": tflops, "unit": "TFLOP/s", "n_gpus": 1, "steps": K_steps, "warmup": W,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "dtype_note": "bf16 tensor-core operands (tcgen05), fp32 accumulate in TMEM", "data": "synthetic",
+        "config": {"workload": f"chunk of {n_q} causal query tokens per sequence at the end of a {T}-token compressed cache, "
+                               f"B={B} Hq={Hq} Hkv={Hkv} r_k={r_k} r_v={r_v}: query projection + causal attention + back-projection, one launch",
+                   "l2": f"steps alternate over {n_caches} layer caches of {cache_bytes / 2**20:.0f} MiB"},
+        "query_tokens_per_s": B * n_q / (ms * 1e-3), "gpu_launches": K_steps,
+        "roofline": {"bound": "tensor", "kernel": "mq_attention_kernel", "achieved": tflops, "peak": tf_peak, "unit": "TFLOP/s",
+                     "frac": tflops / tf_peak, "peak_kind": peak_kind, "traffic": None, "flops_per_launch": flops,
+                     "avg_launch_ms": ms},
+        "clocks": sampler.summary(t0, t1)}))
+
+
+# ------------------------------------------------------------------------------------------------
 # the 32-layer workloads: config 3 (decode steps over per-layer ranks) and config 5 (prefill + first decode)
 # ------------------------------------------------------------------------------------------------
 def run_multilayer(args):
@@ -681,6 +759,8 @@ def main():
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
     # DRAM read + write bytes per launch of decode_persistent_kernel<64,64> on config 2, from the ncu capture
     # summarised in profiles/decode_persistent_kernel_config2.md (mean of two launches); null for other workloads
+    ap.add_argument("--mq", action="store_true", help="measure the multi-query (chunked prefill) attention kernel on the config-2 shape")
+    ap.add_argument("--n-q", dest="n_q", type=int, default=2048, help="query tokens per sequence for --mq")
     ap.add_argument("--rho", type=float, default=None, help="multi-layer workloads: take the per-layer ranks from stief_select_ranks at this cache ratio instead of the seeded random profile")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()
@@ -692,6 +772,8 @@ def main():
         run_reference(args)
     elif args.q8:
         run_q8(args)
+    elif args.mq:
+        run_mq(args)
     elif args.workload in SINGLE_LAYER:
         run_ours(args)
     else:

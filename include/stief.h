@@ -271,6 +271,31 @@ int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, co
  * cancels a pending request. */
 int stief_time_next_decode_kernel(void* start_event, void* stop_event);
 
+/* ---- several causal query rows per head (chunked prefill, speculative decode) --------------------------------
+ * App. A.1 of the paper: during prefilling Q has one row per prefix token and Eq. 18 holds per row; the layer being
+ * a decoder layer, row i of sequence b sits at absolute position p = seq_lens[b] - q_len_b + i and attends the cached
+ * positions 0 .. p.  The cache must already hold the query tokens' own rows (stief_prefill_compress / stief_append
+ * first), i.e. the queries are the LAST q_len_b tokens of each cached sequence.  Evaluated in the compressed space
+ * like stief_decode_attention (q' = q U_k, scores and mixing on the compressed rows, one back-projection), on the
+ * tcgen05 tensor cores; q' and the probabilities pass through bf16, scores, sums and the compressed output keep fp32
+ * accuracy.
+ *
+ *   q        device, bf16 [B][n_q][Hq][d_q] with element strides q_stride_b / q_stride_t between sequences / tokens
+ *            (heads and elements contiguous, strides multiples of 8); d_q = 128, or r_k when U_k is NULL (folded keys)
+ *   n_q      query tokens per sequence in q and out (> 0)
+ *   q_lens   device int32 [B] or NULL: how many of the n_q rows of each sequence are real (clamped to 0 .. n_q; rows
+ *            beyond are neither computed nor written); NULL = n_q for every sequence.  q_len_b > seq_lens[b] sets
+ *            STIEF_ERR_BOUNDS in the status word and skips the sequence
+ *   out      device, bf16 [B][n_q][Hq][d_out], strides as for q; d_out = 128, or r_v when U_v is NULL (folded values:
+ *            the compressed output is returned for a folded output projection)
+ *   out_lse  optional device fp32 [B][n_q][Hq] (contiguous): natural-log-sum-exp of each row's scaled scores
+ *   flags    must be 0
+ * All ranks 32/48/64/96/128; Hq / Hkv must divide 128 (a 128-row tile holds whole tokens), else
+ * STIEF_ERR_UNSUPPORTED.  No workspace; nothing is allocated.  Asynchronous on `stream`. */
+int stief_mq_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int64_t q_stride_b,
+                       int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, uint16_t* out, int64_t out_stride_b,
+                       int64_t out_stride_t, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+
 /* ---- rank selection (host only) --------------------------------------------------------------------------
  * Sequential budgeted rank selection, Algorithm 2 of the paper (Sec. 3.4, Eq. 15-17; cost c = (r_K + r_V) / (2 d_h),
  * Eq. 23): turns a target cache ratio rho into the per-layer (r_k, r_v) that stief_layer descriptors carry.  The

@@ -1,0 +1,186 @@
+"""Several causal query rows per head over the compressed cache (chunked prefill / speculative decode) against the
+oracle's row-by-row definition (App. A.1, Eq. 18 per row), on the cache rows the GPU itself stored."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2601_21686_b200 as S
+from oracle import stief_oracle as O
+from paper_2601_21686_b200 import inputs as I
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _queries(seed, B, n_q, Hq, d=128, scale=1.0):
+    return I.normal_bf16(I.stream_key(seed, I.TAG_Q, 77), (B, n_q, Hq, d), scale=scale)
+
+
+def _run(c, q, q_lens=None, lse=True):
+    B, n_q, Hq = q.shape[:3]
+    d_out = 128 if c.U_v is not None else c.r_v
+    out = torch.full((B, n_q, Hq, d_out), float("nan"), dtype=torch.bfloat16, device=DEV)
+    out_lse = torch.full((B, n_q, Hq), float("nan"), dtype=torch.float32, device=DEV) if lse else None
+    ql = None if q_lens is None else torch.tensor(q_lens, dtype=torch.int32, device=DEV)
+    S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, q_lens=ql, out_lse=out_lse, status=c.status)
+    torch.cuda.synchronize()
+    return out, out_lse
+
+
+def _reference(c, q, q_lens):
+    """Oracle rows on the cache the GPU holds: returns (ref [B, n_q, Hq, d_out] with NaN where no row is due, lse)."""
+    B, n_q, Hq = q.shape[:3]
+    G = Hq // c.Hkv
+    d_out = 128 if c.U_v is not None else c.r_v
+    ref = np.full((B, n_q, Hq, d_out), np.nan)
+    lse = np.full((B, n_q, Hq), np.nan)
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    for b in range(B):
+        n, ql = int(c.seq_lens[b]), int(q_lens[b])
+        if ql == 0:
+            continue
+        Kd = U.f64(U.gpu_cache_rows(c, c.layer.k_pool, b, n))
+        Vd = U.f64(U.gpu_cache_rows(c, c.layer.v_pool, b, n))
+        for g in range(Hq):
+            h = g // G
+            o, l = O.attend_rows_causal(U.f64(q)[b, :ql, g], Kd[:, h], Vd[:, h], O.basis_of(Uk, h), O.basis_of(Uv, h), n - ql)
+            ref[b, :ql, g], lse[b, :ql, g] = o, l
+    return ref, lse
+
+
+def _compare(out, out_lse, ref, lse):
+    due = ~np.isnan(ref[..., 0])
+    g = out.double().cpu().numpy()
+    assert np.all(np.isnan(g[~due])), "rows beyond q_lens were written"
+    U.check_out(out[torch.from_numpy(due)], ref[due])
+    if out_lse is not None:
+        gl = out_lse.double().cpu().numpy()
+        # q' is rounded to bf16 (relative 2^-9 per element), so a score, and with it the LSE, carries an error of up to
+        # about 2^-9 of its own magnitude on top of the fp32 arithmetic
+        assert np.all(np.isnan(gl[~due])) and np.abs(gl[due] - lse[due]).max() < 2e-2 + 2.0 ** -8 * np.abs(lse[due]).max()
+
+
+@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 128), (32, 48), (96, 32), (48, 96), (64, 128), (128, 64)])
+def test_chunk_of_queries_all_rank_pairs(r_k, r_v):
+    c = U.make_case(900 + r_k + r_v, 2, 8, 2, r_k, r_v, [300, 200], lowrank=True)
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(1, 2, 70, 8, scale=1.5)
+    q_lens = [70, 33]
+    out, out_lse = _run(c, q, q_lens)
+    assert int(c.status.item()) == 0
+    _compare(out, out_lse, *_reference(c, q, q_lens))
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (16, 2), (8, 1)])
+def test_group_sizes(Hq, Hkv):
+    c = U.make_case(77 + Hq, 2, Hq, Hkv, 64, 64, [257, 129])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    n_q = 150 if Hq == Hkv else 40
+    q = _queries(2, 2, n_q, Hq)
+    q_lens = [n_q, min(n_q, 129)]
+    out, out_lse = _run(c, q, q_lens)
+    assert int(c.status.item()) == 0
+    _compare(out, out_lse, *_reference(c, q, q_lens))
+
+
+def test_whole_prompt_as_queries_and_single_rows():
+    # q_len = seq_len (plain causal prefill attention, first row sees one position); q_len = 1 (decode); q_len = 0
+    c = U.make_case(5, 3, 8, 2, 64, 64, [130, 64, 90])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(3, 3, 130, 8)
+    q_lens = [130, 1, 0]
+    out, out_lse = _run(c, q, q_lens)
+    assert int(c.status.item()) == 0
+    ref, lse = _reference(c, q, q_lens)
+    _compare(out, out_lse, ref, lse)
+    # the single row of sequence 1 is what the decode kernel returns for the same query
+    ws = U.workspace_for(c, 2)
+    dq = torch.zeros(3, 8, 128, dtype=torch.bfloat16)
+    dq[1] = q[1, 0]
+    dout = torch.zeros(3, 8, 128, dtype=torch.bfloat16, device=DEV)
+    S.stief_decode_attention(c.layer, c.batch, dq.to(DEV), ws, 2, dout, status=c.status)
+    torch.cuda.synchronize()
+    assert np.abs(dout[1].double().cpu().numpy() - out[1, 0].double().cpu().numpy()).max() < 1e-2
+
+
+def test_growing_scores_force_the_accumulator_rescale():
+    # keys aligned with the queries and growing with the position: every page raises the row maxima by far more than
+    # the lazy-rescale threshold, so the TMEM accumulator is rescaled page after page
+    B, Hq, Hkv, T, n_q = 1, 4, 1, 520, 40
+    c = U.make_case(41, B, Hq, Hkv, 64, 64, [T])
+    Uk = U.f64(c.U_k)[0]
+    direction = Uk[:, 0] / np.linalg.norm(Uk[:, 0])                       # lies in the key basis: survives the projection
+    ramp = np.linspace(0.0, 60.0, T)[:, None] * direction[None, :]
+    K = torch.from_numpy(ramp + 0.05 * U.f64(c.K)[0, :, 0]).to(torch.bfloat16)[None, :, None, :]
+    c.K = K.contiguous()
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = torch.from_numpy(np.tile(12.0 * direction, (B, n_q, Hq, 1)) + 0.1 * U.f64(_queries(4, B, n_q, Hq))).to(torch.bfloat16)
+    out, out_lse = _run(c, q, [n_q])
+    assert int(c.status.item()) == 0
+    ref, lse = _reference(c, q, [n_q])
+    # the spread of scores is ~ 60 * 12 / sqrt(128) = 64 nats over the sequence: far beyond the threshold
+    assert lse[0, -1, 0] - lse[0, 0, 0] > 1.0
+    _compare(out, out_lse, ref, lse)
+
+
+@pytest.mark.parametrize("fold_k,fold_v", [(True, True), (True, False), (False, True)])
+def test_folded_sides(fold_k, fold_v):
+    r_k, r_v, B, Hq, Hkv = 64, 96, 2, 8, 2
+    c = U.make_case(123, B, Hq, Hkv, r_k, r_v, [200, 140])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)     # cache built with the bases
+    q = _queries(6, B, 50, Hq)
+    Uk = U.f64(c.U_k)
+    G = Hq // Hkv
+    q_in = q
+    if fold_k:      # what a folded W_Q hands over: q' rounded to bf16
+        qp = np.stack([np.stack([U.f64(q)[b, :, g] @ Uk[g // G] for g in range(Hq)], axis=1) for b in range(B)])
+        q_in = torch.from_numpy(qp).to(torch.float32).to(torch.bfloat16)
+        c.layer.U_k, c.U_k = None, None
+    if fold_v:
+        c.layer.U_v, c.U_v = None, None
+    out, out_lse = _run(c, q_in, [50, 50])
+    assert int(c.status.item()) == 0 and out.shape[-1] == (r_v if fold_v else 128)
+    _compare(out, out_lse, *_reference(c, q_in, [50, 50]))
+
+
+def test_strided_tensors_and_untouched_padding():
+    c = U.make_case(9, 2, 8, 2, 64, 64, [190, 100])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    n_q = 37
+    q = _queries(8, 2, n_q, 8)
+    qbig = torch.zeros(2, n_q + 3, 8 * 128 + 64, dtype=torch.bfloat16, device=DEV)
+    qv = torch.as_strided(qbig, (2, n_q, 8, 128), (qbig.stride(0), qbig.stride(1), 128, 1))
+    qv.copy_(q.to(DEV))
+    obig = torch.full((2, n_q + 1, 8 * 128 + 8), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ov = torch.as_strided(obig, (2, n_q, 8, 128), (obig.stride(0), obig.stride(1), 128, 1))
+    S.stief_mq_attention(c.layer, c.batch, qv, ov, status=c.status)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    ref, _ = _reference(c, q, [n_q, n_q])
+    U.check_out(ov.contiguous(), ref)
+    assert torch.isnan(obig[:, n_q:]).all() and torch.isnan(obig[:, :, 8 * 128:]).all()
+
+
+def test_more_queries_than_cached_tokens_is_reported():
+    c = U.make_case(10, 2, 8, 2, 64, 64, [100, 20])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(9, 2, 40, 8)
+    out, _ = _run(c, q, [40, 40], lse=False)
+    assert int(c.status.item()) == S.STIEF_ERR_BOUNDS
+    assert torch.isnan(out[1]).all() and not torch.isnan(out[0]).any()
+
+
+def test_unsupported_group_size_and_bad_arguments():
+    c = U.make_case(11, 1, 6, 2, 64, 64, [100])          # G = 3 does not divide 128
+    q = _queries(10, 1, 8, 6)
+    out = torch.zeros(1, 8, 6, 128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(S.StiefError) as e:
+        S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status)
+    assert e.value.code == S.STIEF_ERR_UNSUPPORTED
+    c = U.make_case(12, 1, 8, 2, 64, 64, [100])
+    q = _queries(10, 1, 8, 8)
+    out = torch.zeros(1, 8, 8, 128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(S.StiefError) as e:
+        S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, flags=4)
+    assert e.value.code == S.STIEF_ERR_INVALID_ARG
