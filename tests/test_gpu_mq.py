@@ -53,7 +53,9 @@ def _compare(out, out_lse, ref, lse):
     due = ~np.isnan(ref[..., 0])
     g = out.double().cpu().numpy()
     assert np.all(np.isnan(g[~due])), "rows beyond q_lens were written"
-    U.check_out(out[torch.from_numpy(due)], ref[due])
+    # the absolute bound of the decode tests (1e-2) presumes outputs of order one; a bf16 output of magnitude x is
+    # spaced 2^-8 x apart, so for peaked attention (outputs near single value rows, |x| up to 4) it scales with x
+    U.check_out(out[torch.from_numpy(due)], ref[due], max_abs=max(1e-2, 2.0 ** -7 * np.abs(ref[due]).max()))
     if out_lse is not None:
         gl = out_lse.double().cpu().numpy()
         # q' is rounded to bf16 (relative 2^-9 per element), so a score, and with it the LSE, carries an error of up to
