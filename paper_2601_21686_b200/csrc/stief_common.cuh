@@ -68,6 +68,28 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   report(status, STIEF_ERR_TIMEOUT);
 }
 
+// The same bounded wait on the non-blocking form.  mbarrier.try_wait may park the thread for a while before it looks
+// again; where a short wait sits on a latency-critical chain between a few warps, polling test_wait reacts at once.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t i = 0; i < (kWaitSpins << 2); ++i) {
+    if (mbar_test_wait(bar, parity)) return;
+    if ((i & 4095u) == 4095u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  report(status, STIEF_ERR_TIMEOUT);
+}
+
 // Programmatic dependent launch.  launch_dependents lets the next kernel on the stream (if it was
 // launched with programmatic stream serialization) start as soon as every CTA of this grid has passed
 // this point or exited; grid_dependency_wait blocks until the grids this one depends on have completed

@@ -6,12 +6,12 @@
 //
 // A work unit is (sequence b, KV head h, 256 query rows): two row tiles of 128 rows, a row being (token i, query
 // head g of the group of h), token-major.  Both tiles use every cache page once it is in shared memory.
-// One persistent CTA per SM, 320 threads, warp-specialised:
+// One persistent CTA per SM, 352 threads, warp-specialised:
 //   warp 0      producer.  Items go through a ring of 32 KiB stages, in the order the MMA warp consumes them: the
 //               raw query tiles and U_k (unless the key side is folded), the cache pages (K page | V page), U_v
 //               (unless the value side is folded).  Everything arrives by tiled TMA loads, in the swizzled blocks
 //               that tcgen05.mma reads (see Blocks); block-table entries are fetched 32 at a time, a batch ahead.
-//   warp 1      MMA issue (one lane) and TMEM allocation.  Per unit: Q' = Q U_k  (A = raw q rows, B = U_k as an
+//   warps 1,10  MMA issue, one thread per tile (warp 1 also allocates TMEM).  Per unit: Q' = Q U_k  (A = raw q rows, B = U_k as an
 //               MN-major operand) into the tile's accumulator columns; per page j and tile: S = Q' K_j^T (N = 64
 //               positions) into one of two score buffers, then O += P_j V_j (B = the V page, MN-major) once the
 //               softmax warps have published P_j; finally OUT = O_down U_v^T (B = U_v, K-major).  QK of page j+1 is
@@ -41,7 +41,7 @@ namespace mq {
 
 using namespace tc;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kRows = 128;                      // rows per tile
 constexpr int kStageBytes = 32768;              // one ring stage
 constexpr int kPBytes = kRows * kPage * 2;      // one tile's P operand: 128 rows x 64 positions bf16
@@ -122,24 +122,24 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const uint32_t ring = base;
   const uint32_t qp = ring + nst * kStageBytes;                 // Q' / O_down operands, one region per tile
   uint8_t* qp_ptr = base_ptr + nst * kStageBytes;
-  const uint32_t pb = qp + 2 * a.qp_bytes;                      // P operands
+  const uint32_t pb = qp + 2 * a.qp_bytes;                      // P operands, two buffers per tile
   uint8_t* pb_ptr = qp_ptr + 2 * a.qp_bytes;
-  const uint32_t ctrl = pb + 2 * kPBytes;
-  uint8_t* ctrl_ptr = pb_ptr + 2 * kPBytes;
+  const uint32_t ctrl = pb + 4 * kPBytes;
+  uint8_t* ctrl_ptr = pb_ptr + 4 * kPBytes;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (6 + s) * 8; };
   auto s_full = [&](int t, int i) { return ctrl + (12 + t * 2 + i) * 8; };
   auto s_free = [&](int t, int i) { return ctrl + (16 + t * 2 + i) * 8; };
-  auto p_full = [&](int t) { return ctrl + (20 + t) * 8; };
-  auto p_free = [&](int t) { return ctrl + (22 + t) * 8; };
-  auto qacc_full = [&](int t) { return ctrl + (24 + t) * 8; };
-  auto qp_ready = [&](int t) { return ctrl + (26 + t) * 8; };
-  auto o_full = [&](int t) { return ctrl + (28 + t) * 8; };
-  auto od_ready = [&](int t) { return ctrl + (30 + t) * 8; };
-  auto out_full = [&](int t) { return ctrl + (32 + t) * 8; };
-  auto unit_done = [&](int t) { return ctrl + (34 + t) * 8; };
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 36 * 8);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + 36 * 8 + 4);
+  auto p_full = [&](int t, int i) { return ctrl + (20 + t * 2 + i) * 8; };
+  auto p_free = [&](int t, int i) { return ctrl + (24 + t * 2 + i) * 8; };
+  auto qacc_full = [&](int t) { return ctrl + (28 + t) * 8; };
+  auto qp_ready = [&](int t) { return ctrl + (30 + t) * 8; };
+  auto o_full = [&](int t) { return ctrl + (32 + t) * 8; };
+  auto od_ready = [&](int t) { return ctrl + (34 + t) * 8; };
+  auto out_full = [&](int t) { return ctrl + (36 + t) * 8; };
+  auto unit_done = [&](int t) { return ctrl + (38 + t) * 8; };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 40 * 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + 40 * 8 + 4);
 
   const int RK = a.L.r_k, RV = a.L.r_v, G = a.L.G, Hkv = a.L.Hkv;
   const bool fold_k = a.L.U_k == nullptr, fold_v = a.L.U_v == nullptr;
@@ -151,15 +151,15 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+      mbar_init(empty_bar(s), 2);        // one arrival from each tile's MMA thread
     }
     for (int t = 0; t < 2; ++t) {
       for (int i = 0; i < 2; ++i) {
         mbar_init(s_full(t, i), 1);
         mbar_init(s_free(t, i), 4);       // one arrival per softmax warp of the tile
+        mbar_init(p_full(t, i), 4);
+        mbar_init(p_free(t, i), 1);
       }
-      mbar_init(p_full(t), 4);
-      mbar_init(p_free(t), 1);
       mbar_init(qacc_full(t), 1);
       mbar_init(qp_ready(t), fold_k ? 1 : 4);   // folded keys: the producer's TMA load completes it
       mbar_init(o_full(t), 1);
@@ -258,9 +258,16 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       for (int t = 0; t < 2; ++t) kt[t] += w.np[t] > 0;
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 10) {
     // ------------------------------------------------------------------------------------------ MMA issue
+    // One thread per tile feeds the tensor core (warp 1 for tile 0, warp 10 for tile 1): issuing a tcgen05.mma costs
+    // the issuing thread some tens of cycles, more than these small MMAs (N = 64, K = 16) occupy the tensor pipe, so
+    // two issuers keep it busier than one.  Every instruction between two MMAs is on the critical path: descriptors
+    // are a per-buffer base plus an offset that is a shift and a mask, and the K loops are unrolled.
+    // Both threads walk ALL ring items in order; an item a thread has no use for is released with a plain arrive
+    // once it has landed, so each stage always collects two arrivals.
     if (lane == 0) {
+      const int mt = warp == 1 ? 0 : 1;
       const uint32_t id_qk = idesc_bf16_f32(kRows, kPage);
       const uint32_t id_pv = idesc_bf16_f32_bmn(kRows, RV);
       const uint32_t id_pj = idesc_bf16_f32_bmn(kRows, RK);
@@ -270,9 +277,19 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const uint64_t d_sw128 = desc_template(2, 16, 1024);                          // raw q rows, P rows
       const uint64_t d_vpage = desc_template(bv.layout, kPage * bv.span, 8 * bv.span);   // V page, MN-major
       const uint64_t d_uk = desc_template(bk.layout, kD * bk.span, 8 * bk.span);    // U_k, MN-major
-      const int kper = bk.bw / 16, vper = bv.bw / 16;                               // K = 16 steps per block
+      const int nk = RK / 16, nv = RV / 16;
+      // descriptor offset (in 16-byte units) of K step k of a K-major operand: inside a block 2 units (32 bytes) per
+      // step, then the next block.  Steps per block are 4, 2 or 1: a shift and a mask.
+      const int lgk = bk.bw == 64 ? 2 : bk.bw == 32 ? 1 : 0, lgv = bv.bw == 64 ? 2 : bv.bw == 32 ? 1 : 0;
+      const uint32_t qblk = (uint32_t)(kRows * bk.span) >> 4, kblk = (uint32_t)(kPage * bk.span) >> 4;
+      const uint32_t oblk = (uint32_t)(kRows * bv.span) >> 4;
+      auto koff = [](int k, int lg, uint32_t blk) { return (uint32_t)(k >> lg) * blk + (uint32_t)(k & ((1 << lg) - 1)) * 2u; };
+      const uint32_t pv_b = (uint32_t)(16 * bv.span) >> 4;                          // V page: 16 rows per K step
+      const uint64_t dq = desc_at(d_kmaj_k, qp + mt * a.qp_bytes);                  // this tile's Q' operand
+      const uint64_t dod = desc_at(d_kmaj_v, qp + mt * a.qp_bytes);                 // and its O_down operand (same region)
+      const uint32_t t_s = tmem_base + mt * 256, t_o = t_s + 128;                   // score buffers; Q' / O accumulator
       int st = 0, use = 0;
-      int kt[2] = {0, 0}, pn[2] = {0, 0};
+      int kt = 0, pn = 0;
       auto consume = [&](uint32_t& addr, int& stage) {          // next item of the ring, once it has landed
         mbar_wait(full_bar(st), use & 1, abort_flag, status);
         addr = ring + st * kStageBytes;
@@ -282,105 +299,101 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           ++use;
         }
       };
+      auto release = [&](int stage, bool used) {                // after the MMAs that read it, or at once when unused
+        if (used) umma_commit(empty_bar(stage));
+        else mbar_arrive(empty_bar(stage));
+      };
       for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const Unit w = decode_unit(a, u, TT);
         if (!w.valid) continue;
-        const int npmax = max(w.np[0], w.np[1]);
+        const int np = mt ? w.np[1] : w.np[0], np_other = mt ? w.np[0] : w.np[1];
+        const int npmax = max(np, np_other);
+        const bool active = np > 0;
         if (!fold_k) {
-          uint32_t qa[2] = {0, 0}, ua;
-          int qs[2] = {-1, -1}, us;
-          for (int t = 0; t < 2; ++t)
-            if (w.np[t] > 0) consume(qa[t], qs[t]);
+          uint32_t qa = 0, ua, tmp;
+          int qs = -1, us, ts;
+          if (w.np[0] > 0) {                                    // tile 0's raw queries
+            if (mt == 0) consume(qa, qs);
+            else { consume(tmp, ts); release(ts, false); }
+          }
+          if (w.np[1] > 0) {                                    // tile 1's
+            if (mt == 1) consume(qa, qs);
+            else { consume(tmp, ts); release(ts, false); }
+          }
           consume(ua, us);
-          for (int t = 0; t < 2; ++t) {
-            if (w.np[t] == 0) continue;
-            if (kt[t] > 0) mbar_wait(unit_done(t), (kt[t] - 1) & 1, abort_flag, status);   // the tile's accumulator columns are free
+          if (active) {
+            if (kt > 0) mbar_wait(unit_done(mt), (kt - 1) & 1, abort_flag, status);   // the tile's accumulator columns are free
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + t * 256 + 128;
+            const uint64_t da = desc_at(d_sw128, qa), db = desc_at(d_uk, ua);
 #pragma unroll
             for (int k = 0; k < kD / 16; ++k)
-              umma_bf16(d_tmem, desc_at(d_sw128, qa[t] + (k >> 2) * (kStageBytes / 2) + (k & 3) * 32),
-                        desc_at(d_uk, ua + k * 16 * bk.span), id_pj, k > 0 ? 1u : 0u);
-            umma_commit(qacc_full(t));
+              umma_bf16(t_o, da + (uint32_t)(((k >> 2) * (kStageBytes / 2) + (k & 3) * 32) >> 4), db + (uint32_t)(k * bk.span),
+                        id_pj, k > 0 ? 1u : 0u);
+            umma_commit(qacc_full(mt));
+            release(qs, true);
           }
-          for (int t = 0; t < 2; ++t)
-            if (qs[t] >= 0) umma_commit(empty_bar(qs[t]));
-          umma_commit(empty_bar(us));
+          release(us, active);
         }
-        for (int t = 0; t < 2; ++t)
-          if (w.np[t] > 0) mbar_wait(qp_ready(t), kt[t] & 1, abort_flag, status);
+        if (active) mbar_wait(qp_ready(mt), kt & 1, abort_flag, status);
         tc_fence_after();
 
         uint32_t prev_v = 0;
         int prev_stage = -1;
         auto issue_pv = [&](int jj, uint32_t vaddr, int stage) {
-          for (int t = 0; t < 2; ++t) {
-            if (jj >= w.np[t]) continue;
-            const int n = pn[t] + jj;
-            mbar_wait(p_full(t), n & 1, abort_flag, status);
+          if (jj < np) {
+            const int n = pn + jj;
+            mbar_wait(p_full(mt, n & 1), (n >> 1) & 1, abort_flag, status);
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + t * 256 + 128;
-            const uint32_t pa = pb + t * kPBytes;
+            const uint64_t da = desc_at(d_sw128, pb + (mt * 2 + (n & 1)) * kPBytes), db = desc_at(d_vpage, vaddr);
 #pragma unroll
             for (int k = 0; k < kPage / 16; ++k)
-              umma_bf16(d_tmem, desc_at(d_sw128, pa + k * 32), desc_at(d_vpage, vaddr + k * 16 * bv.span), id_pv,
-                        (jj > 0 || k > 0) ? 1u : 0u);
-            umma_commit(p_free(t));
+              umma_bf16(t_o, da + (uint32_t)(2 * k), db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
+            umma_commit(p_free(mt, n & 1));
           }
-          umma_commit(empty_bar(stage));                        // K and V of this page have been read
+          release(stage, jj < np);                              // K and V of this page are no longer needed by this tile
         };
         for (int j = 0; j < npmax; ++j) {
           uint32_t kaddr;
           int stage;
           consume(kaddr, stage);
-          tc_fence_after();
-          for (int t = 0; t < 2; ++t) {
-            if (j >= w.np[t]) continue;
-            const int n = pn[t] + j;
-            if (n >= 2) mbar_wait(s_free(t, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);
+          if (j < np) {
+            const int n = pn + j;
+            if (n >= 2) mbar_wait(s_free(mt, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + t * 256 + (n & 1) * 64;
-            const uint32_t qa = qp + t * a.qp_bytes;
-            for (int k = 0; k < RK / 16; ++k) {
-              const int blk = k / kper, in = k - blk * kper;
-              umma_bf16(d_tmem, desc_at(d_kmaj_k, qa + blk * kRows * bk.span + in * 32),
-                        desc_at(d_kmaj_k, kaddr + blk * kPage * bk.span + in * 32), id_qk, k > 0 ? 1u : 0u);
-            }
-            umma_commit(s_full(t, n & 1));
+            const uint32_t d_tmem = t_s + (n & 1) * 64;
+            const uint64_t db = desc_at(d_kmaj_k, kaddr);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              if (k < nk) umma_bf16(d_tmem, dq + koff(k, lgk, qblk), db + koff(k, lgk, kblk), id_qk, k > 0 ? 1u : 0u);
+            umma_commit(s_full(mt, n & 1));
           }
           if (j > 0) issue_pv(j - 1, prev_v, prev_stage);
           prev_v = kaddr + kPage * RK * 2;
           prev_stage = stage;
         }
         issue_pv(npmax - 1, prev_v, prev_stage);
-        for (int t = 0; t < 2; ++t)
-          if (w.np[t] > 0) umma_commit(o_full(t));
+        if (active) umma_commit(o_full(mt));
         if (!fold_v) {
           // OUT = O_down U_v^T with O_down handed over as two bf16 terms (value, then residual): two accumulating
           // passes into the tile's score columns, which are idle by now
           uint32_t ua;
           int us;
           consume(ua, us);
-          for (int pass = 0; pass < 2; ++pass)
-            for (int t = 0; t < 2; ++t) {
-              if (w.np[t] == 0) continue;
-              mbar_wait(od_ready(t), pass, abort_flag, status);
+          if (active) {
+            const uint64_t db = desc_at(d_kmaj_v, ua);
+            for (int pass = 0; pass < 2; ++pass) {
+              mbar_wait(od_ready(mt), pass, abort_flag, status);
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + t * 256;
-              const uint32_t oa = qp + t * a.qp_bytes;
-              for (int k = 0; k < RV / 16; ++k) {
-                const int blk = k / vper, in = k - blk * vper;
-                umma_bf16(d_tmem, desc_at(d_kmaj_v, oa + blk * kRows * bv.span + in * 32),
-                          desc_at(d_kmaj_v, ua + blk * kD * bv.span + in * 32), id_bp, (pass > 0 || k > 0) ? 1u : 0u);
-              }
-              umma_commit(out_full(t));
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                if (k < nv) umma_bf16(t_s, dod + koff(k, lgv, oblk), db + koff(k, lgv, oblk), id_bp, (pass > 0 || k > 0) ? 1u : 0u);
+              umma_commit(out_full(mt));
             }
-          umma_commit(empty_bar(us));
+          }
+          release(us, active);
         }
-        for (int t = 0; t < 2; ++t) {
-          pn[t] += w.np[t];
-          kt[t] += w.np[t] > 0;
-        }
+        pn += np;
+        kt += active;
       }
     }
   } else {
@@ -391,7 +404,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t t_lane = tmem_base + ((uint32_t)(32 * q4) << 16) + t * 256;
     const uint32_t t_out = t_lane + 128;                        // Q' / O columns
     uint8_t* my_qp = qp_ptr + t * a.qp_bytes;
-    uint8_t* my_p = pb_ptr + t * kPBytes + row * 128;
+    uint8_t* my_p = pb_ptr + t * 2 * kPBytes + row * 128;           // this row in the tile's first P buffer
     const float c = kLog2e * rsqrtf((float)kD);                 // scores are scaled by 1/sqrt(d_h); exponent in base 2
     const int d_out = fold_v ? RV : kD;
     int kt = 0, pn = 0;
@@ -449,12 +462,11 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         float mx = s[0];
 #pragma unroll
         for (int i = 1; i < 64; ++i) mx = fmaxf(mx, s[i]);
-        // P_(n-1) has been consumed (and with it every earlier update of the accumulator is complete)
-        if (n >= 1) mbar_wait(p_free(t), (n - 1) & 1, abort_flag, status);
         if (j == 0) {
           m_ref = mx;                                           // position 0 is visible to every row: finite
           l = 0.f;
         } else if (__any_sync(0xffffffffu, (mx - m_ref) * c > kRescaleLog2)) {
+          mbar_wait(p_free(t, (n - 1) & 1), ((n - 1) >> 1) & 1, abort_flag, status);   // every earlier update of O is complete
           tc_fence_after();
           const float m_new = fmaxf(m_ref, mx);
           const float f = fast_exp2((m_ref - m_new) * c);
@@ -482,6 +494,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             *reinterpret_cast<uint4*>(vrows + (ch / cpr) * kPage * bv.span + r * bv.span + (ch % cpr) * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
         }
+        if (n >= 2) mbar_wait(p_free(t, sb), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2) has left this buffer
         const float neg = -m_ref * c;
         uint32_t pk[32];
 #pragma unroll
@@ -492,10 +505,10 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          *reinterpret_cast<uint4*>(my_p + ((k ^ (row & 7)) << 4)) = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+          *reinterpret_cast<uint4*>(my_p + sb * kPBytes + ((k ^ (row & 7)) << 4)) = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
         fence_proxy_async_smem();
         tc_fence_before();
-        arrive_warp(p_full(t));
+        arrive_warp(p_full(t, sb));
       }
 
       // ---- epilogue of the unit
@@ -648,10 +661,10 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
   a.out_lse = out_lse;
   a.status = status;
   a.qp_bytes = mq::kRows * 2 * (fold_v ? RK : (RK > RV ? RK : RV));
-  const int fixed = 1024 + 2 * a.qp_bytes + 2 * mq::kPBytes + mq::kCtrlBytes;
+  const int fixed = 1024 + 2 * a.qp_bytes + 4 * mq::kPBytes + mq::kCtrlBytes;
   a.nst = (mq::kSmemLimit - fixed) / mq::kStageBytes;
   if (a.nst > mq::kMaxStages) a.nst = mq::kMaxStages;
-  if (a.nst < 4) return STIEF_ERR_UNSUPPORTED;
+  if (a.nst < 3) return STIEF_ERR_UNSUPPORTED;       // two query tiles and U_k are in the ring together
   const int smem = fixed + a.nst * mq::kStageBytes;
 
   const long long n_units = (long long)((n_q + 2 * TT - 1) / (2 * TT)) * batch->B * layer->Hkv;
