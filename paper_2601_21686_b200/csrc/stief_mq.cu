@@ -266,8 +266,13 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // are a per-buffer base plus an offset that is a shift and a mask, and the K loops are unrolled.
     // Both threads walk ALL ring items in order; an item a thread has no use for is released with a plain arrive
     // once it has landed, so each stage always collects two arrivals.
-    if (lane == 0) {
-      const int mt = warp == 1 ? 0 : 1;
+    // The whole warp runs the role's control flow and address arithmetic (so the compiler can keep the descriptors in
+    // uniform registers, which is where tcgen05.mma takes them from); only the MMA, commit and arrive instructions
+    // themselves are predicated on the leader lane.
+    {
+      const bool leader = lane == 0;
+      const int mt = __shfl_sync(0xffffffffu, warp, 0) == 1 ? 0 : 1;
+      const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
       const uint32_t id_qk = idesc_bf16_f32(kRows, kPage);
       const uint32_t id_pv = idesc_bf16_f32_bmn(kRows, RV);
       const uint32_t id_pj = idesc_bf16_f32_bmn(kRows, RK);
@@ -287,7 +292,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const uint32_t pv_b = (uint32_t)(16 * bv.span) >> 4;                          // V page: 16 rows per K step
       const uint64_t dq = desc_at(d_kmaj_k, qp + mt * a.qp_bytes);                  // this tile's Q' operand
       const uint64_t dod = desc_at(d_kmaj_v, qp + mt * a.qp_bytes);                 // and its O_down operand (same region)
-      const uint32_t t_s = tmem_base + mt * 256, t_o = t_s + 128;                   // score buffers; Q' / O accumulator
+      const uint32_t t_s = tmem_u + mt * 256, t_o = t_s + 128;                   // score buffers; Q' / O accumulator
       int st = 0, use = 0;
       int kt = 0, pn = 0;
       auto consume = [&](uint32_t& addr, int& stage) {          // next item of the ring, once it has landed
@@ -300,8 +305,10 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
       };
       auto release = [&](int stage, bool used) {                // after the MMAs that read it, or at once when unused
-        if (used) umma_commit(empty_bar(stage));
-        else mbar_arrive(empty_bar(stage));
+        if (leader) {
+          if (used) umma_commit(empty_bar(stage));
+          else mbar_arrive(empty_bar(stage));
+        }
       };
       for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const Unit w = decode_unit(a, u, TT);
@@ -327,9 +334,9 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const uint64_t da = desc_at(d_sw128, qa), db = desc_at(d_uk, ua);
 #pragma unroll
             for (int k = 0; k < kD / 16; ++k)
-              umma_bf16(t_o, da + (uint32_t)(((k >> 2) * (kStageBytes / 2) + (k & 3) * 32) >> 4), db + (uint32_t)(k * bk.span),
+              if (leader) umma_bf16(t_o, da + (uint32_t)(((k >> 2) * (kStageBytes / 2) + (k & 3) * 32) >> 4), db + (uint32_t)(k * bk.span),
                         id_pj, k > 0 ? 1u : 0u);
-            umma_commit(qacc_full(mt));
+            if (leader) umma_commit(qacc_full(mt));
             release(qs, true);
           }
           release(us, active);
@@ -347,8 +354,8 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const uint64_t da = desc_at(d_sw128, pb + (mt * 2 + (n & 1)) * kPBytes), db = desc_at(d_vpage, vaddr);
 #pragma unroll
             for (int k = 0; k < kPage / 16; ++k)
-              umma_bf16(t_o, da + (uint32_t)(2 * k), db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
-            umma_commit(p_free(mt, n & 1));
+              if (leader) umma_bf16(t_o, da + (uint32_t)(2 * k), db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
+            if (leader) umma_commit(p_free(mt, n & 1));
           }
           release(stage, jj < np);                              // K and V of this page are no longer needed by this tile
         };
@@ -364,15 +371,15 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const uint64_t db = desc_at(d_kmaj_k, kaddr);
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-              if (k < nk) umma_bf16(d_tmem, dq + koff(k, lgk, qblk), db + koff(k, lgk, kblk), id_qk, k > 0 ? 1u : 0u);
-            umma_commit(s_full(mt, n & 1));
+              if (k < nk && leader) umma_bf16(d_tmem, dq + koff(k, lgk, qblk), db + koff(k, lgk, kblk), id_qk, k > 0 ? 1u : 0u);
+            if (leader) umma_commit(s_full(mt, n & 1));
           }
           if (j > 0) issue_pv(j - 1, prev_v, prev_stage);
           prev_v = kaddr + kPage * RK * 2;
           prev_stage = stage;
         }
         issue_pv(npmax - 1, prev_v, prev_stage);
-        if (active) umma_commit(o_full(mt));
+        if (active && leader) umma_commit(o_full(mt));
         if (!fold_v) {
           // OUT = O_down U_v^T with O_down handed over as two bf16 terms (value, then residual): two accumulating
           // passes into the tile's score columns, which are idle by now
@@ -386,8 +393,8 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
               tc_fence_after();
 #pragma unroll
               for (int k = 0; k < 8; ++k)
-                if (k < nv) umma_bf16(t_s, dod + koff(k, lgv, oblk), db + koff(k, lgv, oblk), id_bp, (pass > 0 || k > 0) ? 1u : 0u);
-              umma_commit(out_full(mt));
+                if (k < nv && leader) umma_bf16(t_s, dod + koff(k, lgv, oblk), db + koff(k, lgv, oblk), id_bp, (pass > 0 || k > 0) ? 1u : 0u);
+              if (leader) umma_commit(out_full(mt));
             }
           }
           release(us, active);
