@@ -312,18 +312,21 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       };
       for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
         const Unit w = decode_unit(a, u, TT);
-        if (!w.valid) continue;
-        const int np = mt ? w.np[1] : w.np[0], np_other = mt ? w.np[0] : w.np[1];
+        // the unit's shape comes from global loads; broadcasting it from lane 0 tells the compiler that the control
+        // flow and the addresses below are the same in every lane
+        if (!__shfl_sync(0xffffffffu, (int)w.valid, 0)) continue;
+        const int wnp0 = __shfl_sync(0xffffffffu, w.np[0], 0), wnp1 = __shfl_sync(0xffffffffu, w.np[1], 0);
+        const int np = mt ? wnp1 : wnp0, np_other = mt ? wnp0 : wnp1;
         const int npmax = max(np, np_other);
         const bool active = np > 0;
         if (!fold_k) {
           uint32_t qa = 0, ua, tmp;
           int qs = -1, us, ts;
-          if (w.np[0] > 0) {                                    // tile 0's raw queries
+          if (wnp0 > 0) {                                       // tile 0's raw queries
             if (mt == 0) consume(qa, qs);
             else { consume(tmp, ts); release(ts, false); }
           }
-          if (w.np[1] > 0) {                                    // tile 1's
+          if (wnp1 > 0) {                                       // tile 1's
             if (mt == 1) consume(qa, qs);
             else { consume(tmp, ts); release(ts, false); }
           }
