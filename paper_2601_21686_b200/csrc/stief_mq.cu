@@ -104,6 +104,29 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int u, int TT) {
   return w;
 }
 
+// packed fp32 pairs (sm_100): one instruction for two lanes of arithmetic
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // 16 fp32 values of a row -> 8 packed bf16 words
 __device__ __forceinline__ void pack16(const uint32_t (&v)[16], float scale, uint32_t (&w)[8]) {
 #pragma unroll
@@ -469,9 +492,13 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int i = 0; i < 64; ++i)
             if (p0 + i > q_pos) s[i] = -INFINITY;
         }
-        float mx = s[0];
+        float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);     // two chains of three-input maxima
 #pragma unroll
-        for (int i = 1; i < 64; ++i) mx = fmaxf(mx, s[i]);
+        for (int i = 6; i < 62; i += 4) {
+          mx0 = max3(mx0, s[i], s[i + 1]);
+          mx1 = max3(mx1, s[i + 2], s[i + 3]);
+        }
+        const float mx = fmaxf(max3(mx0, s[62], s[63]), mx1);
         if (j == 0) {
           m_ref = mx;                                           // position 0 is visible to every row: finite
           l = 0.f;
@@ -505,13 +532,21 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
         }
         if (n >= 2) mbar_wait(p_free(t, sb), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2) has left this buffer
-        const float neg = -m_ref * c;
+        const uint64_t c2 = pack2(c, c), neg2 = pack2(-m_ref * c, -m_ref * c);
+        uint64_t sum2 = pack2(0.f, 0.f);
         uint32_t pk[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float e0 = fast_exp2(fmaf(s[2 * i], c, neg)), e1 = fast_exp2(fmaf(s[2 * i + 1], c, neg));
-          l += e0 + e1;
+          float x0, x1;
+          unpack2(fma2(pack2(s[2 * i], s[2 * i + 1]), c2, neg2), x0, x1);
+          const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
+          sum2 = add2(sum2, pack2(e0, e1));
           pk[i] = pack_bf16(e0, e1);
+        }
+        {
+          float a0, a1;
+          unpack2(sum2, a0, a1);
+          l += a0 + a1;
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k)
