@@ -36,6 +36,8 @@ def _units():
     for rk in KEY_RANKS:
         units.append((os.path.join(CSRC, "stief_decode_inst.cu"), os.path.join(OBJ, f"stief_decode_rk{rk}.o"),
                       [f"-DSTIEF_RK={rk}"]))
+        units.append((os.path.join(CSRC, "stief_mq_inst.cu"), os.path.join(OBJ, f"stief_mq_rk{rk}.o"),
+                      [f"-DSTIEF_RK={rk}"]))
     return units
 
 
