@@ -108,6 +108,20 @@ int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, c
 int stief_append(const stief_layer* layer, const stief_batch* batch, const uint16_t* k_new,
                  const uint16_t* v_new, int32_t* status, void* stream);
 
+/* Eq. 1 for a run of new tokens per sequence (the cache-write half of chunked prefill, App. A.1: a later chunk of the
+ * prompt is projected and stored behind what is cached already).  K, V are device bf16 [B][T_chunk][Hkv][128]
+ * (r elements per head on a side without basis) with element strides as in stief_prefill_compress; chunk_lens is a
+ * device int32 [B] (rows of each sequence that are real, clamped to 0 .. T_chunk) or NULL = T_chunk for all.
+ *   ends_at_len = 0: row i is stored at position seq_lens[b] + i (like stief_append; advance seq_lens afterwards);
+ *   ends_at_len = 1: seq_lens already counts the chunk: row i is stored at seq_lens[b] - chunk_len_b + i, the
+ *                    convention of stief_mq_attention, which can follow on the same stream with the same lengths.
+ * The pages of every written position must be assigned in block_table; a position outside it sets STIEF_ERR_BOUNDS.
+ * Each row gets the same bits as stief_append would give it.  The whole-prompt path stays stief_prefill_compress
+ * (tensor cores, HBM-bound); this one is for chunks, where the projection is a small part of the step. */
+int stief_append_chunk(const stief_layer* layer, const stief_batch* batch, const uint16_t* K, const uint16_t* V,
+                       int64_t stride_b, int64_t stride_t, int64_t v_stride_b, int64_t v_stride_t, int32_t T_chunk,
+                       const int32_t* chunk_lens, int32_t ends_at_len, int32_t* status, void* stream);
+
 /* Split-T planning.  The page tiles of the whole batch (one tile = 64 tokens of one KV head) are laid
  * end to end -- units (sequence, KV head, tile of up to 8 query heads) in that order -- and cut into
  * num_parts contiguous ranges of equal cost, one per CTA of a persistent kernel (cost = page tiles,

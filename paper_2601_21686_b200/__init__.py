@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         sig = {
             "stief_prefill_compress": (ctypes.c_int, [LP, BP, P, P, I64, I64, I64, I64, I32, U32, P, P]),
             "stief_append": (ctypes.c_int, [LP, BP, P, P, P, P]),
+            "stief_append_chunk": (ctypes.c_int, [LP, BP, P, P, I64, I64, I64, I64, I32, P, I32, P, P]),
             "stief_decode_num_parts": (I32, []),
             "stief_decode_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
             "stief_decode_workspace_init": (ctypes.c_int, [P, SZ, P]),
@@ -370,3 +371,16 @@ def stief_mq_attention(layer: Layer, batch: Batch, q: torch.Tensor, out: torch.T
     _check(lib().stief_mq_attention(ctypes.byref(layer.c()), ctypes.byref(batch.c()), _ptr(q), q.stride(0), q.stride(1),
                                     q.shape[1], _ptr(q_lens), _ptr(out), out.stride(0), out.stride(1), _ptr(out_lse),
                                     flags, _ptr(status), _stream()), "stief_mq_attention")
+
+
+def stief_append_chunk(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Tensor, chunk_lens: Optional[torch.Tensor] = None,
+                       ends_at_len: bool = False, status: Optional[torch.Tensor] = None):
+    """K, V [B, T_chunk, Hkv, 128 (or r on a side without basis)] bf16: project and store a run of new tokens per sequence,
+    starting at seq_lens[b] (default) or ending at seq_lens[b] - 1 (``ends_at_len``)."""
+    assert K.dtype == torch.bfloat16 and V.dtype == torch.bfloat16 and K.dim() == 4 and V.dim() == 4
+    assert K.stride(3) == 1 and K.stride(2) == K.shape[3] and V.stride(3) == 1 and V.stride(2) == V.shape[3]
+    assert K.shape[3] == (D_HEAD if layer.U_k is not None else layer.r_k) and V.shape[3] == (D_HEAD if layer.U_v is not None else layer.r_v)
+    assert K.shape[:3] == V.shape[:3]
+    _check(lib().stief_append_chunk(ctypes.byref(layer.c()), ctypes.byref(batch.c()), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
+                                    V.stride(0), V.stride(1), K.shape[1], _ptr(chunk_lens), 1 if ends_at_len else 0,
+                                    _ptr(status), _stream()), "stief_append_chunk")

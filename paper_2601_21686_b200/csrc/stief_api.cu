@@ -241,6 +241,31 @@ int stief_append(const stief_layer* layer, const stief_batch* batch, const uint1
   return launch_append(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
+int stief_append_chunk(const stief_layer* layer, const stief_batch* batch, const uint16_t* K, const uint16_t* V,
+                       int64_t stride_b, int64_t stride_t, int64_t v_stride_b, int64_t v_stride_t, int32_t T_chunk,
+                       const int32_t* chunk_lens, int32_t ends_at_len, int32_t* status, void* stream) {
+  int rc = check_layer(layer);
+  if (rc) return rc;
+  rc = check_batch(batch);
+  if (rc) return rc;
+  if (!K || !V || !aligned(K, 16) || !aligned(V, 16) || T_chunk <= 0 || T_chunk > 65535 * 8) return STIEF_ERR_INVALID_ARG;
+  const long long dk = layer->U_k ? kD : layer->r_k, dv = layer->U_v ? kD : layer->r_v;
+  if (stride_t < dk * layer->Hkv || stride_b < stride_t || stride_t % 8 || stride_b % 8 || v_stride_t < dv * layer->Hkv ||
+      v_stride_b < v_stride_t || v_stride_t % 8 || v_stride_b % 8)
+    return STIEF_ERR_INVALID_ARG;
+  if ((long long)batch->B * 2 > 65535) return STIEF_ERR_INVALID_ARG;
+  AppendChunkArgs a;
+  a.L = to_dev(layer); a.Bt = host::to_dev(batch);
+  a.K = reinterpret_cast<const __nv_bfloat16*>(K);
+  a.V = reinterpret_cast<const __nv_bfloat16*>(V);
+  a.k_stride_b = stride_b; a.k_stride_t = stride_t; a.v_stride_b = v_stride_b; a.v_stride_t = v_stride_t;
+  a.T_chunk = T_chunk;
+  a.chunk_lens = chunk_lens;
+  a.ends_at_len = ends_at_len ? 1 : 0;
+  a.status = status;
+  return launch_append_chunk(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
+
 int32_t stief_decode_num_parts(void) { return sm_count(); }
 
 size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t r_v, int32_t num_parts) {

@@ -13,6 +13,18 @@ struct AppendArgs {
   int32_t* status;
 };
 
+struct AppendChunkArgs {
+  LayerDev L;
+  BatchDev Bt;
+  const __nv_bfloat16* K;       // [B][T_chunk][Hkv][128 or r_k]
+  const __nv_bfloat16* V;
+  long long k_stride_b, k_stride_t, v_stride_b, v_stride_t;   // elements
+  int T_chunk;
+  const int32_t* chunk_lens;    // [B] or NULL = T_chunk
+  int ends_at_len;              // 1: the chunk's last row is position seq_lens[b] - 1; 0: its first row is position seq_lens[b]
+  int32_t* status;
+};
+
 struct CombineArgs {
   LayerDev L;
   BatchDev Bt;
@@ -42,6 +54,7 @@ struct DecodeLaunch {
 };
 
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+cudaError_t launch_append_chunk(const AppendChunkArgs& a, cudaStream_t st);
 cudaError_t launch_combine(const CombineArgs& a, cudaStream_t st);
 cudaError_t launch_advance(int32_t* seq_lens, int B, int delta, cudaStream_t st);
 cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st);

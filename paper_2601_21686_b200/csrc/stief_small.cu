@@ -74,6 +74,58 @@ append_kernel(const AppendArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// append_chunk_kernel: the same projection for a run of new tokens per sequence (the cache-write half of chunked
+// prefill).  A block takes kChunkTok consecutive tokens of one (sequence, KV head, side); the basis stays in L1
+// across them.  The work is tiny next to the attention that follows (128 r MACs per row), so it stays on the FMA
+// pipe with the accumulation order of the single-token kernel: a token appended alone or inside a chunk gets the
+// same bits.
+// ---------------------------------------------------------------------------------------------
+constexpr int kChunkTok = 8;
+
+__global__ void __launch_bounds__(kAppThreads)
+append_chunk_kernel(const AppendChunkArgs a) {
+  __shared__ float x[kD];
+  __shared__ float red[8 * kD];
+  const int h = blockIdx.x, tile = blockIdx.y, b = blockIdx.z >> 1, which = blockIdx.z & 1;
+  int len = a.chunk_lens ? a.chunk_lens[b] : a.T_chunk;
+  len = min(max(len, 0), a.T_chunk);
+  const int t0 = tile * kChunkTok;
+  if (t0 >= len) return;
+  const int sl = a.Bt.seq_lens[b];
+  const int pos0 = a.ends_at_len ? sl - len : sl;          // position of the chunk's row 0
+  if (pos0 < 0 || sl < 0) {
+    if (threadIdx.x == 0) report(a.status, STIEF_ERR_BOUNDS);
+    return;
+  }
+  const __nv_bfloat16* Ub = which ? a.L.U_v : a.L.U_k;
+  const __nv_bfloat16* U = Ub ? Ub + (size_t)h * (which ? a.L.uv_stride : a.L.uk_stride) : nullptr;
+  const int R = which ? a.L.r_v : a.L.r_k;
+  const int d_in = U ? kD : R;
+  const __nv_bfloat16* X = which ? a.V : a.K;
+  const long long sb = which ? a.v_stride_b : a.k_stride_b, stt = which ? a.v_stride_t : a.k_stride_t;
+  for (int t = t0; t < min(t0 + kChunkTok, len); ++t) {
+    const int pos = pos0 + t, pi = pos / kPage;
+    int page = -1;
+    if (pi < a.Bt.max_pages) page = a.Bt.block_table[(size_t)b * a.Bt.max_pages + pi];
+    if (page < 0 || page >= a.L.num_pages) {              // uniform over the block
+      if (threadIdx.x == 0) report(a.status, STIEF_ERR_BOUNDS);
+      return;
+    }
+    const __nv_bfloat16* src = X + (size_t)b * sb + (size_t)t * stt + (size_t)h * d_in;
+    __nv_bfloat16* dst = (which ? a.L.v_pool : a.L.k_pool) + (((size_t)page * a.L.Hkv + h) * kPage + (pos % kPage)) * R;
+    __syncthreads();                                       // the previous token's results have been read
+    if (threadIdx.x < d_in) x[threadIdx.x] = __bfloat162float(src[threadIdx.x]);
+    __syncthreads();
+    const float* res = x;
+    if (U) {
+      project_row(x, U, R, red);
+      res = red;
+    }
+    for (int j = threadIdx.x; j < R; j += kAppThreads) dst[j] = __float2bfloat16_rn(res[j]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // combine_kernel
 // ---------------------------------------------------------------------------------------------
 constexpr int kCombThreads = 128;
@@ -116,6 +168,10 @@ __global__ void advance_kernel(int32_t* seq_lens, int B, int delta) {
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st) {
   append_kernel<<<dim3(a.L.Hkv, a.Bt.B, 2), kAppThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+cudaError_t launch_append_chunk(const AppendChunkArgs& a, cudaStream_t st) {
+  append_chunk_kernel<<<dim3(a.L.Hkv, (a.T_chunk + kChunkTok - 1) / kChunkTok, a.Bt.B * 2), kAppThreads, 0, st>>>(a);
   return cudaGetLastError();
 }
 cudaError_t launch_combine(const CombineArgs& a, cudaStream_t st) {

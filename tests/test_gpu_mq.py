@@ -186,3 +186,76 @@ def test_unsupported_group_size_and_bad_arguments():
     with pytest.raises(S.StiefError) as e:
         S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, flags=4)
     assert e.value.code == S.STIEF_ERR_INVALID_ARG
+
+
+def test_chunked_prefill_end_to_end():
+    # A prompt processed in chunks of 96 tokens: every chunk is projected and stored behind the cache (stief_append_chunk),
+    # then attends causally to everything cached so far (stief_mq_attention).  All rows together are plain causal
+    # attention of the whole prompt; the cache must equal the oracle's projection of the whole prompt.
+    B, Hq, Hkv, r_k, r_v, chunk = 2, 8, 2, 64, 96, 96
+    final = np.array([300, 170], dtype=np.int32)
+    c = U.make_case(321, B, Hq, Hkv, r_k, r_v, final, lowrank=True)
+    T = int(final.max())
+    q = _queries(12, B, T, Hq)
+    c.batch.seq_lens.zero_()
+    outs = torch.full((B, T, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    Kd, Vd, qd = c.K.to(DEV), c.V.to(DEV), q.to(DEV)
+    done = np.zeros(B, dtype=np.int32)
+    step = 0
+    while (done < final).any():
+        lens = np.minimum(chunk, final - done).astype(np.int32)
+        lens_d = torch.from_numpy(lens).to(DEV)
+        # gather each sequence's next rows into a [B, chunk] batch (rows beyond lens are never read into the cache)
+        Kc = torch.zeros(B, chunk, Hkv, 128, dtype=torch.bfloat16, device=DEV)
+        Vc, qc = torch.zeros_like(Kc), torch.zeros(B, chunk, Hq, 128, dtype=torch.bfloat16, device=DEV)
+        for b in range(B):
+            n = int(lens[b])
+            Kc[b, :n], Vc[b, :n], qc[b, :n] = Kd[b, done[b]:done[b] + n], Vd[b, done[b]:done[b] + n], qd[b, done[b]:done[b] + n]
+        oc = torch.full((B, chunk, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+        if step % 2 == 0:      # both position conventions
+            S.stief_append_chunk(c.layer, c.batch, Kc, Vc, chunk_lens=lens_d, status=c.status)
+            c.batch.seq_lens += lens_d
+        else:
+            c.batch.seq_lens += lens_d
+            S.stief_append_chunk(c.layer, c.batch, Kc, Vc, chunk_lens=lens_d, ends_at_len=True, status=c.status)
+        S.stief_mq_attention(c.layer, c.batch, qc, oc, q_lens=lens_d, status=c.status)
+        torch.cuda.synchronize()
+        assert int(c.status.item()) == 0
+        for b in range(B):
+            n = int(lens[b])
+            outs[b, done[b]:done[b] + n] = oc[b, :n]
+            assert torch.isnan(oc[b, n:]).all()
+        done += lens
+        step += 1
+    assert np.array_equal(c.batch.seq_lens.cpu().numpy(), final)
+    Kd_o, Vd_o = U.oracle_cache(c)
+    for b in range(B):
+        n = int(final[b])
+        gk, gv = U.gpu_cache_rows(c, c.layer.k_pool, b, n), U.gpu_cache_rows(c, c.layer.v_pool, b, n)
+        for h in range(Hkv):
+            U.check_cache(gk[:, h], U.f64(c.K)[b, :n, h], U.f64(c.U_k)[h], Kd_o[b][:, h])
+            U.check_cache(gv[:, h], U.f64(c.V)[b, :n, h], U.f64(c.U_v)[h], Vd_o[b][:, h])
+    ref, _ = _reference(c, q, final)
+    _compare(outs, None, ref, None)
+
+
+def test_chunk_rows_have_the_bits_of_single_token_append():
+    c1 = U.make_case(55, 2, 4, 2, 48, 128, [70, 3], full_rank_v=True)
+    c2 = U.make_case(55, 2, 4, 2, 48, 128, [70, 3], full_rank_v=True)
+    n_new = 5
+    Kn = I.gaussian_kv(8, I.TAG_K, 3, 2, n_new, 2)
+    Vn = I.gaussian_kv(8, I.TAG_V, 3, 2, n_new, 2)
+    S.stief_append_chunk(c1.layer, c1.batch, Kn.to(DEV), Vn.to(DEV), status=c1.status)
+    for i in range(n_new):
+        S.stief_append(c2.layer, c2.batch, Kn[:, i].contiguous().to(DEV), Vn[:, i].contiguous().to(DEV), status=c2.status)
+        S.stief_advance_seq_lens(c2.batch.seq_lens, 1)
+    torch.cuda.synchronize()
+    assert int(c1.status.item()) == 0 and int(c2.status.item()) == 0
+    assert torch.equal(c1.layer.k_pool.view(torch.int16), c2.layer.k_pool.view(torch.int16))
+    assert torch.equal(c1.layer.v_pool.view(torch.int16), c2.layer.v_pool.view(torch.int16))
+    # positions without a page are reported, not written
+    c3 = U.make_case(56, 1, 4, 2, 64, 64, [60], reserve=2)
+    big = I.gaussian_kv(9, I.TAG_K, 3, 1, 200, 2)
+    S.stief_append_chunk(c3.layer, c3.batch, big.to(DEV), big.to(DEV), status=c3.status)
+    torch.cuda.synchronize()
+    assert int(c3.status.item()) == S.STIEF_ERR_BOUNDS
