@@ -464,12 +464,14 @@ def run_mq(args):
         layers.append(layer)
     qs = [I.normal_bf16(I.stream_key(SEED, I.TAG_Q, 100 + i), (B, n_q, Hq, 128), device=dev) for i in range(2)]
     out = torch.empty(B, n_q, Hq, 128, dtype=torch.bfloat16, device=dev)
+    n_split = S.stief_mq_num_splits(B, n_q, Hq, Hkv, batch.block_table.shape[1]) if args.splits is None else args.splits
+    ws = torch.empty(max(S.stief_mq_workspace_bytes(B, n_q, Hq, r_v, n_split) // 4, 1), dtype=torch.float32, device=dev) if n_split > 1 else None
     torch.cuda.synchronize()
 
     def step(i):
-        S.stief_mq_attention(layers[i % n_caches], batch, qs[i % 2], out, status=status)
+        S.stief_mq_attention(layers[i % n_caches], batch, qs[i % 2], out, status=status, workspace=ws, num_splits=n_split)
 
-    K_steps, W = min(args.steps, 50), max(min(args.warmup, 5), 3)
+    K_steps, W = min(args.steps, 50 if n_q >= 256 else 2000), max(min(args.warmup, 5), 3)
     sampler = ClockSampler(0)
     sampler.start()
     time.sleep(0.3)
@@ -496,9 +498,11 @@ def run_mq(args):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "dtype_note": "bf16 tensor-core operands (tcgen05), fp32 accumulate in TMEM", "data": "synthetic",
         "config": {"workload": f"chunk of {n_q} causal query tokens per sequence at the end of a {T}-token compressed cache, "
-                               f"B={B} Hq={Hq} Hkv={Hkv} r_k={r_k} r_v={r_v}: query projection + causal attention + back-projection, one launch",
+                               f"B={B} Hq={Hq} Hkv={Hkv} r_k={r_k} r_v={r_v}: query projection + causal attention + back-projection"
+                               + (f", page ranges split {n_split} ways + merge kernel" if n_split > 1 else ", one launch"),
                    "l2": f"steps alternate over {n_caches} layer caches of {cache_bytes / 2**20:.0f} MiB"},
-        "query_tokens_per_s": B * n_q / (ms * 1e-3), "gpu_launches": K_steps,
+        "query_tokens_per_s": B * n_q / (ms * 1e-3), "gpu_launches": K_steps * (2 if n_split > 1 else 1),
+        "cache_read_gbs": cache_bytes / (ms * 1e-3) / 1e9, "cache_read_frac_of_hbm_peak": cache_bytes / (ms * 1e-3) / 1e9 / hbm_peak,
         "roofline": {"bound": "tensor", "kernel": "mq_attention_kernel", "achieved": tflops, "peak": tf_peak, "unit": "TFLOP/s",
                      "frac": tflops / tf_peak, "peak_kind": peak_kind, "traffic": None, "flops_per_launch": flops,
                      "avg_launch_ms": ms},
@@ -761,6 +765,7 @@ def main():
     # summarised in profiles/decode_persistent_kernel_config2.md (mean of two launches); null for other workloads
     ap.add_argument("--mq", action="store_true", help="measure the multi-query (chunked prefill) attention kernel on the config-2 shape")
     ap.add_argument("--n-q", dest="n_q", type=int, default=2048, help="query tokens per sequence for --mq")
+    ap.add_argument("--splits", type=int, default=None, help="--mq: parts per page range (default: the library's proposal)")
     ap.add_argument("--rho", type=float, default=None, help="multi-layer workloads: take the per-layer ranks from stief_select_ranks at this cache ratio instead of the seeded random profile")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
     args = ap.parse_args()

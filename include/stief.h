@@ -303,12 +303,23 @@ int stief_time_next_decode_kernel(void* start_event, void* stop_event);
  *   out      device, bf16 [B][n_q][Hq][d_out], strides as for q; d_out = 128, or r_v when U_v is NULL (folded values:
  *            the compressed output is returned for a folded output projection)
  *   out_lse  optional device fp32 [B][n_q][Hq] (contiguous): natural-log-sum-exp of each row's scaled scores
+ *   workspace, workspace_bytes, num_splits
+ *            With few query rows and a long cache (speculative decode) the (sequence, KV head, 256-row) work units are too
+ *            few to fill the GPU.  num_splits > 1 cuts every unit's page range into that many parts, which run as units of
+ *            their own and leave partial results in `workspace` (device, 128-byte aligned, at least
+ *            stief_mq_workspace_bytes(...) bytes, contents irrelevant on entry); a second small kernel merges them
+ *            (log-sum-exp), normalises and back-projects.  num_splits = 1: no workspace (NULL, 0).  stief_mq_num_splits
+ *            proposes a value: 1 when the units already fill the GPU, else about SMs / units, at most 64 and at most a
+ *            quarter of max_pages_per_seq.  Too small a workspace: STIEF_ERR_WORKSPACE, nothing is launched.
  *   flags    must be 0
  * All ranks 32/48/64/96/128; Hq / Hkv must divide 128 (a 128-row tile holds whole tokens), else
- * STIEF_ERR_UNSUPPORTED.  No workspace; nothing is allocated.  Asynchronous on `stream`. */
+ * STIEF_ERR_UNSUPPORTED.  Nothing is allocated.  Asynchronous on `stream`. */
+int32_t stief_mq_num_splits(int32_t B, int32_t n_q, int32_t Hq, int32_t Hkv, int32_t max_pages_per_seq);
+size_t stief_mq_workspace_bytes(int32_t B, int32_t n_q, int32_t Hq, int32_t r_v, int32_t num_splits);
 int stief_mq_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int64_t q_stride_b,
-                       int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, uint16_t* out, int64_t out_stride_b,
-                       int64_t out_stride_t, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+                       int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, void* workspace, size_t workspace_bytes,
+                       int32_t num_splits, uint16_t* out, int64_t out_stride_b, int64_t out_stride_t, float* out_lse,
+                       uint32_t flags, int32_t* status, void* stream);
 
 /* ---- rank selection (host only) --------------------------------------------------------------------------
  * Sequential budgeted rank selection, Algorithm 2 of the paper (Sec. 3.4, Eq. 15-17; cost c = (r_K + r_V) / (2 d_h),

@@ -88,7 +88,9 @@ def lib() -> ctypes.CDLL:
             "stief_q8_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
             "stief_q8_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
             "stief_q8_decode_step": (ctypes.c_int, [QP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
-            "stief_mq_attention": (ctypes.c_int, [LP, BP, P, I64, I64, I32, P, P, I64, I64, P, U32, P, P]),
+            "stief_mq_attention": (ctypes.c_int, [LP, BP, P, I64, I64, I32, P, P, SZ, I32, P, I64, I64, P, U32, P, P]),
+            "stief_mq_num_splits": (I32, [I32, I32, I32, I32, I32]),
+            "stief_mq_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
             "stief_select_ranks": (ctypes.c_int, [I32, I32, P, I32, P, I32, ctypes.c_double, P, _SURFACE_FN, P, P, P, P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
@@ -358,19 +360,30 @@ def stief_select_ranks(L: int, cand_k: Sequence[int], cand_v: Sequence[int], rho
     return [(rk[l], rv[l]) for l in range(L)], spent.value
 
 
+def stief_mq_num_splits(B: int, n_q: int, Hq: int, Hkv: int, max_pages_per_seq: int) -> int:
+    return lib().stief_mq_num_splits(B, n_q, Hq, Hkv, max_pages_per_seq)
+
+
+def stief_mq_workspace_bytes(B: int, n_q: int, Hq: int, r_v: int, num_splits: int) -> int:
+    return lib().stief_mq_workspace_bytes(B, n_q, Hq, r_v, num_splits)
+
+
 def stief_mq_attention(layer: Layer, batch: Batch, q: torch.Tensor, out: torch.Tensor, q_lens: Optional[torch.Tensor] = None,
-                       out_lse: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, flags: int = 0):
+                       out_lse: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, flags: int = 0,
+                       workspace: Optional[torch.Tensor] = None, num_splits: int = 1):
     """Several causal query rows per head: q [B, n_q, Hq, d_q] bf16 -> out [B, n_q, Hq, d_out] bf16 (strides over b and
-    t free).  The queries are the last q_lens[b] (default n_q) tokens of each cached sequence."""
+    t free).  The queries are the last q_lens[b] (default n_q) tokens of each cached sequence.  num_splits > 1 needs a
+    workspace tensor of stief_mq_workspace_bytes(...) bytes."""
     assert q.dtype == torch.bfloat16 and out.dtype == torch.bfloat16 and q.dim() == 4 and out.dim() == 4
     assert q.stride(3) == 1 and q.stride(2) == q.shape[3] and out.stride(3) == 1 and out.stride(2) == out.shape[3]
     assert q.shape[3] == (D_HEAD if layer.U_k is not None else layer.r_k)
     assert out.shape[3] == (D_HEAD if layer.U_v is not None else layer.r_v) and out.shape[:3] == q.shape[:3]
     if out_lse is not None:
         assert out_lse.dtype == torch.float32 and out_lse.is_contiguous() and tuple(out_lse.shape) == tuple(q.shape[:3])
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().stief_mq_attention(ctypes.byref(layer.c()), ctypes.byref(batch.c()), _ptr(q), q.stride(0), q.stride(1),
-                                    q.shape[1], _ptr(q_lens), _ptr(out), out.stride(0), out.stride(1), _ptr(out_lse),
-                                    flags, _ptr(status), _stream()), "stief_mq_attention")
+                                    q.shape[1], _ptr(q_lens), _ptr(workspace), ws_bytes, num_splits, _ptr(out), out.stride(0),
+                                    out.stride(1), _ptr(out_lse), flags, _ptr(status), _stream()), "stief_mq_attention")
 
 
 def stief_append_chunk(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Tensor, chunk_lens: Optional[torch.Tensor] = None,

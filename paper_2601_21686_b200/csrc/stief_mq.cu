@@ -19,11 +19,42 @@ bool rank_ok(int r) { return r == 32 || r == 48 || r == 64 || r == 96 || r == 12
 
 using namespace stief;
 
+namespace stief {
+cudaError_t launch_mq_combine(const mq::Args& a, cudaStream_t st) {
+  mq::mq_combine_kernel<0><<<dim3(a.n_q, a.L.Hkv, a.Bt.B), mq::kCombineThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+}  // namespace stief
+
+extern "C" int32_t stief_mq_num_splits(int32_t B, int32_t n_q, int32_t Hq, int32_t Hkv, int32_t max_pages_per_seq) {
+  if (B <= 0 || n_q <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || max_pages_per_seq <= 0) return 0;
+  const int G = Hq / Hkv;
+  if (G > mq::kRows || mq::kRows % G != 0) return 0;
+  const int TT = mq::kRows / G;
+  const long long base = (long long)((n_q + 2 * TT - 1) / (2 * TT)) * B * Hkv;      // units without splitting
+  long long s = host::sm_count() / base;                                           // parts so that the units about fill the GPU
+  if (s > 64) s = 64;
+  if (s > max_pages_per_seq / 4) s = max_pages_per_seq / 4;                        // at least a few pages per part
+  return (int32_t)(s < 1 ? 1 : s);
+}
+
+extern "C" size_t stief_mq_workspace_bytes(int32_t B, int32_t n_q, int32_t Hq, int32_t r_v, int32_t num_splits) {
+  if (B <= 0 || n_q <= 0 || Hq <= 0 || r_v <= 0 || num_splits < 1) return 0;
+  if (num_splits == 1) return 0;
+  return host::align_up((size_t)B * n_q * Hq * num_splits * (r_v + 2) * sizeof(float), 128);
+}
+
 extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int64_t q_stride_b,
-                                  int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, uint16_t* out,
-                                  int64_t out_stride_b, int64_t out_stride_t, float* out_lse, uint32_t flags,
-                                  int32_t* status, void* stream) {
-  if (!layer || !q || !out || flags != 0u) return STIEF_ERR_INVALID_ARG;
+                                  int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, void* workspace,
+                                  size_t workspace_bytes, int32_t num_splits, uint16_t* out, int64_t out_stride_b,
+                                  int64_t out_stride_t, float* out_lse, uint32_t flags, int32_t* status, void* stream) {
+  if (!layer || !q || !out || flags != 0u || num_splits < 1 || num_splits > 64) return STIEF_ERR_INVALID_ARG;
+  if (num_splits > 1) {
+    if (!workspace || !host::aligned(workspace, 128)) return STIEF_ERR_INVALID_ARG;
+    if (workspace_bytes < stief_mq_workspace_bytes(batch ? batch->B : 0, n_q, layer->Hq, layer->r_v, num_splits) ||
+        n_q > 65535 || (batch && batch->B > 65535))
+      return STIEF_ERR_WORKSPACE;
+  }
   const int rc = host::check_batch(batch);
   if (rc != STIEF_OK) return rc;
   if (layer->Hq <= 0 || layer->Hkv <= 0 || layer->Hq % layer->Hkv != 0 || layer->num_pages <= 0 || !layer->k_pool || !layer->v_pool ||
@@ -85,13 +116,16 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
   a.out_stride_t = out_stride_t;
   a.out_lse = out_lse;
   a.status = status;
+  a.n_split = num_splits;
+  a.part_o = static_cast<float*>(workspace);
+  a.part_ml = a.part_o ? a.part_o + (size_t)batch->B * n_q * layer->Hq * num_splits * RV : nullptr;
   a.qp_bytes = mq::kRows * 2 * (fold_v ? RK : (RK > RV ? RK : RV));
   const int fixed = 1024 + 2 * a.qp_bytes + 4 * mq::kPBytes + mq::kCtrlBytes;
   a.nst = (mq::kSmemLimit - fixed) / mq::kStageBytes;
   if (a.nst > mq::kMaxStages) a.nst = mq::kMaxStages;
   if (a.nst < 3) return STIEF_ERR_UNSUPPORTED;       // two query tiles and U_k are in the ring together
   L.smem = fixed + a.nst * mq::kStageBytes;
-  const long long n_units = (long long)((n_q + 2 * TT - 1) / (2 * TT)) * batch->B * layer->Hkv;
+  const long long n_units = (long long)((n_q + 2 * TT - 1) / (2 * TT)) * batch->B * layer->Hkv * num_splits;
   L.grid = (int)(n_units < host::sm_count() ? n_units : host::sm_count());
   cudaError_t e = cudaErrorInvalidValue;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -102,5 +136,6 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
     case 96: e = launch_mq_rk96(L, st); break;
     case 128: e = launch_mq_rk128(L, st); break;
   }
+  if (e == cudaSuccess && num_splits > 1) e = launch_mq_combine(a, st);
   return e == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }

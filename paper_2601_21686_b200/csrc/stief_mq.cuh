@@ -27,6 +27,9 @@
 // TMEM (512 columns): per tile two score buffers of 64 columns (which also take OUT at the end of a unit) and
 // 128 columns for Q' / O.
 // Units are taken round-robin (unit u -> CTA u mod grid), heaviest (latest query tokens) first.
+// With few query rows and a long cache (speculative decode) the units are too few to fill the GPU: the host then cuts
+// every unit's page range into n_split parts, which run as units of their own and leave partial results (unnormalised
+// mix, reference maximum, row sum) that mq_combine_kernel merges, normalises and back-projects.
 //
 // Precision: q' and P pass through bf16 (as the cache itself does); scores, sums and O_down keep fp32 accuracy.
 // Every wait is bounded (see mbar_wait): on a timeout the status word says so, later waits return at once, every
@@ -62,13 +65,20 @@ struct Args {
   int32_t* status;
   int nst;                       // ring stages
   int qp_bytes;                  // bytes of one tile's Q' / O_down operand region
+  // Split-T (few query rows, long cache): every unit's page range is cut into n_split parts that run as separate
+  // units and leave partial results; mq_combine_kernel merges them.  n_split = 1: results are final.
+  int n_split;
+  float* part_o;                 // [B * n_q * Hq][n_split][r_v]  unnormalised mix, relative to the part's own reference
+  float* part_ml;                // [B * n_q * Hq][n_split][2]    that reference in base-2 units, and the row sum
 };
 
 // A unit as every role derives it (same loads, same arithmetic)
 struct Unit {
   int b, h;
   int tok0[2];                   // first query token of each tile
-  int np[2];                     // cache pages each tile reads (0 = tile has no valid row)
+  int np[2];                     // cache pages each tile reads in this unit (0 = none)
+  int p_lo;                      // first of those pages (0 unless the sequence's pages are split over several units)
+  int split;                     // which part of the page range this unit is
   int q_len, q_start;            // query tokens of the sequence; absolute position of its query token 0
   int seq_len;                   // cached tokens of the sequence
   bool valid;
@@ -78,8 +88,11 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int u, int TT) {
   Unit w;
   const int bh = a.Bt.B * a.L.Hkv;
   const int n_t2 = (a.n_q + 2 * TT - 1) / (2 * TT);
-  const int t2 = n_t2 - 1 - u / bh;              // heaviest tiles first
-  const int r = u % bh;
+  const int ub = u / a.n_split;
+  w.split = u - ub * a.n_split;
+  w.p_lo = 0;
+  const int t2 = n_t2 - 1 - ub / bh;             // heaviest tiles first
+  const int r = ub % bh;
   w.b = r / a.L.Hkv;
   w.h = r - w.b * a.L.Hkv;
   int ql = a.q_lens ? a.q_lens[w.b] : a.n_q;
@@ -97,10 +110,16 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int u, int TT) {
     report(a.status, STIEF_ERR_BOUNDS);
     return w;
   }
-  w.valid = true;
+  int full[2] = {0, 0};                          // pages each tile attends in all
 #pragma unroll
   for (int t = 0; t < 2; ++t)
-    if (w.tok0[t] < ql) w.np[t] = (w.q_start + min(w.tok0[t] + TT, ql) - 1) / kPage + 1;
+    if (w.tok0[t] < ql) full[t] = (w.q_start + min(w.tok0[t] + TT, ql) - 1) / kPage + 1;
+  const int all = max(full[0], full[1]);
+  const int lo = (int)((long long)w.split * all / a.n_split), hi = (int)((long long)(w.split + 1) * all / a.n_split);
+  w.p_lo = lo;
+#pragma unroll
+  for (int t = 0; t < 2; ++t) w.np[t] = max(0, min(hi, full[t]) - lo);
+  w.valid = (w.np[0] | w.np[1]) != 0;            // a part may be empty when there are fewer pages than parts
   return w;
 }
 
@@ -171,7 +190,8 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const bool fold_k = a.L.U_k == nullptr, fold_v = a.L.U_v == nullptr;
   const int TT = kRows / G;                                     // query tokens per tile
   const Blocks bk = blocks_of(RK), bv = blocks_of(RV);
-  const int n_units = ((a.n_q + 2 * TT - 1) / (2 * TT)) * a.Bt.B * Hkv;
+  const int n_units = ((a.n_q + 2 * TT - 1) / (2 * TT)) * a.Bt.B * Hkv * a.n_split;
+  const bool backproj = !fold_v && a.n_split == 1;               // else the compressed (partial) result leaves the kernel
   int32_t* status = a.status;
 
   if (tid == 0) {
@@ -208,7 +228,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
       if (!fold_k) tma_prefetch_desc(&tmUk);
-      if (!fold_v) tma_prefetch_desc(&tmUv);
+      if (backproj) tma_prefetch_desc(&tmUv);
       tma_prefetch_desc(&tmQ);
     }
     int st = 0, use = 0;                                        // ring stage of the next item, times it has been used
@@ -228,7 +248,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!w.valid) continue;
       const int npmax = max(w.np[0], w.np[1]);
       const int* bt = a.Bt.block_table + (size_t)w.b * a.Bt.max_pages;
-      int ids = lane < npmax ? bt[lane] : 0;                    // first batch of page ids, in flight during the q loads
+      int ids = lane < npmax ? bt[w.p_lo + lane] : 0;                    // first batch of page ids, in flight during the q loads
       if (lane == 0) {
         if (fold_k) {
           for (int t = 0; t < 2; ++t) {
@@ -255,7 +275,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
       }
       for (int j0 = 0; j0 < npmax; j0 += 32) {
-        const int nxt = j0 + 32 + lane < npmax ? bt[j0 + 32 + lane] : 0;    // the next batch, a batch ahead
+        const int nxt = j0 + 32 + lane < npmax ? bt[w.p_lo + j0 + 32 + lane] : 0;    // the next batch, a batch ahead
         const int cnt = min(32, npmax - j0);
         for (int jj = 0; jj < cnt; ++jj) {
           int pg = __shfl_sync(0xffffffffu, ids, jj);
@@ -275,7 +295,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         ids = nxt;
       }
-      if (lane == 0 && !fold_v) {
+      if (lane == 0 && backproj) {
         const uint32_t dst = acquire();
         mbar_arrive_expect_tx(full_bar(st), kD * RV * 2);
         for (int i = 0; i < bv.nb; ++i)
@@ -409,7 +429,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         issue_pv(npmax - 1, prev_v, prev_stage);
         if (active && leader) umma_commit(o_full(mt));
-        if (!fold_v) {
+        if (backproj) {
           // OUT = O_down U_v^T with O_down handed over as two bf16 terms (value, then residual): two accumulating
           // passes into the tile's score columns, which are idle by now
           uint32_t ua;
@@ -454,7 +474,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!w.valid) continue;
       const int lead = fold_k ? 0 : (w.np[0] > 0) + (w.np[1] > 0) + 1;      // items ahead of the unit's first page
       const int item0 = item + lead;
-      item += lead + max(w.np[0], w.np[1]) + (fold_v ? 0 : 1);
+      item += lead + max(w.np[0], w.np[1]) + (backproj ? 1 : 0);
       if (w.np[t] == 0) continue;
       const int np = w.np[t];
       const int tok = w.tok0[t] + row / G, g = row - (row / G) * G;
@@ -489,7 +509,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc_fence_before();
         arrive_warp(s_free(t, sb));                             // the score buffer may be overwritten
         float* s = reinterpret_cast<float*>(sv);
-        const int p0 = j * kPage;
+        const int p0 = (w.p_lo + j) * kPage;
         if (p0 + kPage - 1 > q_pos) {                           // a boundary page: positions after the row's own are masked
 #pragma unroll
           for (int i = 0; i < 64; ++i)
@@ -503,7 +523,9 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         const float mx = fmaxf(max3(mx0, s[62], s[63]), mx1);
         if (j == 0) {
-          m_ref = mx;                                           // position 0 is visible to every row: finite
+          // The reference is the first page's maximum: finite when position 0 is in it.  A later part of a split range
+          // can be masked entirely for a row; a finite stand-in then gives p = 0 and an empty partial (l = 0).
+          m_ref = fmaxf(mx, -1e30f);
           l = 0.f;
         } else if (__any_sync(0xffffffffu, (mx - m_ref) * c > kRescaleLog2)) {
           mbar_wait(p_free(t, (n - 1) & 1), ((n - 1) >> 1) & 1, abort_flag, status);   // every earlier update of O is complete
@@ -564,7 +586,22 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc_fence_after();
       const float inv = 1.0f / l;
       __nv_bfloat16* orow = a.out + (size_t)w.b * a.out_stride_b + (size_t)tok * a.out_stride_t + (size_t)(w.h * G + g) * d_out;
-      if (fold_v) {
+      if (a.n_split > 1) {
+        // partial result of this part of the page range: unnormalised mix, reference (base-2 units) and row sum
+        const size_t prow = (((size_t)w.b * a.n_q + tok) * a.L.Hq + w.h * G + g) * a.n_split + w.split;
+        for (int c0 = 0; c0 < RV; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(t_out + c0, v);
+          tmem_ld_wait();
+          if (row_valid) {
+            float4* dst = reinterpret_cast<float4*>(a.part_o + prow * RV + c0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+          }
+        }
+        if (row_valid) *reinterpret_cast<float2*>(a.part_ml + prow * 2) = make_float2(m_ref * c, l);
+      } else if (fold_v) {
         for (int c0 = 0; c0 < RV; c0 += 16) {
           uint32_t v[16], pk[8];
           tmem_ld16(t_out + c0, v);
@@ -610,7 +647,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
         }
       }
-      if (row_valid && a.out_lse)
+      if (row_valid && a.out_lse && a.n_split == 1)
         a.out_lse[((size_t)w.b * a.n_q + tok) * a.L.Hq + w.h * G + g] = kLn2 * (m_ref * c + log2f(l));
       tc_fence_before();
       arrive_warp(unit_done(t));                                // the tile's TMEM columns and operand region are free
@@ -622,6 +659,76 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// Merges the parts of a split page range (log-sum-exp over the parts' references), normalises, back-projects and
+// writes the rows.  One block per (token, KV head, sequence): its G query rows share U_v.  A part that had no page
+// for the row's tile was never written and is skipped by redoing the range arithmetic of decode_unit.
+constexpr int kCombineThreads = 128;
+template <int kInstance>                                         // a template only so that the header can be included by several units
+__global__ void __launch_bounds__(kCombineThreads)
+mq_combine_kernel(const Args a) {
+  __shared__ float od[16][kD];                                   // up to 16 query rows of the group at a time
+  __shared__ float lse_s[16];
+  const int tok = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int G = a.L.G, RV = a.L.r_v, TT = kRows / G;
+  int ql = a.q_lens ? a.q_lens[b] : a.n_q;
+  ql = min(max(ql, 0), a.n_q);
+  const int sl = a.Bt.seq_lens[b], q_start = sl - ql;
+  if (tok >= ql || q_start < 0 || (sl + kPage - 1) / kPage > a.Bt.max_pages) return;
+  // pages of the row's tile and of the unit (both tiles), as decode_unit derives them
+  const int t2 = tok / (2 * TT), first = t2 * 2 * TT;
+  int full[2] = {0, 0};
+  for (int t = 0; t < 2; ++t)
+    if (first + t * TT < ql) full[t] = (q_start + min(first + (t + 1) * TT, ql) - 1) / kPage + 1;
+  const int all = max(full[0], full[1]), mine = full[(tok - first) / TT];
+  const bool fold_v = a.L.U_v == nullptr;
+  const int d_out = fold_v ? RV : kD;
+  const __nv_bfloat16* Uv = fold_v ? nullptr : a.L.U_v + (size_t)h * a.L.uv_stride;
+  for (int g0 = 0; g0 < G; g0 += 16) {
+    const int ng = min(16, G - g0);
+    __syncthreads();
+    for (int e = threadIdx.x; e < ng * RV; e += kCombineThreads) {
+      const int g = e / RV, cidx = e - g * RV;
+      const size_t prow = (((size_t)b * a.n_q + tok) * a.L.Hq + h * G + g0 + g) * a.n_split;
+      float M = -INFINITY;
+      for (int s = 0; s < a.n_split; ++s)
+        if ((int)((long long)s * all / a.n_split) < min((int)((long long)(s + 1) * all / a.n_split), mine)) M = fmaxf(M, a.part_ml[(prow + s) * 2]);
+      float num = 0.f, den = 0.f;
+      for (int s = 0; s < a.n_split; ++s)
+        if ((int)((long long)s * all / a.n_split) < min((int)((long long)(s + 1) * all / a.n_split), mine)) {
+          const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (prow + s) * 2);
+          const float wgt = fast_exp2(ml.x - M);
+          den += ml.y * wgt;
+          num += a.part_o[(prow + s) * RV + cidx] * wgt;
+        }
+      od[g][cidx] = num / den;
+      if (cidx == 0) lse_s[g] = kLn2 * (M + log2f(den));
+    }
+    __syncthreads();
+    for (int g = 0; g < ng; ++g) {
+      const int hq = h * G + g0 + g;
+      __nv_bfloat16* orow = a.out + (size_t)b * a.out_stride_b + (size_t)tok * a.out_stride_t + (size_t)hq * d_out;
+      if (fold_v) {
+        for (int cidx = threadIdx.x; cidx < RV; cidx += kCombineThreads) orow[cidx] = __float2bfloat16_rn(od[g][cidx]);
+      } else {
+        const int d = threadIdx.x;                               // one output element per thread: row d of U_v
+        const uint4* urow = reinterpret_cast<const uint4*>(Uv + (size_t)d * RV);
+        float acc = 0.f;
+        for (int c8 = 0; c8 < RV / 8; ++c8) {
+          const uint4 u = urow[c8];
+          const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            acc = fmaf(od[g][c8 * 8 + 2 * i], bf16_lo(wv[i]), acc);
+            acc = fmaf(od[g][c8 * 8 + 2 * i + 1], bf16_hi(wv[i]), acc);
+          }
+        }
+        orow[d] = __float2bfloat16_rn(acc);
+      }
+      if (threadIdx.x == 0 && a.out_lse) a.out_lse[((size_t)b * a.n_q + tok) * a.L.Hq + hq] = lse_s[g];
+    }
+  }
 }
 
 // What the host hands to a launcher: the argument block, the five tensor maps, the launch shape.
@@ -639,6 +746,7 @@ cudaError_t launch_mq_rk48(const mq::Launch& l, cudaStream_t st);
 cudaError_t launch_mq_rk64(const mq::Launch& l, cudaStream_t st);
 cudaError_t launch_mq_rk96(const mq::Launch& l, cudaStream_t st);
 cudaError_t launch_mq_rk128(const mq::Launch& l, cudaStream_t st);
+cudaError_t launch_mq_combine(const mq::Args& a, cudaStream_t st);
 
 
 }  // namespace stief

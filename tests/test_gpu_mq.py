@@ -259,3 +259,62 @@ def test_chunk_rows_have_the_bits_of_single_token_append():
     S.stief_append_chunk(c3.layer, c3.batch, big.to(DEV), big.to(DEV), status=c3.status)
     torch.cuda.synchronize()
     assert int(c3.status.item()) == S.STIEF_ERR_BOUNDS
+
+
+@pytest.mark.parametrize("num_splits", [2, 4, 13])
+@pytest.mark.parametrize("fold_v", [False, True])
+def test_split_page_ranges_for_few_query_rows(num_splits, fold_v):
+    # speculative-decode shape: a handful of query tokens over a long cache, the page range cut into parts (13 parts
+    # against 5 pages of the short sequence leaves some parts empty); masked-out parts of a row must drop out
+    c = U.make_case(77, 2, 8, 2, 64, 48, [700, 300], lowrank=True)
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    if fold_v:
+        c.layer.U_v, c.U_v = None, None
+    q = _queries(13, 2, 6, 8, scale=1.5)
+    q_lens = [6, 3]
+    d_out = 48 if fold_v else 128
+    ws = torch.full((S.stief_mq_workspace_bytes(2, 6, 8, 48, num_splits) // 4,), float("nan"), dtype=torch.float32, device=DEV)
+    out = torch.full((2, 6, 8, d_out), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((2, 6, 8), float("nan"), dtype=torch.float32, device=DEV)
+    S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, q_lens=torch.tensor(q_lens, dtype=torch.int32, device=DEV),
+                         out_lse=lse, status=c.status, workspace=ws, num_splits=num_splits)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    _compare(out, lse, *_reference(c, q, q_lens))
+    one, _ = _run(c, q, q_lens)                                  # unsplit: same rows up to the rounding of the merge
+    due = ~torch.isnan(one[..., 0])
+    assert (out[due].float() - one[due].float()).abs().max() < 2e-2
+
+
+def test_split_across_a_page_boundary_masks_whole_parts():
+    # 8 query tokens ending at position 64*5 + 2: the first rows sit on page 4, the last on page 5, so the part that holds
+    # only page 5 is entirely masked for the early rows
+    c = U.make_case(78, 1, 4, 1, 64, 64, [64 * 5 + 3])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(14, 1, 8, 4)
+    ws = torch.empty(S.stief_mq_workspace_bytes(1, 8, 4, 64, 6) // 4, dtype=torch.float32, device=DEV)
+    out = torch.full((1, 8, 4, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, workspace=ws, num_splits=6)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    ref, _ = _reference(c, q, [8])
+    _compare(out, None, ref, None)
+
+
+def test_split_planning_and_workspace_errors():
+    assert S.stief_mq_num_splits(4, 2048, 32, 8, 513) == 1                      # a chunk fills the GPU by itself
+    s = S.stief_mq_num_splits(4, 8, 32, 8, 513)
+    assert 2 <= s <= 64 and 32 * s <= 148
+    assert S.stief_mq_num_splits(1, 4, 32, 8, 8) <= 2                          # never more parts than a quarter of the pages
+    assert S.stief_mq_workspace_bytes(4, 8, 32, 64, 1) == 0
+    assert S.stief_mq_workspace_bytes(4, 8, 32, 64, 4) >= 4 * 8 * 32 * 4 * 66 * 4
+    c = U.make_case(79, 1, 8, 2, 64, 64, [200])
+    q = _queries(15, 1, 4, 8)
+    out = torch.zeros(1, 4, 8, 128, dtype=torch.bfloat16, device=DEV)
+    small = torch.empty(64, dtype=torch.float32, device=DEV)
+    with pytest.raises(S.StiefError) as e:
+        S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, workspace=small, num_splits=3)
+    assert e.value.code == S.STIEF_ERR_WORKSPACE
+    with pytest.raises(S.StiefError) as e:
+        S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, num_splits=3)
+    assert e.value.code == S.STIEF_ERR_INVALID_ARG
