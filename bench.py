@@ -14,7 +14,7 @@ several independent layer caches, each larger than L2, so no step finds its cach
 
 metric  = effective HBM bandwidth over the compressed cache bytes a step must read
           (B * Hkv * (T+1) * 2 * (r_k + r_v) bytes per step); tokens/s is reported next to it.
-Prints one JSON line (see the design doc for every key).  `--impl reference` times the CPU oracle instead.
+Prints one JSON line.  `--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
 

@@ -191,3 +191,71 @@ def test_config3_steps_with_per_layer_ranks():
     assert np.array_equal(lens_dev.cpu().numpy(), np.full(4, 32768 + n_steps, dtype=np.int32))
     for i, c in enumerate(cs):              # last step's outputs against the oracle on the grown cache
         check_pair(c, 2, 5, qs[i], outs[i], new_kv=hist[i], lens=c.seq_lens + n_steps)
+
+
+def _mq_sample_check(c: DevCase, q, out, lse, n_q, samples):
+    """Sampled rows (b, query token i, query head g) of a multi-query call against the oracle's single-row definition
+    on the cache rows the GPU holds: row i sits at position seq_len - n_q + i and attends positions 0 .. that."""
+    G = c.Hq // c.Hkv
+    worst = 0.0
+    cache = {}
+    for b, i, g in samples:
+        h = g // G
+        if (b, h) not in cache:
+            n = int(c.seq_lens[b])
+            cache[(b, h)] = (c.rows(c.layer.k_pool, b, h, 0, n).double().numpy(), c.rows(c.layer.v_pool, b, h, 0, n).double().numpy())
+        Kd, Vd = cache[(b, h)]
+        p = int(c.seq_lens[b]) - n_q + i
+        ref, ref_lse = O.attend_path_b(q[b, i, g].double().cpu().numpy(), Kd[:p + 1], Vd[:p + 1],
+                                       O.basis_of(U.f64(c.U_k), h), O.basis_of(U.f64(c.U_v), h))
+        got = out[b, i, g].double().cpu().numpy()
+        assert np.all(np.isfinite(got))
+        err = np.abs(got - ref).max()
+        rl = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert err <= max(1e-2, 2.0 ** -7 * np.abs(ref).max()) and rl <= 5e-3, (b, i, g, err, rl)
+        if lse is not None:
+            assert abs(float(lse[b, i, g]) - ref_lse) < 2e-2 + 2.0 ** -8 * abs(ref_lse), (b, i, g)
+        worst = max(worst, rl)
+    return worst
+
+
+@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 128)])
+def test_mq_chunk_at_bench_size(r_k, r_v):
+    # the `bench.py --mq` workload: a 2048-token chunk at the end of the 32768-token config-2 cache; every CTA works
+    # through about 14 units, which the small cases never do
+    B, Hq, Hkv, T, n_q = 4, 32, 8, 32768, 2048
+    c = DevCase(21, 0, B, Hq, Hkv, r_k, r_v, [T] * B, reserve=1)
+    S.stief_prefill_compress(c.layer, c.batch, c.K, c.V, status=c.status)
+    del c.K, c.V
+    q = I.normal_bf16(I.stream_key(21, I.TAG_Q, 100), (B, n_q, Hq, 128), device=DEV)
+    out = torch.full((B, n_q, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, n_q, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    for _ in range(2):                                   # twice: the second launch finds every barrier phase advanced
+        S.stief_mq_attention(c.layer, c.batch, q, out, out_lse=lse, status=c.status)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    assert not torch.isnan(out).any() and not torch.isnan(lse).any()
+    idx = I.randint(I.stream_key(21, I.TAG_PERM, 7), 3 * 40, 0, 2 ** 20)
+    samples = [(int(idx[3 * k]) % B, int(idx[3 * k + 1]) % n_q, int(idx[3 * k + 2]) % Hq) for k in range(40)]
+    samples += [(0, 0, 0), (B - 1, n_q - 1, Hq - 1), (1, 63, 5), (2, 64, 9), (3, 1023, 31), (0, 1024, 16)]   # tile and unit edges
+    _mq_sample_check(c, q, out, lse, n_q, samples)
+
+
+def test_mq_few_rows_at_bench_size_split_ranges():
+    # the speculative-decode shape of `bench.py --mq --n-q 8`: page ranges cut as the library proposes, merged by the
+    # combine kernel; every row is checked
+    B, Hq, Hkv, T, n_q = 4, 32, 8, 32768, 8
+    c = DevCase(22, 0, B, Hq, Hkv, 64, 64, [T] * B, reserve=1)
+    S.stief_prefill_compress(c.layer, c.batch, c.K, c.V, status=c.status)
+    del c.K, c.V
+    q = I.normal_bf16(I.stream_key(22, I.TAG_Q, 100), (B, n_q, Hq, 128), device=DEV)
+    n_split = S.stief_mq_num_splits(B, n_q, Hq, Hkv, c.batch.block_table.shape[1])
+    assert n_split > 1
+    ws = torch.full((S.stief_mq_workspace_bytes(B, n_q, Hq, 64, n_split) // 4,), float("nan"), dtype=torch.float32, device=DEV)
+    out = torch.full((B, n_q, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, n_q, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    S.stief_mq_attention(c.layer, c.batch, q, out, out_lse=lse, status=c.status, workspace=ws, num_splits=n_split)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0 and not torch.isnan(out).any()
+    samples = [(b, i, g) for b in (0, 3) for i in range(n_q) for g in (0, 13, 31)]
+    _mq_sample_check(c, q, out, lse, n_q, samples)
