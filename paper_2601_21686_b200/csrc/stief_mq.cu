@@ -120,7 +120,7 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
   a.part_o = static_cast<float*>(workspace);
   a.part_ml = a.part_o ? a.part_o + (size_t)batch->B * n_q * layer->Hq * num_splits * RV : nullptr;
   a.qp_bytes = mq::kRows * 2 * (fold_v ? RK : (RK > RV ? RK : RV));
-  const int fixed = 1024 + 2 * a.qp_bytes + 4 * mq::kPBytes + mq::kCtrlBytes;
+  const int fixed = 1024 + 2 * a.qp_bytes + mq::kCtrlBytes;
   a.nst = (mq::kSmemLimit - fixed) / mq::kStageBytes;
   if (a.nst > mq::kMaxStages) a.nst = mq::kMaxStages;
   if (a.nst < 3) return STIEF_ERR_UNSUPPORTED;       // two query tiles and U_k are in the ring together

@@ -13,12 +13,12 @@
 //               that tcgen05.mma reads (see Blocks); block-table entries are fetched 32 at a time, a batch ahead.
 //   warps 1,10  MMA issue, one thread per tile (warp 1 also allocates TMEM).  Per unit: Q' = Q U_k  (A = raw q rows, B = U_k as an
 //               MN-major operand) into the tile's accumulator columns; per page j and tile: S = Q' K_j^T (N = 64
-//               positions) into one of two score buffers, then O += P_j V_j (B = the V page, MN-major) once the
-//               softmax warps have published P_j; finally OUT = O_down U_v^T (B = U_v, K-major).  QK of page j+1 is
+//               positions) into one of two score buffers, then O += P_j V_j (A = P_j read from TMEM, B = the V page,
+//               MN-major) once the softmax warps have published P_j; finally OUT = O_down U_v^T (B = U_v, K-major).  QK of page j+1 is
 //               issued before PV of page j, so the tensor pipe works on the next scores while P_j is being made.
 //   warps 2-5   softmax / epilogue of tile 0, warps 6-9 of tile 1; thread = row (TMEM lane).  Round Q' to bf16 into
 //               the A operand; per page: tcgen05.ld the scores, causal mask on the boundary pages, running
-//               reference maximum, p = 2^(c s - c m) to bf16 into the P operand, row sum.  The accumulator in TMEM
+//               reference maximum, p = 2^(c s - c m) as bf16 pairs back into the score buffer (TMEM), row sum.  The accumulator in TMEM
 //               is rescaled only when a row's maximum has grown by more than 2^8 since the reference was set
 //               (p <= 256 stays exact enough in bf16/fp32); that is decided per warp and done with tcgen05.ld/st
 //               after the previous PV has completed.  Epilogue: O / l as two bf16 terms (value and residual), the A
@@ -47,7 +47,6 @@ using namespace tc;
 constexpr int kThreads = 352;
 constexpr int kRows = 128;                      // rows per tile
 constexpr int kStageBytes = 32768;              // one ring stage
-constexpr int kPBytes = kRows * kPage * 2;      // one tile's P operand: 128 rows x 64 positions bf16
 constexpr int kCtrlBytes = 1024;
 constexpr int kSmemLimit = 232448;              // 227 KiB per CTA
 constexpr int kTmemCols = 512;
@@ -167,14 +166,11 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const uint32_t ring = base;
   const uint32_t qp = ring + nst * kStageBytes;                 // Q' / O_down operands, one region per tile
   uint8_t* qp_ptr = base_ptr + nst * kStageBytes;
-  const uint32_t pb = qp + 2 * a.qp_bytes;                      // P operands, two buffers per tile
-  uint8_t* pb_ptr = qp_ptr + 2 * a.qp_bytes;
-  const uint32_t ctrl = pb + 4 * kPBytes;
-  uint8_t* ctrl_ptr = pb_ptr + 4 * kPBytes;
+  const uint32_t ctrl = qp + 2 * a.qp_bytes;
+  uint8_t* ctrl_ptr = qp_ptr + 2 * a.qp_bytes;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (6 + s) * 8; };
   auto s_full = [&](int t, int i) { return ctrl + (12 + t * 2 + i) * 8; };
-  auto s_free = [&](int t, int i) { return ctrl + (16 + t * 2 + i) * 8; };
   auto p_full = [&](int t, int i) { return ctrl + (20 + t * 2 + i) * 8; };
   auto p_free = [&](int t, int i) { return ctrl + (24 + t * 2 + i) * 8; };
   auto qacc_full = [&](int t) { return ctrl + (28 + t) * 8; };
@@ -202,8 +198,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int t = 0; t < 2; ++t) {
       for (int i = 0; i < 2; ++i) {
         mbar_init(s_full(t, i), 1);
-        mbar_init(s_free(t, i), 4);       // one arrival per softmax warp of the tile
-        mbar_init(p_full(t, i), 4);
+        mbar_init(p_full(t, i), 4);       // one arrival per softmax warp of the tile
         mbar_init(p_free(t, i), 1);
       }
       mbar_init(qacc_full(t), 1);
@@ -400,10 +395,11 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int n = pn + jj;
             mbar_wait(p_full(mt, n & 1), (n >> 1) & 1, abort_flag, status);
             tc_fence_after();
-            const uint64_t da = desc_at(d_sw128, pb + (mt * 2 + (n & 1)) * kPBytes), db = desc_at(d_vpage, vaddr);
+            const uint32_t pa = t_s + (n & 1) * 64;                     // P_n: packed bf16 pairs in the score buffer's first 32 columns
+            const uint64_t db = desc_at(d_vpage, vaddr);
 #pragma unroll
             for (int k = 0; k < kPage / 16; ++k)
-              if (leader) umma_bf16(t_o, da + (uint32_t)(2 * k), db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
+              if (leader) umma_bf16_ts(t_o, pa + 8 * k, db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
             if (leader) umma_commit(p_free(mt, n & 1));
           }
           release(stage, jj < np);                              // K and V of this page are no longer needed by this tile
@@ -414,7 +410,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           consume(kaddr, stage);
           if (j < np) {
             const int n = pn + j;
-            if (n >= 2) mbar_wait(s_free(mt, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);
+            if (n >= 2) mbar_wait(p_free(mt, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2), which sat in this buffer, has been consumed
             tc_fence_after();
             const uint32_t d_tmem = t_s + (n & 1) * 64;
             const uint64_t db = desc_at(d_kmaj_k, kaddr);
@@ -460,7 +456,6 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t t_lane = tmem_base + ((uint32_t)(32 * q4) << 16) + t * 256;
     const uint32_t t_out = t_lane + 128;                        // Q' / O columns
     uint8_t* my_qp = qp_ptr + t * a.qp_bytes;
-    uint8_t* my_p = pb_ptr + t * 2 * kPBytes + row * 128;           // this row in the tile's first P buffer
     const float c = kLog2e * rsqrtf((float)kD);                 // scores are scaled by 1/sqrt(d_h); exponent in base 2
     const int d_out = fold_v ? RV : kD;
     int kt = 0, pn = 0;
@@ -506,8 +501,6 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int i = 0; i < 4; ++i) tmem_ld16(t_lane + sb * 64 + i * 16, *reinterpret_cast<uint32_t(*)[16]>(&sv[16 * i]));
         tmem_ld_wait();
-        tc_fence_before();
-        arrive_warp(s_free(t, sb));                             // the score buffer may be overwritten
         float* s = reinterpret_cast<float*>(sv);
         const int p0 = (w.p_lo + j) * kPage;
         if (p0 + kPage - 1 > q_pos) {                           // a boundary page: positions after the row's own are masked
@@ -555,8 +548,8 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int r = lo + e / per_row, ch = e % per_row;
             *reinterpret_cast<uint4*>(vrows + (ch / cpr) * kPage * bv.span + r * bv.span + (ch % cpr) * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
+          fence_proxy_async_smem();                              // generic writes -> visible to the tensor core's reads
         }
-        if (n >= 2) mbar_wait(p_free(t, sb), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2) has left this buffer
         const uint64_t c2 = pack2(c, c), neg2 = pack2(-m_ref * c, -m_ref * c);
         uint64_t sum2 = pack2(0.f, 0.f);
         uint32_t pk[32];
@@ -573,10 +566,11 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           unpack2(sum2, a0, a1);
           l += a0 + a1;
         }
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          *reinterpret_cast<uint4*>(my_p + sb * kPBytes + ((k ^ (row & 7)) << 4)) = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
-        fence_proxy_async_smem();
+        // P_n replaces the scores in TMEM: bf16 pairs in the first 32 columns of the buffer, where the P V MMA reads
+        // its A operand (no trip through shared memory, no proxy fence)
+        tmem_st16(t_lane + sb * 64, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
+        tmem_st16(t_lane + sb * 64 + 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
+        tmem_st_wait();
         tc_fence_before();
         arrive_warp(p_full(t, sb));
       }
