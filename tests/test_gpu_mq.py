@@ -318,3 +318,21 @@ def test_split_planning_and_workspace_errors():
     with pytest.raises(S.StiefError) as e:
         S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, status=c.status, num_splits=3)
     assert e.value.code == S.STIEF_ERR_INVALID_ARG
+
+
+def test_shared_key_basis_and_wide_groups():
+    # one key basis for all heads (the paper's head sharing: uk_head_stride = 0), and a group of 32 query heads per KV
+    # head (a 128-row tile then holds 4 tokens)
+    c = U.make_case(88, 2, 8, 2, 48, 64, [260, 131], shared_key_basis=True)
+    assert c.U_k.shape[0] == 1
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(21, 2, 45, 8)
+    out, lse = _run(c, q, [45, 20])
+    assert int(c.status.item()) == 0
+    _compare(out, lse, *_reference(c, q, [45, 20]))
+    c = U.make_case(89, 1, 32, 1, 64, 64, [200])
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(22, 1, 11, 32)
+    out, lse = _run(c, q, [11])
+    assert int(c.status.item()) == 0
+    _compare(out, lse, *_reference(c, q, [11]))
