@@ -309,8 +309,9 @@ int stief_time_next_decode_kernel(void* start_event, void* stop_event);
  *            their own and leave partial results in `workspace` (device, 128-byte aligned, at least
  *            stief_mq_workspace_bytes(...) bytes, contents irrelevant on entry); a second small kernel merges them
  *            (log-sum-exp), normalises and back-projects.  num_splits = 1: no workspace (NULL, 0).  stief_mq_num_splits
- *            proposes a value: 1 when the units already fill the GPU, else about SMs / units, at most 64 and at most a
- *            quarter of max_pages_per_seq.  Too small a workspace: STIEF_ERR_WORKSPACE, nothing is launched.
+ *            proposes a value: 1 when the units already fill the GPU, else about SMs / units, at most 32 and at most a
+ *            quarter of max_pages_per_seq.  When a (sequence, KV head) has at most 128 query rows, each part is further
+ *            worked through as two interleaved streams inside its CTA (the workspace size allows for that).  Too small a workspace: STIEF_ERR_WORKSPACE, nothing is launched.
  *   flags    must be 0
  * All ranks 32/48/64/96/128; Hq / Hkv must divide 128 (a 128-row tile holds whole tokens), else
  * STIEF_ERR_UNSUPPORTED.  Nothing is allocated.  Asynchronous on `stream`. */

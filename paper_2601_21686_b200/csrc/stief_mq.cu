@@ -33,7 +33,7 @@ extern "C" int32_t stief_mq_num_splits(int32_t B, int32_t n_q, int32_t Hq, int32
   const int TT = mq::kRows / G;
   const long long base = (long long)((n_q + 2 * TT - 1) / (2 * TT)) * B * Hkv;      // units without splitting
   long long s = host::sm_count() / base;                                           // parts so that the units about fill the GPU
-  if (s > 64) s = 64;
+  if (s > 32) s = 32;
   if (s > max_pages_per_seq / 4) s = max_pages_per_seq / 4;                        // at least a few pages per part
   return (int32_t)(s < 1 ? 1 : s);
 }
@@ -41,14 +41,15 @@ extern "C" int32_t stief_mq_num_splits(int32_t B, int32_t n_q, int32_t Hq, int32
 extern "C" size_t stief_mq_workspace_bytes(int32_t B, int32_t n_q, int32_t Hq, int32_t r_v, int32_t num_splits) {
   if (B <= 0 || n_q <= 0 || Hq <= 0 || r_v <= 0 || num_splits < 1) return 0;
   if (num_splits == 1) return 0;
-  return host::align_up((size_t)B * n_q * Hq * num_splits * (r_v + 2) * sizeof(float), 128);
+  // two result slots per part: with few query rows a CTA runs two softmax streams over alternate pages of its part
+  return host::align_up((size_t)B * n_q * Hq * 2 * num_splits * (r_v + 2) * sizeof(float), 128);
 }
 
 extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* batch, const uint16_t* q, int64_t q_stride_b,
                                   int64_t q_stride_t, int32_t n_q, const int32_t* q_lens, void* workspace,
                                   size_t workspace_bytes, int32_t num_splits, uint16_t* out, int64_t out_stride_b,
                                   int64_t out_stride_t, float* out_lse, uint32_t flags, int32_t* status, void* stream) {
-  if (!layer || !q || !out || flags != 0u || num_splits < 1 || num_splits > 64) return STIEF_ERR_INVALID_ARG;
+  if (!layer || !q || !out || flags != 0u || num_splits < 1 || num_splits > 32) return STIEF_ERR_INVALID_ARG;
   if (num_splits > 1) {
     if (!workspace || !host::aligned(workspace, 128)) return STIEF_ERR_INVALID_ARG;
     if (workspace_bytes < stief_mq_workspace_bytes(batch ? batch->B : 0, n_q, layer->Hq, layer->r_v, num_splits) ||
@@ -117,8 +118,10 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
   a.out_lse = out_lse;
   a.status = status;
   a.n_split = num_splits;
+  a.dual = (num_splits > 1 && (long long)n_q * G <= mq::kRows) ? 1 : 0;       // the second tile would have no rows of its own
+  a.n_parts = num_splits * (1 + a.dual);
   a.part_o = static_cast<float*>(workspace);
-  a.part_ml = a.part_o ? a.part_o + (size_t)batch->B * n_q * layer->Hq * num_splits * RV : nullptr;
+  a.part_ml = a.part_o ? a.part_o + (size_t)batch->B * n_q * layer->Hq * a.n_parts * RV : nullptr;
   a.qp_bytes = mq::kRows * 2 * (fold_v ? RK : (RK > RV ? RK : RV));
   const int fixed = 1024 + 2 * a.qp_bytes + mq::kCtrlBytes;
   a.nst = (mq::kSmemLimit - fixed) / mq::kStageBytes;

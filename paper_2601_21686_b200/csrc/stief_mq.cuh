@@ -67,8 +67,14 @@ struct Args {
   // Split-T (few query rows, long cache): every unit's page range is cut into n_split parts that run as separate
   // units and leave partial results; mq_combine_kernel merges them.  n_split = 1: results are final.
   int n_split;
-  float* part_o;                 // [B * n_q * Hq][n_split][r_v]  unnormalised mix, relative to the part's own reference
-  float* part_ml;                // [B * n_q * Hq][n_split][2]    that reference in base-2 units, and the row sum
+  // With at most 128 query rows per (sequence, KV head) the second tile of a unit would idle.  dual = 1 gives it the
+  // SAME rows and lets the two tiles take alternate pages of the unit's range (two independent softmax streams per
+  // CTA, each with its own partial result): a single stream is bound by the latency of its score -> softmax -> P V
+  // chain, two overlap.  Parts per row in the workspace: n_parts = n_split * (1 + dual).
+  int dual;
+  int n_parts;
+  float* part_o;                 // [B * n_q * Hq][n_parts][r_v]  unnormalised mix, relative to the part's own reference
+  float* part_ml;                // [B * n_q * Hq][n_parts][2]    that reference in base-2 units, and the row sum
 };
 
 // A unit as every role derives it (same loads, same arithmetic)
@@ -76,6 +82,7 @@ struct Unit {
   int b, h;
   int tok0[2];                   // first query token of each tile
   int np[2];                     // cache pages each tile reads in this unit (0 = none)
+  int cnt;                       // pages of the unit that go through the ring (dual: the tiles take alternate ones)
   int p_lo;                      // first of those pages (0 unless the sequence's pages are split over several units)
   int split;                     // which part of the page range this unit is
   int q_len, q_start;            // query tokens of the sequence; absolute position of its query token 0
@@ -102,8 +109,9 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int u, int TT) {
   w.seq_len = sl;
   w.valid = false;
   w.np[0] = w.np[1] = 0;
+  w.cnt = 0;
   w.tok0[0] = t2 * 2 * TT;
-  w.tok0[1] = w.tok0[0] + TT;
+  w.tok0[1] = a.dual ? w.tok0[0] : w.tok0[0] + TT;
   if (w.tok0[0] >= ql) return w;
   if (w.q_start < 0 || (sl + kPage - 1) / kPage > a.Bt.max_pages) {   // fewer cached tokens than query rows, or a table too short
     report(a.status, STIEF_ERR_BOUNDS);
@@ -116,9 +124,16 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int u, int TT) {
   const int all = max(full[0], full[1]);
   const int lo = (int)((long long)w.split * all / a.n_split), hi = (int)((long long)(w.split + 1) * all / a.n_split);
   w.p_lo = lo;
+  if (a.dual) {                                  // page lo + j goes to tile j & 1
+    w.cnt = max(0, min(hi, all) - lo);
+    w.np[0] = (w.cnt + 1) >> 1;
+    w.np[1] = w.cnt >> 1;
+  } else {
 #pragma unroll
-  for (int t = 0; t < 2; ++t) w.np[t] = max(0, min(hi, full[t]) - lo);
-  w.valid = (w.np[0] | w.np[1]) != 0;            // a part may be empty when there are fewer pages than parts
+    for (int t = 0; t < 2; ++t) w.np[t] = max(0, min(hi, full[t]) - lo);
+    w.cnt = max(w.np[0], w.np[1]);
+  }
+  w.valid = w.cnt != 0;                          // a part may be empty when there are fewer pages than parts
   return w;
 }
 
@@ -259,7 +274,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
       const Unit w = decode_unit(a, u, TT);
       if (!w.valid) continue;
-      const int npmax = max(w.np[0], w.np[1]);
+      const int npmax = w.cnt;
       const int* bt = a.Bt.block_table + (size_t)w.b * a.Bt.max_pages;
       int ids = lane < npmax ? bt[w.p_lo + lane] : 0;                    // first batch of page ids, in flight during the q loads
       if (lane == 0) {
@@ -375,9 +390,10 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // flow and the addresses below are the same in every lane
         if (!__shfl_sync(0xffffffffu, (int)w.valid, 0)) continue;
         const int wnp0 = __shfl_sync(0xffffffffu, w.np[0], 0), wnp1 = __shfl_sync(0xffffffffu, w.np[1], 0);
-        const int np = mt ? wnp1 : wnp0, np_other = mt ? wnp0 : wnp1;
-        const int npmax = max(np, np_other);
+        const int np = mt ? wnp1 : wnp0;
+        const int npmax = __shfl_sync(0xffffffffu, w.cnt, 0);
         const bool active = np > 0;
+        const bool dual = a.dual != 0;
         if (!fold_k) {
           uint32_t qa = 0, ua, tmp;
           int qs = -1, us, ts;
@@ -406,42 +422,46 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (active) mbar_wait(qp_ready(mt), kt & 1, abort_flag, status);
         tc_fence_after();
 
-        uint32_t prev_v = 0;
-        int prev_stage = -1;
-        auto issue_pv = [&](int jj, uint32_t vaddr, int stage) {
-          if (jj < np) {
-            const int n = pn + jj;
-            mbar_wait(p_full(mt, n & 1), (n >> 1) & 1, abort_flag, status);
-            tc_fence_after();
-            const uint32_t pa = t_s + (n & 1) * 64;                     // P_n: packed bf16 pairs in the score buffer's first 32 columns
-            const uint64_t db = desc_at(d_vpage, vaddr);
+        // jo counts this tile's own pages within the unit (every page it shares with the other tile, or every second
+        // page of the range when the tiles run as two streams over the same rows)
+        auto issue_pv = [&](int jo, uint32_t vaddr, int stage) {
+          const int n = pn + jo;
+          mbar_wait(p_full(mt, n & 1), (n >> 1) & 1, abort_flag, status);
+          tc_fence_after();
+          const uint32_t pa = t_s + (n & 1) * 64;                       // P_n: packed bf16 pairs in the score buffer's first 32 columns
+          const uint64_t db = desc_at(d_vpage, vaddr);
 #pragma unroll
-            for (int k = 0; k < kPage / 16; ++k)
-              if (leader) umma_bf16_ts(t_o, pa + 8 * k, db + (uint32_t)k * pv_b, id_pv, (jj > 0 || k > 0) ? 1u : 0u);
-            if (leader) umma_commit(p_free(mt, n & 1));
-          }
-          release(stage, jj < np);                              // K and V of this page are no longer needed by this tile
+          for (int k = 0; k < kPage / 16; ++k)
+            if (leader) umma_bf16_ts(t_o, pa + 8 * k, db + (uint32_t)k * pv_b, id_pv, (jo > 0 || k > 0) ? 1u : 0u);
+          if (leader) umma_commit(p_free(mt, n & 1));
+          release(stage, true);                                 // K and V of this page are no longer needed by this tile
         };
+        uint32_t prev_v = 0;
+        int prev_stage = -1, jo = 0;                            // the page whose P V is still to be issued; own pages so far
         for (int j = 0; j < npmax; ++j) {
           uint32_t kaddr;
           int stage;
           consume(kaddr, stage);
-          if (j < np) {
-            const int n = pn + j;
-            if (n >= 2) mbar_wait(p_free(mt, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2), which sat in this buffer, has been consumed
-            tc_fence_after();
-            const uint32_t d_tmem = t_s + (n & 1) * 64;
-            const uint64_t db = desc_at(d_kmaj_k, kaddr);
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              if (k < nk && leader) umma_bf16(d_tmem, dq + koff(k, lgk, qblk), db + koff(k, lgk, kblk), id_qk, k > 0 ? 1u : 0u);
-            if (leader) umma_commit(s_full(mt, n & 1));
+          const bool mine = dual ? (j & 1) == mt : j < np;
+          if (!mine) {
+            release(stage, false);
+            continue;
           }
-          if (j > 0) issue_pv(j - 1, prev_v, prev_stage);
+          const int n = pn + jo;
+          if (n >= 2) mbar_wait(p_free(mt, n & 1), ((n >> 1) - 1) & 1, abort_flag, status);   // P_(n-2), which sat in this buffer, has been consumed
+          tc_fence_after();
+          const uint32_t d_tmem = t_s + (n & 1) * 64;
+          const uint64_t db = desc_at(d_kmaj_k, kaddr);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (k < nk && leader) umma_bf16(d_tmem, dq + koff(k, lgk, qblk), db + koff(k, lgk, kblk), id_qk, k > 0 ? 1u : 0u);
+          if (leader) umma_commit(s_full(mt, n & 1));
+          if (jo > 0) issue_pv(jo - 1, prev_v, prev_stage);
           prev_v = kaddr + kPage * RK * 2;
           prev_stage = stage;
+          ++jo;
         }
-        issue_pv(npmax - 1, prev_v, prev_stage);
+        if (jo > 0) issue_pv(jo - 1, prev_v, prev_stage);
         if (active && leader) umma_commit(o_full(mt));
         if (backproj) {
           // OUT = O_down U_v^T with O_down handed over as two bf16 terms (value, then residual): two accumulating
@@ -487,7 +507,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!w.valid) continue;
       const int lead = fold_k ? 0 : (w.np[0] > 0) + (w.np[1] > 0) + 1;      // items ahead of the unit's first page
       const int item0 = item + lead;
-      item += lead + max(w.np[0], w.np[1]) + (backproj ? 1 : 0);
+      item += lead + w.cnt + (backproj ? 1 : 0);
       if (w.np[t] == 0) continue;
       const int np = w.np[t];
       const int tok = w.tok0[t] + row / G, g = row - (row / G) * G;
@@ -511,8 +531,9 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
 
       float m_ref = 0.f, l = 0.f;
-      for (int j = 0; j < np; ++j) {
-        const int n = pn + j, sb = n & 1;
+      for (int jo = 0; jo < np; ++jo) {
+        const int j = a.dual ? 2 * jo + t : jo;                 // the page within the unit's range
+        const int n = pn + jo, sb = n & 1;
         mbar_wait(s_full(t, sb), (n >> 1) & 1, abort_flag, status);
         tc_fence_after();
         uint32_t sv[64];
@@ -533,7 +554,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           mx1 = max3(mx1, s[i + 2], s[i + 3]);
         }
         const float mx = fmaxf(max3(mx0, s[62], s[63]), mx1);
-        if (j == 0) {
+        if (jo == 0) {
           // The reference is the first page's maximum: finite when position 0 is in it.  A later part of a split range
           // can be masked entirely for a row; a finite stand-in then gives p = 0 and an empty partial (l = 0).
           m_ref = fmaxf(mx, -1e30f);
@@ -606,7 +627,7 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       __nv_bfloat16* orow = a.out + (size_t)w.b * a.out_stride_b + (size_t)tok * a.out_stride_t + (size_t)(w.h * G + g) * d_out;
       if (a.n_split > 1) {
         // partial result of this part of the page range: unnormalised mix, reference (base-2 units) and row sum
-        const size_t prow = (((size_t)w.b * a.n_q + tok) * a.L.Hq + w.h * G + g) * a.n_split + w.split;
+        const size_t prow = (((size_t)w.b * a.n_q + tok) * a.L.Hq + w.h * G + g) * a.n_parts + (a.dual ? 2 * w.split + t : w.split);
         for (int c0 = 0; c0 < RV; c0 += 16) {
           uint32_t v[16];
           tmem_ld16(t_out + c0, v);
@@ -708,17 +729,22 @@ mq_combine_kernel(const Args a) {
     __syncthreads();
     for (int e = threadIdx.x; e < ng * RV; e += kCombineThreads) {
       const int g = e / RV, cidx = e - g * RV;
-      const size_t prow = (((size_t)b * a.n_q + tok) * a.L.Hq + h * G + g0 + g) * a.n_split;
+      const size_t prow = (((size_t)b * a.n_q + tok) * a.L.Hq + h * G + g0 + g) * a.n_parts;
+      // part i exists for this row if its share of the page range reaches into the pages of the row's tile
+      auto exists = [&](int i) {
+        const int sp = a.dual ? i >> 1 : i, off = a.dual ? i & 1 : 0;
+        return (int)((long long)sp * all / a.n_split) + off < min((int)((long long)(sp + 1) * all / a.n_split), mine);
+      };
       float M = -INFINITY;
-      for (int s = 0; s < a.n_split; ++s)
-        if ((int)((long long)s * all / a.n_split) < min((int)((long long)(s + 1) * all / a.n_split), mine)) M = fmaxf(M, a.part_ml[(prow + s) * 2]);
+      for (int i = 0; i < a.n_parts; ++i)
+        if (exists(i)) M = fmaxf(M, a.part_ml[(prow + i) * 2]);
       float num = 0.f, den = 0.f;
-      for (int s = 0; s < a.n_split; ++s)
-        if ((int)((long long)s * all / a.n_split) < min((int)((long long)(s + 1) * all / a.n_split), mine)) {
-          const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (prow + s) * 2);
+      for (int i = 0; i < a.n_parts; ++i)
+        if (exists(i)) {
+          const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (prow + i) * 2);
           const float wgt = fast_exp2(ml.x - M);
           den += ml.y * wgt;
-          num += a.part_o[(prow + s) * RV + cidx] * wgt;
+          num += a.part_o[(prow + i) * RV + cidx] * wgt;
         }
       od[g][cidx] = num / den;
       if (cidx == 0) lse_s[g] = kLn2 * (M + log2f(den));

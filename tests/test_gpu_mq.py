@@ -304,10 +304,10 @@ def test_split_across_a_page_boundary_masks_whole_parts():
 def test_split_planning_and_workspace_errors():
     assert S.stief_mq_num_splits(4, 2048, 32, 8, 513) == 1                      # a chunk fills the GPU by itself
     s = S.stief_mq_num_splits(4, 8, 32, 8, 513)
-    assert 2 <= s <= 64 and 32 * s <= 148
+    assert 2 <= s <= 32 and 32 * s <= 148
     assert S.stief_mq_num_splits(1, 4, 32, 8, 8) <= 2                          # never more parts than a quarter of the pages
     assert S.stief_mq_workspace_bytes(4, 8, 32, 64, 1) == 0
-    assert S.stief_mq_workspace_bytes(4, 8, 32, 64, 4) >= 4 * 8 * 32 * 4 * 66 * 4
+    assert S.stief_mq_workspace_bytes(4, 8, 32, 64, 4) >= 4 * 8 * 32 * 2 * 4 * 66 * 4
     c = U.make_case(79, 1, 8, 2, 64, 64, [200])
     q = _queries(15, 1, 4, 8)
     out = torch.zeros(1, 4, 8, 128, dtype=torch.bfloat16, device=DEV)
@@ -336,3 +336,19 @@ def test_shared_key_basis_and_wide_groups():
     out, lse = _run(c, q, [11])
     assert int(c.status.item()) == 0
     _compare(out, lse, *_reference(c, q, [11]))
+
+
+def test_split_ranges_with_two_row_tiles():
+    # more than 128 rows per (sequence, KV head): both tiles have rows of their own, so parts are plain page ranges
+    c = U.make_case(90, 2, 8, 2, 64, 64, [500, 260], lowrank=True)
+    S.stief_prefill_compress(c.layer, c.batch, c.K.to(DEV), c.V.to(DEV), status=c.status)
+    q = _queries(23, 2, 50, 8)
+    q_lens = [50, 37]
+    ws = torch.full((S.stief_mq_workspace_bytes(2, 50, 8, 64, 3) // 4,), float("nan"), dtype=torch.float32, device=DEV)
+    out = torch.full((2, 50, 8, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((2, 50, 8), float("nan"), dtype=torch.float32, device=DEV)
+    S.stief_mq_attention(c.layer, c.batch, q.to(DEV), out, q_lens=torch.tensor(q_lens, dtype=torch.int32, device=DEV),
+                         out_lse=lse, status=c.status, workspace=ws, num_splits=3)
+    torch.cuda.synchronize()
+    assert int(c.status.item()) == 0
+    _compare(out, lse, *_reference(c, q, q_lens))
