@@ -73,8 +73,11 @@ def bf16_ordinal(bits: np.ndarray) -> np.ndarray:
 
 
 def bf16_ulp(x: np.ndarray) -> np.ndarray:
-    """Spacing of bf16 numbers around x."""
-    _, e = np.frexp(np.asarray(x, dtype=np.float64))
+    """Spacing of bf16 numbers around x: 2^(e-8) for |x| in [2^(e-1), 2^e), and 2^-133 from the smallest
+    normal (2^-126) down to and including zero."""
+    x = np.asarray(x, dtype=np.float64)
+    _, e = np.frexp(x)
+    e = np.where(x == 0.0, -125, e)                     # frexp(0) reports exponent 0; zero sits in the subnormal range
     return np.ldexp(1.0, np.maximum(e, -125) - 8)
 
 

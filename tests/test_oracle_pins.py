@@ -65,6 +65,28 @@ def test_rnd_bf16_ties_to_even_and_single_rounding():
     assert list(O.bf16_ordinal(np.array([0x0000, 0x0001, 0x8001, 0x3F80, 0x3F81], dtype=np.uint16))) == [0, 1, -1, 0x3F80, 0x3F81]
 
 
+def test_bf16_ulp_against_fixed_spacings():
+    # bf16 keeps 8 significant bits: numbers in [2^(e-1), 2^e) are 2^(e-8) apart.  The values below are
+    # written out by hand from that rule, not computed by the function under test.
+    cases = {1.0: 2.0 ** -7, 1.5: 2.0 ** -7, 1.9921875: 2.0 ** -7, 2.0: 2.0 ** -6, 0.75: 2.0 ** -8, 0.5: 2.0 ** -8,
+             0.49999: 2.0 ** -9, 3.0: 2.0 ** -6, 100.0: 2.0 ** -1, 255.0: 1.0, 256.0: 2.0, 1e-6: 2.0 ** -27,
+             2.0 ** -126: 2.0 ** -133,            # smallest normal
+             2.0 ** -130: 2.0 ** -133,            # subnormal range keeps the last normal spacing
+             2.0 ** -133: 2.0 ** -133, 0.0: 2.0 ** -133}
+    for x, want in cases.items():
+        assert O.bf16_ulp(np.array([x]))[0] == want, x
+        assert O.bf16_ulp(np.array([-x]))[0] == want, -x            # the spacing does not depend on the sign
+    # the spacing is what separates neighbouring bit patterns: bits -> value, next pattern -> value, difference
+    pat = np.array([0x3F80, 0x3F00, 0x4000, 0x0080, 0x0001, 0x42C8, 0x7F00], dtype=np.uint16)
+    gap = O.bf16_from_bits(pat + np.uint16(1)) - O.bf16_from_bits(pat)
+    assert np.array_equal(O.bf16_ulp(O.bf16_from_bits(pat)), gap)
+    # and torch's own bf16 neighbours agree (nextafter on the bf16 grid), on random magnitudes
+    g = torch.Generator().manual_seed(7)
+    x = (torch.randn(4096, generator=g) * torch.exp(torch.randn(4096, generator=g) * 6)).to(torch.bfloat16)
+    up = torch.nextafter(x.abs(), torch.full_like(x, float("inf")))
+    assert np.array_equal(O.bf16_ulp(x.double().numpy()), (up.double() - x.abs().double()).numpy())
+
+
 # ---------------------------------------------------------------- bases
 
 @pytest.mark.parametrize("r", [32, 48, 64, 96, 128])

@@ -132,6 +132,33 @@ def test_bruteforce_tiny():
         assert np.allclose(out, ref, atol=1e-14) and abs(lse - (m + math.log(sum(w)))) < 1e-14
 
 
+def test_project_f32_against_hand_loops():
+    # Eq. 1 by explicit loops in exact rational arithmetic on bf16-valued inputs, then ONE rounding to fp32
+    from fractions import Fraction
+    g = np.random.default_rng(5)
+    X = O.rnd_bf16(g.standard_normal((3, 6)))
+    Ub = O.rnd_bf16(g.standard_normal((6, 4)))
+    got = Q.project_f32(X, Ub)
+    assert got.dtype == np.float32 and got.shape == (3, 4)
+    for t in range(3):
+        for j in range(4):
+            exact = sum(Fraction(float(X[t, i])) * Fraction(float(Ub[i, j])) for i in range(6))
+            # nearest fp32 to the exact sum: the candidates are the fp32 neighbours of its double approximation
+            c = np.float32(float(exact))
+            cands = [c, np.nextafter(c, np.float32(np.inf)), np.nextafter(c, np.float32(-np.inf))]
+            best = min(cands, key=lambda v: abs(Fraction(float(v)) - exact))
+            assert got[t, j] == best
+    # a sum whose fp32-accumulated value differs from the correctly rounded one: 1 + 2^-24 + 2^-24 -> 1 + 2^-23
+    Xs = np.array([[1.0, 2.0 ** -24, 2.0 ** -24]])
+    assert Q.project_f32(Xs, np.ones((3, 1)))[0, 0] == np.float32(1 + 2.0 ** -23)
+    # transposed operand, wrong axis: a non-square case with distinct entries catches both
+    Xn = np.array([[1.0, 2.0, 3.0]])
+    Un = np.array([[1.0, 10.0], [100.0, 1000.0], [10000.0, 100000.0]])
+    assert list(Q.project_f32(Xn, Un)[0]) == [30201.0, 302010.0]
+    # no basis: rows pass through (a side whose projection is folded into the linear layer), rounded to fp32
+    assert np.array_equal(Q.project_f32(Xs, None), Xs.astype(np.float32))
+
+
 def test_byte_accounting():
     assert Q.quantized_cache_bytes(64, 64, 8) == 136 and Q.quantized_cache_bytes(128, 128, 8) == 272
     assert Q.quantized_cache_bytes(64, 64, 4) == 72
