@@ -85,7 +85,7 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                                           "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -221,40 +221,48 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)
 
-    # ---- timed region 1: device-resident inputs
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    def timed_region(fn, n, first=0):
+        """n calls of fn between two events on the launching stream, a barrier and a device synchronise on both sides."""
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record()
+        for i in range(n):
+            fn(first + i)
+        b.record()
+        barrier()
+        return a.elapsed_time(b)
+
+    def repeated(fn, n, seconds, max_regions=2000):
+        """The n-step region repeated until `seconds` of device time have been measured (every rank runs the same
+        number of regions: the count comes from rank 0's first region).  Returns the per-region times."""
+        first = timed_region(fn, n, W)
+        cnt = R.max_over_ranks(me, [first], device=dev)[0]
+        n_regions = int(min(max_regions, max(5, np.ceil(seconds * 1e3 / max(cnt, 1e-3)))))
+        return [first] + [timed_region(fn, n, W + (r + 1) * n) for r in range(n_regions - 1)]
+
+    # ---- timed region 1: device-resident inputs.  A region is exactly K steps from a drained stream to a drained
+    # stream; it is repeated and the MEDIAN region is the reported value (a 20-step region lasts under a millisecond).
     t0 = time.time()
-    e0.record()
-    for i in range(K_steps):
-        step(W + i)
-    e1.record()
-    barrier()
-    t1 = time.time()
-    ms = e0.elapsed_time(e1)
+    regions = repeated(step, K_steps, args.seconds)
+    # ---- the same region with plainly serialised launches
+    regions_serial = repeated(lambda i: step(i, 0), K_steps, args.seconds / 4)
+    # ---- one long region: the launch pipeline in steady state (labelled as such, never the headline)
+    n_long = max(K_steps, args.steady_steps)
+    ms_long = timed_region(step, n_long, W)
 
-    # ---- the same loop with plainly serialised launches
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    s0.record()
-    for i in range(K_steps):
-        step(W + i, 0)
-    s1.record()
-    barrier()
-    ms_serial = s0.elapsed_time(s1)
-
-    # ---- timed region 2: the split-T kernel alone, per launch (events recorded inside the library call)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
+    # ---- the split-T kernel alone, per launch (events recorded inside the library call, serialised launches)
+    n_iso = max(K_steps, 50)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_iso)]
     for a, b in evs:
         a.record(); b.record()
     barrier()
-    for i in range(K_steps):
+    for i in range(n_iso):
         S.stief_time_next_decode_kernel(*evs[i])
         step(W + i, 0)
     barrier()
     kern_ms = [a.elapsed_time(b) for a, b in evs]
 
-    # ---- timed region 3: end to end through the host-buffer entry point
+    # ---- end to end through the host-buffer entry point
     staging = torch.empty(S.stief_host_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
     qh = [q.cpu().pin_memory() for q in qs]
     kh = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kvs]
@@ -267,27 +275,29 @@ def run_ours(args):
 
     for i in range(W):
         step_host(i)
-    barrier()
-    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    h0.record()
-    for i in range(K_steps):
-        step_host(W + i)
-    h1.record()
-    barrier()
-    ms_host = h0.elapsed_time(h1)
+    regions_host = repeated(step_host, K_steps, args.seconds / 4)
+    t1 = time.time()
     if rank == 0:
         sampler.stop()
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
-    # ---- max over ranks
-    ms, ms_host, kern_isolated_ms, ms_serial = R.max_over_ranks(me, [ms, ms_host, float(np.mean(kern_ms)), ms_serial], device=dev)
+    # ---- max over ranks, region by region; then the median region
+    def med(v):
+        v = R.max_over_ranks(me, v, device=dev)
+        return float(np.median(v)), float(min(v)), float(max(v)), len(v)
+
+    ms, ms_min, ms_max, n_reg = med(regions)
+    ms_serial, _, _, n_reg_serial = med(regions_serial)
+    ms_host, ms_host_min, ms_host_max, n_reg_host = med(regions_host)
+    kern_isolated_ms, ms_long = R.max_over_ranks(me, [float(np.mean(kern_ms)), ms_long], device=dev)
     kern_avg_ms = ms / K_steps          # one launch per step: the timed region divided by its launches
 
     if rank == 0:
         hbm_peak, tf_peak, peak_kind = measured_peaks()
         sb = step_bytes(cfg)
-        value = world * sb * K_steps / (ms * 1e-3) / 1e9
-        e2e = world * sb * K_steps / (ms_host * 1e-3) / 1e9
+        gbs = lambda region_ms, n=K_steps: world * sb * n / (region_ms * 1e-3) / 1e9
+        value = gbs(ms)
+        e2e = gbs(ms_host)
         achieved = sb / (kern_avg_ms * 1e-3) / 1e9
         pf_ms = float(np.median(prefill_ms))
         n_tok = sum(seq_lengths(cfg))
@@ -303,35 +313,125 @@ def run_ours(args):
                        "launch": ("programmatic dependent launch: each step's kernel may start while the previous step's drains"
                                   if overlap else "serialised launches"),
                        "l2": f"steps rotate over {n_caches} layer caches of {sb / 2**20:.0f} MiB each (> 126 MB L2)",
+                       "timing": f"value = median of {n_reg} timed regions of exactly {K_steps} steps, each from a drained stream "
+                                 "to a drained stream (barrier + synchronise on both sides), max over ranks per region",
                        "parallelism": f"replicas x{world} (independent batches, no collective)"},
+            "regions": {"count": n_reg, "median_ms": ms, "min_ms": ms_min, "max_ms": ms_max,
+                        "value_at_min_ms": gbs(ms_min), "value_at_max_ms": gbs(ms_max)},
             "tokens_per_s": world * B * K_steps / (ms * 1e-3), "seq_lens": seq_lengths(cfg) if cfg.get("ragged") else None,
             "frac_of_hbm_peak": value / world / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
             "frac_of_hbm_spec_8000": value / world / 8000.0,
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
+                    "regions": {"count": n_reg_host, "median_ms": ms_host, "min_ms": ms_host_min, "max_ms": ms_host_max},
                     "transfer": "q, k_new, v_new and out are pinned mapped HOST buffers handed to stief_decode_step_host: the kernel "
                                 "reads and writes them across the bus itself; the stream is synchronised after every step",
                     "tokens_per_s": world * B * K_steps / (ms_host * 1e-3)},
             "gpu_launches": K_steps,
             "roofline": {"bound": "hbm", "kernel": f"decode_persistent_kernel<{r_k},{r_v}>", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": peak_kind, "traffic": args.traffic,
+                         "traffic_source": args.traffic_source if args.traffic is not None else None,
                          "bytes_per_launch": sb, "avg_launch_ms": kern_avg_ms,
                          "isolated_launch_ms": kern_isolated_ms, "isolated_min_launch_ms": float(min(kern_ms)),
                          "isolated_frac": sb / (kern_isolated_ms * 1e-3) / 1e9 / hbm_peak},
-            "serial_launches": {"value": world * sb * K_steps / (ms_serial * 1e-3) / 1e9, "unit": UNIT,
-                                "ms_per_step": ms_serial / K_steps,
-                                "frac_of_hbm_peak": sb * K_steps / (ms_serial * 1e-3) / 1e9 / hbm_peak},
+            "serial_launches": {"value": gbs(ms_serial), "unit": UNIT, "ms_per_step": ms_serial / K_steps, "regions": n_reg_serial,
+                                "frac_of_hbm_peak": gbs(ms_serial) / world / hbm_peak},
+            "steady_state": {"what": f"ONE region of {n_long} back-to-back overlapped steps: the launch pipeline in steady state, "
+                                     "where the first launch's ramp and the last one's tail no longer count; not the headline",
+                             "steps": n_long, "ms_per_step": ms_long / n_long, "value": gbs(ms_long, n_long), "unit": UNIT,
+                             "frac_of_hbm_peak": gbs(ms_long, n_long) / world / hbm_peak},
             "prefill": {"ms_per_layer": pf_ms, "gbs": pf_bytes / (pf_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pf_bytes / (pf_ms * 1e-3) / 1e9 / hbm_peak,
                         "tflops": pf_flops / (pf_ms * 1e-3) / 1e12, "frac_of_bf16_peak": pf_flops / (pf_ms * 1e-3) / 1e12 / tf_peak,
                         "workload": f"K,V [B={B},T={T},Hkv={Hkv},128] bf16 -> paged cache; per-layer time over back-to-back "
                                     f"overlapped launches on {n_caches} layers",
                         "kernel": "prefill_tc_kernel (TMA + tcgen05/TMEM)", "bound": "hbm"},
-            "clocks": sampler.summary(t0, time.time()),
+            "clocks": sampler.summary(t0, t1),
         }
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=10.0)
+        if not args.no_cpu_baseline:
+            # world > 1: the other ranks wait in the final barrier meanwhile, so the sample is kept short
+            line["cpu_baseline"] = cpu_baseline(cfg, seconds_budget=10.0 if world == 1 else 3.0)
         print(json.dumps(line))
     R.finish(me)
+
+
+# ------------------------------------------------------------------------------------------------
+# where a lone decode launch spends its time: per-CTA time stamps written by the kernel itself
+# ------------------------------------------------------------------------------------------------
+def run_trace(args):
+    import paper_2601_21686_b200 as S
+    from paper_2601_21686_b200 import inputs as I
+    from paper_2601_21686_b200 import build as Bld
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Bld.build()
+    S.lib()
+    cfg = dict(SINGLE_LAYER[args.workload])
+    if args.ranks:
+        cfg["r_k"], cfg["r_v"] = (int(x) for x in args.ranks.split(","))
+    B, Hq, Hkv, T, r_k, r_v = (cfg[k] for k in ("B", "Hq", "Hkv", "T", "r_k", "r_v"))
+    n_caches = args.caches
+    layers, batch, status, _ = build_caches(cfg, n_caches, dev, S, I)
+    ns = args.num_parts or S.stief_decode_num_parts()
+    ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, Hkv, r_v, ns) // 4, dtype=torch.float32, device=dev)
+    S.stief_decode_workspace_init(ws)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    q = I.queries(SEED, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev)
+    k_new, v_new = I.new_token_kv(SEED, 0, B, Hkv, device=dev)
+    n = max(args.steps, 20)
+    for i in range(5):
+        S.stief_decode_step(layers[i % n_caches], batch, q, k_new, v_new, ws, out, num_parts=ns, status=status)
+    torch.cuda.synchronize()
+    names = ["entry", "partition known", "first page request", "first projections done", "first page landed", "last page request",
+             "last page consumed", "last partial stored", "last combine done", "exit"]
+    rel, dur_ev, spans, segs, combs = [], [], [], [], []
+    for i in range(n):
+        tr = torch.zeros(ns, S.TRACE_SLOTS, dtype=torch.int64, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); e1.record()
+        torch.cuda.synchronize()
+        S.stief_trace_next_decode_kernel(tr)
+        S.stief_time_next_decode_kernel(e0, e1)
+        S.stief_decode_step(layers[i % n_caches], batch, q, k_new, v_new, ws, out, num_parts=ns, status=status)
+        torch.cuda.synchronize()
+        t = tr.cpu().numpy().astype(np.float64)
+        stamps = t[:, :10]
+        t0 = stamps[:, 0].min()
+        r = np.where(stamps > 0, (stamps - t0) * 1e-3, np.nan)          # microseconds after the first CTA's entry
+        rel.append(r)
+        dur_ev.append(e0.elapsed_time(e1) * 1e3)
+        spans.append(np.nanmax(r[:, 9]))
+        segs.append(t[:, 10])
+        combs.append(t[:, 11])
+    assert int(status.item()) == 0
+    rel = np.stack(rel)                                                  # [launch, cta, slot]
+    if args.trace_dump:                                                  # per-CTA table of the last launch, one line per CTA
+        with open(args.trace_dump, "w") as f:
+            f.write("cta segments combines " + " ".join(n.replace(" ", "_") for n in names) + "\n")
+            for cta in range(ns):
+                f.write(f"{cta} {int(segs[-1][cta])} {int(combs[-1][cta])} " + " ".join(f"{x:.3f}" for x in rel[-1, cta]) + "\n")
+    hbm_peak, _, peak_kind = measured_peaks()
+    sb = step_bytes(cfg)
+    rows = {}
+    for k, name in enumerate(names):
+        x = rel[:, :, k]
+        rows[name] = {"median_over_ctas_us": float(np.nanmedian(np.nanmedian(x, axis=1))),
+                      "last_cta_us": float(np.nanmedian(np.nanmax(x, axis=1))),
+                      "first_cta_us": float(np.nanmedian(np.nanmin(x, axis=1)))}
+    print(json.dumps({
+        "what": "time stamps written by decode_persistent_kernel itself (GPU nanosecond timer), microseconds after the first CTA's "
+                "entry; one serialised launch at a time, median over launches; per point: median CTA, first CTA, last CTA",
+        "workload": cfg["name"], "launches": n, "num_parts": ns, "points": rows,
+        "kernel_span_us": float(np.median(spans)), "event_timed_launch_us": float(np.median(dur_ev)),
+        "outside_the_kernel_us": float(np.median(dur_ev) - np.median(spans)),
+        "roofline_time_us": sb / hbm_peak / 1e3, "peak_kind": peak_kind, "bytes_per_launch": sb,
+        "stream_phase_us": {"median_cta": float(np.nanmedian(rel[:, :, 6] - rel[:, :, 4])),
+                            "effective_gbs_over_first_landed_to_last_consumed":
+                                sb / (float(np.nanmedian(np.nanmax(rel[:, :, 6], axis=1) - np.nanmin(rel[:, :, 4], axis=1))) * 1e-6) / 1e9},
+        "segments_per_cta": {"mean": float(np.mean(segs)), "max": float(np.max(segs))},
+        "combines_per_cta": {"mean": float(np.mean(combs)), "max": float(np.max(combs))}}))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -362,7 +462,9 @@ def run_q8(args):
         U_k, U_v = I.stiefel_bases(SEED, l, Hkv, r_k, r_v)
         K = I.lowrank_keys(SEED, l, B, T, Hkv, device=dev)
         V = I.gaussian_kv(SEED, I.TAG_V, l, B, T, Hkv, device=dev)
-        # static key parameters: calibrated on this prompt's own projected keys (min / max per head and 64-channel group)
+        # CALIBRATION INPUT, outside every timed region: the static key parameters the caller must bring (min / max of
+        # the prompt's own projected keys per head and 64-channel group, widened by 25 %).  A real deployment takes
+        # them from calibration data; this einsum only manufactures that input and is no part of the measured path.
         Kd = torch.einsum("bthd,hdr->bthr", K.float(), U_k.to(dev).float())
         mn = Kd.reshape(B * T, Hkv, r_k // 64, 64).amin(dim=(0, 3))
         mx = Kd.reshape(B * T, Hkv, r_k // 64, 64).amax(dim=(0, 3))
@@ -748,7 +850,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 5000; 128 for config3)")
+    ap.add_argument("--steps", type=int, default=None, help="timed steps per region (default 20; 128 for config3)")
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4a", "config4b", "config5"],
@@ -761,20 +863,27 @@ def main():
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="launch every step's kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--caches", type=int, default=N_CACHES, help="independent layer caches the steps rotate over")
-    # DRAM read + write bytes per launch of decode_persistent_kernel<64,64> on config 2, from the ncu capture
-    # summarised in profiles/decode_persistent_kernel_config2.md (mean of two launches); null for other workloads
     ap.add_argument("--mq", action="store_true", help="measure the multi-query (chunked prefill) attention kernel on the config-2 shape")
     ap.add_argument("--n-q", dest="n_q", type=int, default=2048, help="query tokens per sequence for --mq")
     ap.add_argument("--splits", type=int, default=None, help="--mq: parts per page range (default: the library's proposal)")
     ap.add_argument("--rho", type=float, default=None, help="multi-layer workloads: take the per-layer ranks from stief_select_ranks at this cache ratio instead of the seeded random profile")
-    ap.add_argument("--traffic", type=float, default=None, help="dram bytes per launch of the split-T kernel from an ncu capture")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="dram bytes (read + write) per launch of the split-T kernel from an ncu capture of the CURRENT kernel; "
+                         "without it roofline.traffic is null")
+    ap.add_argument("--traffic-source", default=None, help="where --traffic comes from (profile file and commit of the capture)")
+    ap.add_argument("--trace", action="store_true",
+                    help="single-layer workloads: per-CTA time stamps of lone decode launches (where the time of a launch goes)")
+    ap.add_argument("--trace-dump", default=None, help="--trace: also write the last launch's per-CTA table to this file")
+    ap.add_argument("--seconds", type=float, default=0.6,
+                    help="device time to collect by repeating the K-step timed region (the median region is reported)")
+    ap.add_argument("--steady-steps", type=int, default=4000, help="steps of the one long region reported under steady_state")
     args = ap.parse_args()
-    if args.traffic is None and args.workload == "config2" and not args.ranks:
-        args.traffic = 271.70e6
     if args.steps is None:
-        args.steps = 128 if args.workload == "config3" else 5000
+        args.steps = 128 if args.workload == "config3" else (20 if not (args.q8 or args.mq) else 2000)
     if args.impl == "reference":
         run_reference(args)
+    elif args.trace:
+        run_trace(args)
     elif args.q8:
         run_q8(args)
     elif args.mq:

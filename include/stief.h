@@ -96,7 +96,9 @@ typedef struct stief_batch {
  * that precedes it on the stream has finished, so that the per-layer launches of one prompt run without
  * idle gaps.  By setting it the caller promises that the preceding kernel neither writes this call's
  * inputs (K, V, seq_lens, block_table, the bases) nor touches this layer's pools; consecutive calls for
- * different layers satisfy that.  The kernel still completes only after its predecessor has. */
+ * different layers satisfy that.  The kernel still completes only after its predecessor has.  The grid always has
+ * one CTA per SM and every CTA stays resident until the preceding kernel has completed, so in a run of flagged
+ * calls no more than two kernels overlap: the promise concerns the directly preceding kernel only. */
 #define STIEF_PREFILL_OVERLAP_PREVIOUS 1u
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K,
                            const uint16_t* V, int64_t stride_b, int64_t stride_t, int64_t v_stride_b,
@@ -151,7 +153,12 @@ int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* s
  * (q, k_new, v_new, seq_lens, block_table, the bases, this layer's pools) and does not read the cache
  * rows this call appends.  Two consecutive decode calls of this library on different layers satisfy
  * that; a call that follows stief_advance_seq_lens, or whose q is produced by the preceding kernel,
- * does not.  If the preceding stream operation is not a kernel the flag has no effect. */
+ * does not.  If the preceding stream operation is not a kernel the flag has no effect.
+ * Chains: the promise is about the ONE kernel directly before.  In an unbroken run of flagged calls at most two
+ * kernels are ever on the GPU together: a kernel's CTAs stay resident until the kernel before it has completed
+ * and each fills more than half of an SM, so the kernel after next cannot begin until the one before has gone.
+ * That argument needs a grid of at least one CTA per SM, so the flag is honoured only when num_parts is 0 or at
+ * least the SM count; with fewer parts the launch is silently serialised (same results, no overlap). */
 #define STIEF_DECODE_OVERLAP_PREVIOUS 1u
 
 /* Decode attention (Eq. 18 on the reconstructions of Eq. 7, one query row per head): q [B][Hq][128]
@@ -285,6 +292,17 @@ int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, co
  * cancels a pending request. */
 int stief_time_next_decode_kernel(void* start_event, void* stop_event);
 
+/* Measurement aid (no counterpart in the paper): the next stief_decode_attention / stief_decode_step /
+ * stief_decode_step_host call made by this host thread has its kernel write, per CTA, STIEF_TRACE_SLOTS 64-bit words
+ * into `trace` (device memory the caller has zeroed, 8-byte aligned, at least num_parts * STIEF_TRACE_SLOTS * 8 bytes,
+ * num_parts as resolved by stief_decode_num_parts when 0; a smaller buffer switches tracing off for that call).
+ * Words 0..9 are readings of the GPU's global nanosecond timer at fixed points of the CTA's life, 0 when a point was
+ * never reached: 0 entry, 1 partition known, 2 first page request issued, 3 first segment's projections done,
+ * 4 first page landed, 5 last page request issued, 6 last page consumed, 7 last partial stored, 8 last combine done,
+ * 9 exit; words 10, 11 count the CTA's segments and the unit merges it performed.  One-shot; NULL cancels. */
+#define STIEF_TRACE_SLOTS 16
+int stief_trace_next_decode_kernel(uint64_t* trace, size_t trace_bytes);
+
 /* ---- several causal query rows per head (chunked prefill, speculative decode) --------------------------------
  * App. A.1 of the paper: during prefilling Q has one row per prefix token and Eq. 18 holds per row; the layer being
  * a decoder layer, row i of sequence b sits at absolute position p = seq_lens[b] - q_len_b + i and attends the cached
@@ -350,6 +368,20 @@ typedef int (*stief_surface_fn)(void* ctx, int32_t layer, const int32_t* r_k_cho
 int stief_select_ranks(int32_t L, int32_t d_h, const int32_t* cand_k, int32_t n_k, const int32_t* cand_v, int32_t n_v,
                        double rho, const double* surfaces, stief_surface_fn surface, void* ctx, int32_t* r_k,
                        int32_t* r_v, double* spent, int32_t* failed_layer);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait inside the kernels -- on an
+ * mbarrier that an asynchronous copy or another warp completes, on a shared counter -- polls a limited number of
+ * times; when the limit is reached the CTA raises an abort flag that ends all its later waits at their next look at
+ * it, writes STIEF_ERR_TIMEOUT to the status word and runs on to its normal exit (results are then meaningless, the
+ * context stays healthy).  This call launches one small CTA that makes those very wait routines run out: an mbarrier
+ * that nobody completes is waited on with `poll_limit` polls (1 .. 2^20), then two more waits with the kernels' own
+ * limit must be cut short by the abort flag.  Nothing faults and nothing waits without limit.
+ *   status  device int32, zeroed by the caller: receives STIEF_ERR_TIMEOUT
+ *   report  device int32[8]: [0] first wait satisfied (expected 0), [1] its duration in SM clock cycles, [2] abort flag
+ *           after it (1), [3]/[4] and [5]/[6] the same pair for the two later waits (satisfied = 0, cycles small),
+ *           [7] 0x600d when the kernel reached its end
+ * Asynchronous on `stream`. */
+int stief_selftest_wait_limit(int32_t* status, int32_t* report, int32_t poll_limit, void* stream);
 
 const char* stief_status_string(int status);
 int stief_version(void);

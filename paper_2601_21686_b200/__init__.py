@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
             "stief_mq_num_splits": (I32, [I32, I32, I32, I32, I32]),
             "stief_mq_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
             "stief_select_ranks": (ctypes.c_int, [I32, I32, P, I32, P, I32, ctypes.c_double, P, _SURFACE_FN, P, P, P, P, P]),
+            "stief_selftest_wait_limit": (ctypes.c_int, [P, P, I32, P]),
+            "stief_trace_next_decode_kernel": (ctypes.c_int, [P, SZ]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -397,3 +399,22 @@ def stief_append_chunk(layer: Layer, batch: Batch, K: torch.Tensor, V: torch.Ten
     _check(lib().stief_append_chunk(ctypes.byref(layer.c()), ctypes.byref(batch.c()), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
                                     V.stride(0), V.stride(1), K.shape[1], _ptr(chunk_lens), 1 if ends_at_len else 0,
                                     _ptr(status), _stream()), "stief_append_chunk")
+
+
+def stief_selftest_wait_limit(status: torch.Tensor, report: torch.Tensor, poll_limit: int = 256):
+    """Run the kernels' bounded waits to their limit on purpose (see stief.h): status <- STIEF_ERR_TIMEOUT, report int32[8]."""
+    assert status.dtype == torch.int32 and report.dtype == torch.int32 and report.numel() >= 8
+    _check(lib().stief_selftest_wait_limit(_ptr(status), _ptr(report), poll_limit, _stream()), "stief_selftest_wait_limit")
+
+
+TRACE_SLOTS = 16
+
+
+def stief_trace_next_decode_kernel(trace: Optional[torch.Tensor]):
+    """Have the next decode call of this thread fill `trace` (zeroed int64 [num_parts, TRACE_SLOTS] on the device) with
+    per-CTA time stamps of the GPU's nanosecond timer (slot meanings in stief.h)."""
+    if trace is None:
+        _check(lib().stief_trace_next_decode_kernel(None, 0), "stief_trace_next_decode_kernel")
+        return
+    assert trace.dtype == torch.int64 and trace.is_contiguous()
+    _check(lib().stief_trace_next_decode_kernel(_ptr(trace), trace.numel() * 8), "stief_trace_next_decode_kernel")

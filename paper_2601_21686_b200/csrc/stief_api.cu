@@ -132,6 +132,8 @@ bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
 }
 
 thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+thread_local unsigned long long* g_trace = nullptr;       // one-shot: time-stamp record for the next decode kernel
+thread_local size_t g_trace_bytes = 0;
 
 // Device-visible alias of a host pointer when the memory is pinned and mapped into the device's address space
 // (cudaHostAlloc / cudaHostRegister under unified addressing), else nullptr.
@@ -172,7 +174,11 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
 
   DecodeLaunch dl;
   dl.n_cta = n_cta;
-  dl.overlap_previous = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0;
+  // The early start is only honoured for a grid that covers every SM.  A CTA of these kernels takes more than half of
+  // an SM's shared memory and stays resident until its predecessor grid has completed, so with >= one CTA per SM the
+  // grid after next cannot start before the grid before has left the GPU: at most two kernels of a chain overlap.  A
+  // smaller grid would let a third kernel in, which could append a row its pre-predecessor is still streaming.
+  dl.overlap_previous = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0 && n_cta >= sm_count();
   DecodeArgs& a = dl.args;
   a.L = to_dev(layer);
   a.Bt = host::to_dev(batch);
@@ -187,6 +193,12 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   a.len_add = len_add;
   a.QT = QT;
   a.status = status;
+  a.trace = nullptr;
+  if (g_trace != nullptr) {
+    if (g_trace_bytes >= (size_t)n_cta * kTraceSlots * sizeof(unsigned long long)) a.trace = g_trace;
+    g_trace = nullptr;
+    g_trace_bytes = 0;
+  }
 
   cudaEvent_t ev0 = g_ev_start, ev1 = g_ev_stop;
   g_ev_start = g_ev_stop = nullptr;
@@ -365,6 +377,13 @@ int stief_time_next_decode_kernel(void* start_event, void* stop_event) {
   if ((start_event == nullptr) != (stop_event == nullptr)) return STIEF_ERR_INVALID_ARG;
   g_ev_start = static_cast<cudaEvent_t>(start_event);
   g_ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return STIEF_OK;
+}
+
+int stief_trace_next_decode_kernel(uint64_t* trace, size_t trace_bytes) {
+  if (trace != nullptr && (trace_bytes == 0 || !aligned(trace, 8))) return STIEF_ERR_INVALID_ARG;
+  g_trace = reinterpret_cast<unsigned long long*>(trace);
+  g_trace_bytes = trace ? trace_bytes : 0;
   return STIEF_OK;
 }
 

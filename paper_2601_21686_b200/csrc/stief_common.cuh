@@ -57,15 +57,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` (shared memory) short-circuits every later wait of the CTA once one
 // wait has run out, so a lost copy can never hang the kernel: results are then garbage, the status
 // word says STIEF_ERR_TIMEOUT, and control flow continues to the normal exit.
+// `limit` is the number of polls after which the wait gives up (the kernels use the default; the wait-limit
+// self-test passes a small one).  Returns true when the barrier phase completed, false when the wait gave up.
 constexpr uint32_t kWaitSpins = 1u << 24;
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  for (uint32_t i = 0; i < kWaitSpins; ++i) {
-    if (mbar_try_wait(bar, parity)) return;
-    if ((i & 1023u) == 1023u && *abort_flag) return;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          uint32_t limit = kWaitSpins) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
   *abort_flag = 1;
   report(status, STIEF_ERR_TIMEOUT);
+  return false;
 }
 
 // The same bounded wait on the non-blocking form.  mbarrier.try_wait may park the thread for a while before it looks
@@ -81,13 +85,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  for (uint32_t i = 0; i < (kWaitSpins << 2); ++i) {
-    if (mbar_test_wait(bar, parity)) return;
-    if ((i & 4095u) == 4095u && *abort_flag) return;
+__device__ __forceinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                               uint32_t limit = kWaitSpins << 2) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if ((i & 4095u) == 4095u && *abort_flag) return false;
   }
   *abort_flag = 1;
   report(status, STIEF_ERR_TIMEOUT);
+  return false;
 }
 
 // Programmatic dependent launch.  launch_dependents lets the next kernel on the stream (if it was
@@ -98,13 +104,24 @@ __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontr
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Bounded wait until a shared-memory counter (written by other warps of the CTA after a fence) reaches `target`
-__device__ __forceinline__ void wait_count(volatile int* counter, int target, volatile int* abort_flag, int32_t* status) {
-  for (uint32_t i = 0; i < kWaitSpins; ++i) {
-    if (*counter >= target) return;
-    if ((i & 1023u) == 1023u && *abort_flag) return;
+__device__ __forceinline__ bool wait_count(volatile int* counter, int target, volatile int* abort_flag, int32_t* status,
+                                           uint32_t limit = kWaitSpins) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (*counter >= target) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
   *abort_flag = 1;
   report(status, STIEF_ERR_TIMEOUT);
+  return false;
+}
+
+// Measurement aid: one time stamp of the GPU-wide nanosecond timer into slot k of a per-CTA record (when tracing is on)
+__device__ __forceinline__ void stamp(unsigned long long* rec, int k) {
+  if (rec != nullptr) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    rec[k] = t;
+  }
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {

@@ -157,6 +157,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
   // The next kernel on the stream may take over each SM as soon as this grid's CTA leaves it.
   launch_dependents();
+  unsigned long long* const trc = a.trace ? a.trace + (size_t)c * kTraceSlots : nullptr;
+  if (tid == 0) stamp(trc, kTrEntry);
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(full_bar(s), 1);
@@ -170,6 +172,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const int pad = seg_pad_pages(RK, RV);
   build_page_prefix(pref, a.Bt, a.len_add, pad, c == 0 ? a.status : nullptr);   // ends with __syncthreads
 
+  if (tid == 0) stamp(trc, kTrPrefix);
   const int B = a.Bt.B, Hkv = a.L.Hkv, QT = a.QT, G = a.L.G;
   const int upb = Hkv * QT;
   const int total = pref[B] * upb;
@@ -192,6 +195,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
     int i_base = 0;            // pages of this CTA before the current segment
     int n_append = 0;          // appending segments of this CTA so far
+    bool issued = false;
     while (walk.next(seg)) {
       const int h = seg.j / QT;
       const int npg = seg.p1 - seg.p0;
@@ -232,12 +236,17 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 #pragma unroll
           for (int nb = 0; nb < TV::NB; ++nb)
             tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, TV::tma_x(nb), TV::tma_y(tile), full_bar(slot));
+          if (pw == 0) {
+            if (!issued) stamp(trc, kTrFirstIssue);
+            issued = true;
+          }
         }
         __syncwarp();
       }
       i_base += npg;
       if (wait_append) ++n_append;
     }
+    if (pw == 0 && lane == 0) stamp(trc, kTrLastIssue);
     return;
   }
 
@@ -258,8 +267,10 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   for (int np = 0; np < RV / 16; ++np) voff[np] = TV::chunk(l7 + ((lane >> 3) & 1) * 8, 2 * np + (lane >> 4));
 
   int i_base = 0;              // pages of this CTA before the current segment
+  int n_seg = 0, n_comb = 0;
 
   while (walk.next(seg)) {
+    ++n_seg;
     const int b = seg.b, h = seg.j / QT, qt = seg.j % QT;
     const int npg = seg.p1 - seg.p0;
     const int ng = min(kGroupTile, G - qt * kGroupTile);
@@ -368,6 +379,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       split_bf16(y.x, y.y, qa[ks][2], qa[ks][3]);
     }
 
+    if (tid == 0 && n_seg == 1) stamp(trc, kTrPrologue);
     float m = -INFINITY, l = 0.f;
     float o[RV / 8][4];
 #pragma unroll
@@ -381,6 +393,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       const int kw = (i_base + k) / NP;
       const int slot = pl * SPW + kw % SPW;
       mbar_wait(full_bar(slot), (kw / SPW) & 1, abort_flag, a.status);
+      if (tid == 0 && i_base + k == 0) stamp(trc, kTrFirstPage);
       const uint32_t kt = ring + slot * C::STAGE_BYTES;
       const uint32_t vt = kt + TK::BYTES;
       const bool tail = (seg.p0 + k == seg.npages - 1) && (last_valid < kPage);
@@ -469,6 +482,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       if (lane == 0) mbar_arrive(empty_bar(slot));
     }
     i_base += npg;
+    if (tid == 0) stamp(trc, kTrLastPage);                 // overwritten by every segment: the last one stays
 
     // ------------------------------------------------------------------ merge the warps of this segment
     l += __shfl_xor_sync(0xffffffffu, l, 1);
@@ -506,6 +520,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       if (j == 0) __stcg(a.partial_lse + (size_t)slot_id * kGroupTile + gg, (M + log2f(den)) * kLn2);
     }
 
+    if (tid == 0) stamp(trc, kTrPartial);
     // ------------------------------------------------------------------ the unit's last partial triggers the combine
     if (a.out != nullptr) {
       int first, last;
@@ -524,11 +539,13 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       }
       bar1(NT);
       if (*last_flag) {
+        ++n_comb;
         __threadfence();
         combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, un + kGroupTile * kD, tid, NT);
       }
     }
     bar1(NT);
+    if (tid == 0) stamp(trc, kTrCombined);
   }
 
   // units of empty sequences get their zero rows from CTA (u mod n_cta)
@@ -546,6 +563,11 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
   }
   grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
+  if (tid == 0 && trc) {
+    stamp(trc, kTrExit);
+    trc[kTrSegments] = (unsigned long long)n_seg;
+    trc[kTrCombines] = (unsigned long long)n_comb;
+  }
 }
 
 }  // namespace stief

@@ -19,6 +19,24 @@ struct DecodeArgs {
   int len_add;                   // tokens attended beyond seq_lens (1 when appending)
   int QT;                        // query tiles per KV head = ceil(G / 8)
   int32_t* status;
+  unsigned long long* trace;     // NULL, or [n_cta][kTraceSlots] time stamps (measurement aid, see stamp())
+};
+
+// Slots of the per-CTA time-stamp record (nanoseconds of the GPU's global timer; 0 = never reached).
+enum TraceSlot {
+  kTrEntry = 0,        // first instruction of the CTA
+  kTrPrefix = 1,       // page prefix sums built, partition known
+  kTrFirstIssue = 2,   // producer lane 0: first TMA request issued
+  kTrPrologue = 3,     // consumers: first segment's projections done, about to wait for pages
+  kTrFirstPage = 4,    // consumers (warp 0): first page tile landed
+  kTrLastIssue = 5,    // producer lane 0: last TMA request issued
+  kTrLastPage = 6,     // consumers (warp 0): last page of the last segment consumed
+  kTrPartial = 7,      // last segment's partial stored
+  kTrCombined = 8,     // after the (possible) combine of the last segment's unit
+  kTrExit = 9,         // after the final dependency wait
+  kTrSegments = 10,    // number of segments this CTA worked on (a count, not a time)
+  kTrCombines = 11,    // number of unit combines this CTA performed (a count)
+  kTraceSlots = 16
 };
 
 }  // namespace stief

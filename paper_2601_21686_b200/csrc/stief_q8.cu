@@ -237,7 +237,7 @@ static int run_q8_decode(const stief_qlayer* layer, const stief_batch* batch, co
   a.len_add = len_add;
   a.QT = QT;
   a.status = status;
-  const bool ov = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0;
+  const bool ov = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0 && n_cta >= host::sm_count();   // see run_decode: full grids only
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
   if (layer->r_k == 64 && layer->r_v == 64) e = launch_decode_q8<64, 64>(a, n_cta, ov, st);

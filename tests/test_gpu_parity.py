@@ -272,6 +272,41 @@ def test_overlapped_launches_match_serial_ones():
     U.check_out(res[1][7], ref)
 
 
+@pytest.mark.parametrize("num_parts", [3, 16])
+def test_flagged_chain_with_few_parts_over_two_caches_matches_serial(num_parts):
+    # A grid below the SM count would let a THIRD kernel of a flagged chain start while the first still streams:
+    # step i+2 works on the same cache as step i and rewrites the row step i appended.  The library serialises such
+    # launches, so every step must see exactly its own appended row: bit-equal to the serial run, step by step.
+    B, Hq, Hkv = 2, 8, 2
+    cs = [U.make_case(92 + j, B, Hq, Hkv, 64, 64, [4000, 2500], reserve=8, lowrank=True) for j in range(2)]
+    for c in cs:
+        S.stief_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    ws = U.workspace_for(cs[0], num_parts)
+    n_steps = 12
+    qs = [I.queries(92, 0, B, Hq, step=i).cuda() for i in range(n_steps)]
+    # the new token's key is made large so that whichever appended row a step reads dominates its output
+    kvs = [tuple((t * (8.0 if j == 0 else 1.0)).to(torch.bfloat16).cuda() for j, t in enumerate(I.new_token_kv(92, 0, B, Hkv, step=i)))
+           for i in range(n_steps)]
+    torch.cuda.synchronize()
+    pools0 = [(c.layer.k_pool.clone(), c.layer.v_pool.clone()) for c in cs]
+    res = {}
+    for flags in (0, S.STIEF_DECODE_OVERLAP_PREVIOUS):
+        for c, (kp, vp) in zip(cs, pools0):
+            c.layer.k_pool.copy_(kp)
+            c.layer.v_pool.copy_(vp)
+        torch.cuda.synchronize()
+        outs = [torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(n_steps)]
+        for i in range(n_steps):
+            c = cs[i % 2]
+            S.stief_decode_step(c.layer, c.batch, qs[i], kvs[i][0], kvs[i][1], ws, outs[i], num_parts=num_parts, status=c.status,
+                                flags=flags)
+        torch.cuda.synchronize()
+        assert int(cs[0].status.item()) == 0 and int(cs[1].status.item()) == 0
+        res[flags] = outs
+    for i, (a, b) in enumerate(zip(res[0], res[S.STIEF_DECODE_OVERLAP_PREVIOUS])):
+        assert torch.equal(a, b), f"step {i}"
+
+
 def test_overlapped_prefill_launches_match_serial_ones():
     # the per-layer prefill launches of one prompt, enqueued back to back with STIEF_PREFILL_OVERLAP_PREVIOUS
     B, Hq, Hkv = 2, 8, 2
