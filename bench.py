@@ -385,7 +385,7 @@ def run_trace(args):
         S.stief_decode_step(layers[i % n_caches], batch, q, k_new, v_new, ws, out, num_parts=ns, status=status)
     torch.cuda.synchronize()
     names = ["entry", "partition known", "first page request", "first projections done", "first page landed", "last page request",
-             "last page consumed", "last partial stored", "last combine done", "exit"]
+             "last page consumed", "last partial stored", "last combine done", "exit", "last arrival counted"]
     rel, dur_ev, spans, segs, combs = [], [], [], [], []
     for i in range(n):
         tr = torch.zeros(ns, S.TRACE_SLOTS, dtype=torch.int64, device=dev)
@@ -397,7 +397,7 @@ def run_trace(args):
         S.stief_decode_step(layers[i % n_caches], batch, q, k_new, v_new, ws, out, num_parts=ns, status=status)
         torch.cuda.synchronize()
         t = tr.cpu().numpy().astype(np.float64)
-        stamps = t[:, :10]
+        stamps = np.concatenate([t[:, :10], t[:, 12:13]], axis=1)
         t0 = stamps[:, 0].min()
         r = np.where(stamps > 0, (stamps - t0) * 1e-3, np.nan)          # microseconds after the first CTA's entry
         rel.append(r)

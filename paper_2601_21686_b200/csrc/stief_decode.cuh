@@ -50,17 +50,18 @@ struct DecodeCfg {
   static constexpr int THREADS = NT + NP * 32;           // + one producer warp per page lane
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
   // scratch after the ring
-  static constexpr int CTRL_BYTES = 512;                 // full[NS], empty[NS], append barrier, flags
-  static constexpr int PREF_BYTES = ((kMaxBatch + 1) * 4 + 127) / 128 * 128;
+  static constexpr int CTRL_BYTES = 384;                 // full[16], empty[16], flags
+  static constexpr int PREF_BYTES = ((kMaxBatch + 1) * 4 + 15) / 16 * 16;
   static constexpr int QP_BYTES = kGroupTile * kD * 4;   // q' fp32 [8][RK]
   static constexpr int ROWS_BYTES = 10 * kD * 4;         // vectors to project: 8 queries, the new key, the new value
-  static constexpr int RED_BYTES = NW * 9 * kD * 4;      // per-warp partial projections
-  static constexpr int UNION_BYTES = ROWS_BYTES + RED_BYTES;   // also: merge scratch [NW][8][RV]+[2][NW][8]; combine scratch [8][128]
+  static constexpr int RED_BYTES = NW * 10 * kD * 4;     // per-warp partial projections: 9 rows of the key side, 1 of the value side
+  static constexpr int NEW_BYTES = 2 * kD * 2;           // the appended key and value rows as stored (bf16)
+  static constexpr int UNION_BYTES = ROWS_BYTES + RED_BYTES + NEW_BYTES;   // front part also: merge scratch [NW][8][RV]+[2][NW][8]; combine scratch
   static constexpr int SMEM_BYTES = 1024 + RING_BYTES + CTRL_BYTES + PREF_BYTES + QP_BYTES + UNION_BYTES;
   static_assert(RK % 16 == 0 && RV % 16 == 0 && RK <= 128 && RV <= 128, "ranks are multiples of 16 up to 128");
   static_assert(SPW >= 1 && NS <= 16, "ring shape");
-  static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= UNION_BYTES, "merge scratch must fit");
-  static_assert(kCombineScratchFloats * 4 <= UNION_BYTES && NT >= 96, "combine scratch must fit; combine_unit wants >= 96 threads");
+  static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= ROWS_BYTES + RED_BYTES, "merge scratch must fit in front of the appended rows");
+  static_assert(kCombineScratchFloats * 4 <= UNION_BYTES && NT >= 128, "combine scratch must fit; combine_unit wants >= 128 threads");
   static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KiB shared memory of an SM");
 };
 
@@ -87,9 +88,9 @@ struct BasisSlice {
     }
   }
 
-  // red[(warp*9 + r)*128 + j] = this warp's share of sum_d rows[r][d] U[d][j], for the rows whose bit is
-  // set in row_mask (bit r <-> row r, r < 9)
-  __device__ __forceinline__ void contract(const float* rows, uint32_t row_mask, float* red, int warp, int lane) const {
+  // red[(warp*rpw + r)*128 + j] = this warp's share of sum_d rows[r][d] U[d][j], for the rows whose bit is
+  // set in row_mask (bit r <-> row r, r < 9); rpw = rows each warp keeps in `red`
+  __device__ __forceinline__ void contract(const float* rows, uint32_t row_mask, float* red, int warp, int lane, int rpw = 9) const {
 #pragma unroll
     for (int r = 0; r < 9; ++r) {
       if (!((row_mask >> r) & 1u)) continue;               // uniform over the CTA
@@ -113,7 +114,7 @@ struct BasisSlice {
 #pragma unroll
       for (int p = 0; p < NP; ++p) {
         const int cp = lane + 32 * p;
-        if (cp < R / 2) *reinterpret_cast<float2*>(red + (warp * 9 + r) * kD + 2 * cp) = make_float2(acc[p][0], acc[p][1]);
+        if (cp < R / 2) *reinterpret_cast<float2*>(red + (warp * rpw + r) * kD + 2 * cp) = make_float2(acc[p][0], acc[p][1]);
       }
     }
   }
@@ -121,10 +122,10 @@ struct BasisSlice {
 
 // sum over the warps' shares of (row r, column j)
 template <int NW>
-__device__ __forceinline__ float warp_shares(const float* red, int r, int j) {
+__device__ __forceinline__ float warp_shares(const float* red, int r, int j, int rpw = 9) {
   float s = 0.f;
 #pragma unroll
-  for (int w = 0; w < NW; ++w) s += red[(w * 9 + r) * kD + j];
+  for (int w = 0; w < NW; ++w) s += red[(w * rpw + r) * kD + j];
   return s;
 }
 
@@ -148,9 +149,10 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const uint32_t ctrl = ring + C::RING_BYTES;
   auto full_bar = [&](int s) { return ctrl + s * 8; };
   auto empty_bar = [&](int s) { return ctrl + (16 + s) * 8; };
-  volatile int* append_done = reinterpret_cast<volatile int*>(ctrl_ptr + 32 * 8);   // appending segments whose rows are stored
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);
+  volatile int* n_pending = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);   // segments whose arrival is not yet counted
+  constexpr int kMaxPending = 4;
+  int* pending = reinterpret_cast<int*>(ctrl_ptr + 34 * 8);                           // [kMaxPending][4]: b, j, first CTA or -1, segments
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -164,9 +166,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), HALF);
     }
-    *append_done = 0;
     *abort_flag = 0;
-    *last_flag = 0;
+    *n_pending = 0;
     mbar_fence_init();
   }
   const int pad = seg_pad_pages(RK, RV);
@@ -194,16 +195,10 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       tma_prefetch_desc(&tmV);
     }
     int i_base = 0;            // pages of this CTA before the current segment
-    int n_append = 0;          // appending segments of this CTA so far
     bool issued = false;
     while (walk.next(seg)) {
       const int h = seg.j / QT;
       const int npg = seg.p1 - seg.p0;
-      bool wait_append = false;
-      if (appending && seg.p1 == seg.npages) {
-        const int pos = a.Bt.seq_lens[seg.b];
-        wait_append = pos >= 0 && pos / kPage < a.Bt.max_pages;
-      }
       int tbl = 0, win = -1;
       for (int k = (pw - i_base % NP + NP) % NP; k < npg; k += NP) {
         if ((k >> 5) != win) {                             // block-table entries of a window of 32 pages, one per lane
@@ -221,12 +216,6 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         const int use = kw / SPW;
         if (lane == 0) {
           if (use > 0) mbar_wait(empty_bar(slot), (use - 1) & 1, abort_flag, a.status);
-          if (wait_append && k == npg - 1) {
-            // the sequence's last page receives the new token's rows from this CTA's consumers first
-            wait_count(append_done, n_append + 1, abort_flag, a.status);
-            __threadfence();
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-          }
           const uint32_t st = ring + slot * C::STAGE_BYTES;
           const int tile = page * Hkv + h;
           mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
@@ -244,7 +233,6 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         __syncwarp();
       }
       i_base += npg;
-      if (wait_append) ++n_append;
     }
     if (pw == 0 && lane == 0) stamp(trc, kTrLastIssue);
     return;
@@ -269,44 +257,81 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   int i_base = 0;              // pages of this CTA before the current segment
   int n_seg = 0, n_comb = 0;
 
+  // Counts the arrivals of the noted segments at their units and merges the units this CTA completed (see below).
+  auto settle = [&]() -> int {
+    const int np_ = *n_pending;
+    __threadfence();                                       // this thread's partial stores are visible GPU-wide
+    bar1(NT);
+    if (tid < np_) {
+      const int pb = pending[4 * tid], pj = pending[4 * tid + 1];
+      int first, last;
+      unit_cta_span(pref, upb, pad, P, pb, pj, &first, &last);
+      const int nseg = last - first + 1, u = pb * upb + pj;
+      int is_last = 1;
+      if (nseg > 1) {
+        const int prev = atomicAdd(a.counters + u, 1);
+        is_last = (prev == nseg - 1);
+        if (is_last) a.counters[u] = 0;                    // leave the counter clean for the next call
+      }
+      pending[4 * tid + 2] = is_last ? first : -1;
+      pending[4 * tid + 3] = nseg;
+    }
+    bar1(NT);
+    if (tid == 0) stamp(trc, kTrArrived);
+    int done = 0;
+    for (int e = 0; e < np_; ++e) {
+      const int first = pending[4 * e + 2];
+      if (first < 0) continue;                             // uniform over the CTA
+      const int pb = pending[4 * e], pj = pending[4 * e + 1], nseg = pending[4 * e + 3];
+      __threadfence();
+      combine_unit<RV>(a.L, pb, pj / QT, pj % QT, first + pb * upb + pj, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, tid, NT);
+      ++done;
+    }
+    bar1(NT);
+    if (tid == 0) *n_pending = 0;
+    bar1(NT);
+    return done;
+  };
+
   while (walk.next(seg)) {
     ++n_seg;
     const int b = seg.b, h = seg.j / QT, qt = seg.j % QT;
     const int npg = seg.p1 - seg.p0;
     const int ng = min(kGroupTile, G - qt * kGroupTile);
     const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
-    const int len_raw = a.Bt.seq_lens[b] + a.len_add;
-    const int len = min(max(len_raw, 0), seg.npages * kPage);
-    const int last_valid = len - (seg.npages - 1) * kPage;          // tokens in the sequence's last page (1..64)
+    const int pos_raw = a.Bt.seq_lens[b];                            // first use is well below: the load runs meanwhile
     const bool has_final = seg.p1 == seg.npages;
-    bool do_append = false;
-    size_t new_row = 0;
-    if (appending && has_final) {
-      const int pos = a.Bt.seq_lens[b];
-      if (pos >= 0 && pos / kPage < a.Bt.max_pages) {
-        do_append = true;                                            // the producer waits for our signal
-        const int page = a.Bt.block_table[(size_t)b * a.Bt.max_pages + pos / kPage];
-        if (page < 0 || page >= a.L.num_pages) {
-          new_row = ~(size_t)0;                                      // bad page: signal, but store nothing
-        } else {
-          new_row = ((size_t)page * Hkv + h) * kPage + (pos % kPage);
-        }
-      }
-    }
+    // This step's token is appended by the CTA whose segment holds the sequence's last page.  Its projected rows go to
+    // the pool for later steps; THIS step reads them from shared memory: the page tile arrives with whatever the pool
+    // held at that row and the consumer that owns the row overwrites it in the stage before use.  Nothing therefore
+    // waits for the stores to land, and the producers never wait for the consumers.
+    const bool may_append = appending && has_final;
+    // The page that will take the new rows: when a token is appended the sequence's last page is the one at index
+    // npages - 1 of its block table, which is known without waiting for seq_lens.  Every global load of the prologue
+    // is issued up front: one issued a microsecond later queues behind the page requests of the whole GPU.
+    int new_page = -1;
+    if (may_append) new_page = a.Bt.block_table[(size_t)b * a.Bt.max_pages + seg.npages - 1];
 
     // ---- prologue: q' = q U_k for the unit's queries (rows 0..7), the new key's row k U_k (row 8) and the
     // new value's row v U_v.  All global loads are issued before the first use of any of them.
     float* rows = un;                    // [9][128] fp32
     float* vrow = un + 9 * kD;           // [128]
     float* red = un + 10 * kD;           // [NW][9][128]
+    float* redv = red + NW * 9 * kD;     // [NW][128]
+    __nv_bfloat16* newk = reinterpret_cast<__nv_bfloat16*>(redv + NW * kD);   // [128] the appended key row as stored
+    __nv_bfloat16* newv = newk + kD;                                          // [128] the appended value row
     const __nv_bfloat16* Uk = a.L.U_k ? a.L.U_k + (size_t)h * a.L.uk_stride : nullptr;
     const __nv_bfloat16* Uv = a.L.U_v ? a.L.U_v + (size_t)h * a.L.uv_stride : nullptr;
-    const uint32_t row_mask = ((1u << ng) - 1u) | (do_append ? 0x100u : 0u);
+    const uint32_t row_mask = ((1u << ng) - 1u) | (may_append ? 0x100u : 0u);
     // a side without a basis is handled in its own dimension: its q / k (or v) rows arrive with r elements
     const int dk = Uk ? kD : RK, dv = Uv ? kD : RV;
+    bool do_append = false;
+    size_t new_row = ~(size_t)0;
     {
       BasisSlice<NW, RK> sk;
+      BasisSlice<NW, RV> sv;
       if (Uk) sk.load(Uk, warp, lane);
+      if (may_append && Uv) sv.load(Uv, warp, lane);
       // rows as 16-byte pieces: piece idx -> row idx / 16, elements 8 * (idx % 16) ..
       constexpr int NPC = (9 * 16 + NT - 1) / NT;
       uint4 pc[NPC];
@@ -316,11 +341,11 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         pc[i] = make_uint4(0u, 0u, 0u, 0u);
         if (8 * c < dk) {
           if (r < ng) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (head0 + r) * dk) + c);
-          else if (r == 8 && do_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * dk) + c);
+          else if (r == 8 && may_append) pc[i] = __ldg(reinterpret_cast<const uint4*>(a.k_new + ((size_t)b * Hkv + h) * dk) + c);
         }
       }
       uint4 pv = make_uint4(0u, 0u, 0u, 0u);
-      if (do_append && tid < 16 && 8 * tid < dv) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * dv) + tid);
+      if (may_append && tid < 16 && 8 * tid < dv) pv = __ldg(reinterpret_cast<const uint4*>(a.v_new + ((size_t)b * Hkv + h) * dv) + tid);
 #pragma unroll
       for (int i = 0; i < NPC; ++i) {
         const int idx = tid + i * NT;
@@ -330,16 +355,20 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
           for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(rows + idx * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
         }
       }
-      if (do_append && tid < 16) {
+      if (may_append && tid < 16) {
         const uint32_t w[4] = {pv.x, pv.y, pv.z, pv.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) *reinterpret_cast<float2*>(vrow + tid * 8 + 2 * e) = make_float2(bf16_lo(w[e]), bf16_hi(w[e]));
       }
+      // where the new rows go (pos_raw / 64 == npages - 1 unless the sequence outgrew its block table: then nothing is appended)
+      if (may_append && pos_raw >= 0 && pos_raw / kPage < a.Bt.max_pages && pos_raw / kPage == seg.npages - 1) {
+        do_append = true;
+        if (new_page >= 0 && new_page < a.L.num_pages) new_row = ((size_t)new_page * Hkv + h) * kPage + (pos_raw % kPage);
+      }
       bar1(NT);
       if (Uk) sk.contract(rows, row_mask, red, warp, lane);
+      if (may_append && Uv) sv.contract(vrow, 1u, redv, warp, lane, 1);      // the value row sits where row 0 is expected
     }
-    BasisSlice<NW, RV> sv;
-    if (do_append && Uv) sv.load(Uv, warp, lane);          // in flight while the key side is reduced
     bar1(NT);
     for (int idx = tid; idx < 9 * RK; idx += NT) {
       const int r = idx / RK, j = idx % RK;
@@ -348,26 +377,25 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         continue;
       }
       const float x = Uk ? warp_shares<NW>(red, r, j) : rows[r * kD + j];
-      if (r < 8) qp[r * RK + j] = x * qscale;
-      else if (new_row != ~(size_t)0) a.L.k_pool[new_row * RK + j] = __float2bfloat16_rn(x);
+      if (r < 8) {
+        qp[r * RK + j] = x * qscale;
+      } else {
+        const __nv_bfloat16 xb = __float2bfloat16_rn(x);
+        newk[j] = xb;
+        if (new_row != ~(size_t)0) a.L.k_pool[new_row * RK + j] = xb;
+      }
     }
-    if (do_append) {
-      bar1(NT);                                            // the key side has left `red`
-      if (Uv) {
-        // the value row sits where row 0 is expected: contract one row
-        sv.contract(vrow, 1u, red, warp, lane);
-        bar1(NT);
+    if (may_append) {
+      for (int j = tid; j < RV; j += NT) {
+        const __nv_bfloat16 xb = __float2bfloat16_rn(Uv ? warp_shares<NW>(redv, 0, j, 1) : vrow[j]);
+        newv[j] = xb;
+        if (new_row != ~(size_t)0) a.L.v_pool[new_row * RV + j] = xb;
       }
-      if (new_row != ~(size_t)0) {
-        for (int j = tid; j < RV; j += NT) a.L.v_pool[new_row * RV + j] = __float2bfloat16_rn(Uv ? warp_shares<NW>(red, 0, j) : vrow[j]);
-      } else if (tid == 0) {
-        report(a.status, STIEF_ERR_BOUNDS);
-      }
-      __threadfence();
-      asm volatile("fence.proxy.async.global;" ::: "memory");
+      if (do_append && new_row == ~(size_t)0 && tid == 0) report(a.status, STIEF_ERR_BOUNDS);
     }
     bar1(NT);
-    if (do_append && tid == 0) *append_done = *append_done + 1;       // rows are in the pool: the last page may be fetched
+    const int len = min(max(pos_raw + a.len_add, 0), seg.npages * kPage);
+    const int last_valid = len - (seg.npages - 1) * kPage;          // tokens in the sequence's last page (1..64)
 
     // A operand of the score MMA: rows 0-7 = bf16(q'), rows 8-15 = bf16(q' - bf16(q'))
     uint32_t qa[RK / 16][4];
@@ -396,11 +424,27 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       if (tid == 0 && i_base + k == 0) stamp(trc, kTrFirstPage);
       const uint32_t kt = ring + slot * C::STAGE_BYTES;
       const uint32_t vt = kt + TK::BYTES;
-      const bool tail = (seg.p0 + k == seg.npages - 1) && (last_valid < kPage);
+      const bool final_page = seg.p0 + k == seg.npages - 1;
+      const bool tail = final_page && (last_valid < kPage);
       if (HALF > 1 && tail && last_valid <= tb) {          // none of this warp's tokens exists: nothing to add
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar(slot));
         continue;
+      }
+
+      // this step's own token is the sequence's last one: its rows are put into the tile here (see the prologue)
+      const int tn = last_valid - 1;
+      const bool patch = do_append && final_page && tn >= tb && tn < tb + kPage / HALF;
+      if (patch) {
+        if (lane < RK / 8) {
+          const uint4 w = *reinterpret_cast<const uint4*>(newk + 8 * lane);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(kt + TK::chunk(tn, lane)), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+        }
+        if (lane < RV / 8) {
+          const uint4 w = *reinterpret_cast<const uint4*>(newv + 8 * lane);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(vt + TV::chunk(tn, lane)), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+        }
+        __syncwarp();
       }
 
       // ---- scores of the page: n-tile j covers tokens 8j..8j+7; c0,c1 from bf16(q'), c2,c3 from the remainder
@@ -477,7 +521,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         }
       }
 
-      if (tail) fence_proxy_async_smem();
+      if (tail || patch) fence_proxy_async_smem();          // generic-proxy writes to the stage before TMA refills it
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar(slot));
     }
@@ -522,29 +566,24 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
     if (tid == 0) stamp(trc, kTrPartial);
     // ------------------------------------------------------------------ the unit's last partial triggers the combine
+    // Counting the arrival means a fence and an atomic whose answer must come back: two trips through a memory system
+    // that is busy streaming pages.  Between segments that would stall the consumers while the ring fills up, so the
+    // segment is only noted here; the arrivals of all noted segments are counted together once the CTA has no pages left
+    // (or the list is full), one thread per segment, and whichever of them turn out to be last are merged then.
     if (a.out != nullptr) {
-      int first, last;
-      unit_cta_span(pref, upb, pad, P, b, seg.j, &first, &last);
-      const int nseg = last - first + 1;
-      __threadfence();
-      bar1(NT);
       if (tid == 0) {
-        int is_last = 1;
-        if (nseg > 1) {
-          const int prev = atomicAdd(a.counters + u, 1);
-          is_last = (prev == nseg - 1);
-          if (is_last) a.counters[u] = 0;                  // leave the counter clean for the next call
-        }
-        *last_flag = is_last;
+        int* e = pending + 4 * *n_pending;
+        e[0] = b; e[1] = seg.j;
+        *n_pending = *n_pending + 1;
       }
       bar1(NT);
-      if (*last_flag) {
-        ++n_comb;
-        __threadfence();
-        combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, un + kGroupTile * kD, tid, NT);
-      }
+      if (*n_pending == kMaxPending) n_comb += settle();
+    } else {
+      bar1(NT);
     }
-    bar1(NT);
+  }
+  if (a.out != nullptr) {
+    if (*n_pending > 0) n_comb += settle();
     if (tid == 0) stamp(trc, kTrCombined);
   }
 

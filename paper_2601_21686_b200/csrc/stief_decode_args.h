@@ -36,6 +36,7 @@ enum TraceSlot {
   kTrExit = 9,         // after the final dependency wait
   kTrSegments = 10,    // number of segments this CTA worked on (a count, not a time)
   kTrCombines = 11,    // number of unit combines this CTA performed (a count)
+  kTrArrived = 12,     // last segment: arrival at the unit's counter known (a time)
   kTraceSlots = 16
 };
 

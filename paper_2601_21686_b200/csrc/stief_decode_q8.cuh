@@ -560,7 +560,7 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       bar1(NT);
       if (*last_flag) {
         __threadfence();
-        combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, un + kGroupTile * kD, tid, NT, lse_shift);
+        combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, tid, NT, lse_shift);
       }
     }
     bar1(NT);

@@ -137,163 +137,155 @@ __device__ __forceinline__ void unit_cta_span(const int* pref, int upb, int pad,
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void bar1(int nt) { asm volatile("bar.sync 1, %0;" ::"r"(nt) : "memory"); }
 
-// The merge runs while other CTAs still stream the cache, so a dependent global load costs
-// microseconds.  Loads are therefore issued in bulk before anything waits on them: a thread's row of
-// U_v, the segments' log-sum-exps and the first kSegBatch segments' partials of every output element the
-// thread owns are all in flight together; a unit of up to kSegBatch segments costs one round trip.
-// `od` is shared scratch [8][128] floats, `wsm` shared scratch [kSegChunk][8] + 24 floats; nt >= 96.
+// The merge may run while other CTAs still stream the cache, when a dependent global load costs microseconds, so a
+// thread issues everything it needs at once: the log-sum-exps of up to kSegBatch segments of its row and those
+// segments' partials of the output elements it owns are all in flight together (one round trip for a unit of up to
+// kSegBatch segments; longer units loop with a running maximum).  Every thread of a row derives the row's weights by
+// itself from the same values in the same order, so there is nothing to exchange and the result does not depend on
+// the number of threads.  The back-projection o_down U_v^T runs on the tensor cores: the eight merged rows, split into
+// bf16 value + remainder (rows 0-7 / 8-15 of the A operand, ~16 significant bits), against U_v read from global memory
+// in the order the B fragments want it; warp w of the first four produces output columns 32 w .. 32 w + 31.
+// Called by nt >= 128 threads (a multiple of 32) that share barrier 1; `od` is shared scratch of kCombineScratchFloats.
 constexpr int kSegBatch = 8;       // segments whose partials a thread holds in registers at once
-constexpr int kSegChunk = 32;      // segments whose weights sit in shared memory at once
-constexpr int kCombineScratchFloats = kGroupTile * kD + kSegChunk * kGroupTile + 24;
+constexpr int kCombineScratchFloats = kGroupTile * (kD + 4);
 
 template <int RV>
 __device__ __forceinline__ void combine_unit(const LayerDev& L, int b, int h, int qt, int slot0, int nseg, const float* partial_o,
-                                             const float* partial_lse, __nv_bfloat16* out, float* out_lse, float* od, float* wsm,
+                                             const float* partial_lse, __nv_bfloat16* out, float* out_lse, float* od,
                                              int tid, int nt, const float* lse_shift = nullptr) {
   constexpr int NV = RV / 4;                               // float4 pieces per row
-  constexpr int IPT = 3;                                   // pieces per thread: 8 * NV <= 256 <= 3 * 96
+  constexpr int IPT = 2;                                   // pieces per thread: 8 * NV <= 256 = 2 * 128
+  constexpr int S = RV + 4;                                // row stride of od: keeps the 16-byte reads of phase 2 conflict-free
   const int G = L.G;
   const int ng = min(kGroupTile, G - qt * kGroupTile);
   const int n_items = ng * NV;
   const size_t head0 = (size_t)b * L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
   const __nv_bfloat16* Uv = L.U_v ? L.U_v + (size_t)h * L.uv_stride : nullptr;
-  float* Mrow = wsm + kSegChunk * kGroupTile;              // running max per row
-  float* Drow = Mrow + 8;                                  // running denominator per row
-  float* Srow = Drow + 8;                                  // rescale of what was accumulated before this chunk
+  const int warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tid4 = lane & 3;
 
-  // this thread's row of U_v for the back-projection (output column dd = tid)
-  uint4 urow[RV / 8];
-  if (Uv && tid < kD) {
+  // ---- phase 2's operand from global memory, requested first: warp w, n-tile t covers output columns 32 w + 8 t + gid;
+  // per 32 contraction indices a thread holds the 8 consecutive elements 32 q + 8 tid4 .. + 7 of its column's row of U_v
+  constexpr int QF = RV / 32, REM = RV % 32;               // full groups of 32, and a remainder of 16 (ranks 48)
+  uint4 ub[4][QF > 0 ? QF : 1];
+  uint32_t ur[4][2];
+  if (Uv && warp < 4) {
 #pragma unroll
-    for (int c = 0; c < RV / 8; ++c) urow[c] = __ldg(reinterpret_cast<const uint4*>(Uv + (size_t)tid * RV) + c);
+    for (int t = 0; t < 4; ++t) {
+      const __nv_bfloat16* row = Uv + (size_t)(32 * warp + 8 * t + gid) * RV;
+#pragma unroll
+      for (int q = 0; q < QF; ++q) ub[t][q] = __ldg(reinterpret_cast<const uint4*>(row + 32 * q + 8 * tid4));
+      if constexpr (REM != 0) {
+        ur[t][0] = __ldg(reinterpret_cast<const uint32_t*>(row + 32 * QF + 2 * tid4));
+        ur[t][1] = __ldg(reinterpret_cast<const uint32_t*>(row + 32 * QF + 8 + 2 * tid4));
+      }
+    }
   }
-  if (tid < 8) {
-    Mrow[tid] = -INFINITY;
-    Drow[tid] = 0.f;
-  }
+
+  // ---- phase 1: merge the segments (Eq. 18 re-associated over chunks of the token axis)
   float4 num[IPT];
+  float m_run[IPT], d_run[IPT];
 #pragma unroll
-  for (int i = 0; i < IPT; ++i) num[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-
-  for (int c0 = 0; c0 < nseg; c0 += kSegChunk) {
-    const int n = min(kSegChunk, nseg - c0);
-    const float* lse0 = partial_lse + (size_t)(slot0 + c0) * kGroupTile;       // n * 8 contiguous floats
-    const float4* po0 = reinterpret_cast<const float4*>(partial_o + (size_t)(slot0 + c0) * kGroupTile * RV);
-    float lv[IPT];
-#pragma unroll
-    for (int i = 0; i < IPT; ++i) {
-      const int idx = tid + i * nt;
-      lv[i] = idx < n * kGroupTile ? __ldcg(lse0 + idx) : 0.f;
-    }
-    float4 ov[IPT][kSegBatch];
-    auto fetch = [&](int k0) {
-#pragma unroll
-      for (int i = 0; i < IPT; ++i) {
-        const int item = tid + i * nt;
-#pragma unroll
-        for (int k = 0; k < kSegBatch; ++k) {
-          ov[i][k] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (item < n_items && k0 + k < n) ov[i][k] = __ldcg(po0 + (size_t)(k0 + k) * kGroupTile * NV + item);   // item = r * NV + j4
-        }
-      }
-    };
-    fetch(0);
-#pragma unroll
-    for (int i = 0; i < IPT; ++i) {
-      const int idx = tid + i * nt;
-      if (idx < n * kGroupTile) wsm[idx] = lv[i];
-    }
-    bar1(nt);
-    if (tid < 8) {
-      const float m_old = Mrow[tid];
-      float m = m_old;
-      for (int s = 0; s < n; ++s) m = fmaxf(m, wsm[s * kGroupTile + tid]);
-      float sc = 1.f, d = Drow[tid];
-      if (m > -INFINITY) {
-        sc = __expf(m_old - m);                            // 0 when nothing was accumulated before
-        d *= sc;
-        for (int s = 0; s < n; ++s) d += __expf(wsm[s * kGroupTile + tid] - m);
-      }
-      Mrow[tid] = m;
-      Drow[tid] = d;
-      Srow[tid] = sc;
-    }
-    bar1(nt);
-    for (int idx = tid; idx < n * kGroupTile; idx += nt) {
-      const float m = Mrow[idx % kGroupTile];
-      wsm[idx] = m > -INFINITY ? __expf(wsm[idx] - m) : 0.f;      // an empty segment (lse = -inf) weighs nothing
-    }
-    bar1(nt);
-    for (int k0 = 0; k0 < n; k0 += kSegBatch) {
-      if (k0 > 0) fetch(k0);
-#pragma unroll
-      for (int i = 0; i < IPT; ++i) {
-        const int item = tid + i * nt;
-        if (item >= n_items) continue;
-        const int r = item / NV;
-        if (k0 == 0) {
-          const float sc = Srow[r];
-          num[i].x *= sc; num[i].y *= sc; num[i].z *= sc; num[i].w *= sc;
-        }
-#pragma unroll
-        for (int k = 0; k < kSegBatch; ++k) {
-          if (k0 + k < n) {
-            const float w = wsm[(k0 + k) * kGroupTile + r];
-            num[i].x = fmaf(w, ov[i][k].x, num[i].x);
-            num[i].y = fmaf(w, ov[i][k].y, num[i].y);
-            num[i].z = fmaf(w, ov[i][k].z, num[i].z);
-            num[i].w = fmaf(w, ov[i][k].w, num[i].w);
-          }
-        }
-      }
-    }
-    bar1(nt);                                              // the next chunk overwrites wsm
+  for (int i = 0; i < IPT; ++i) {
+    num[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    m_run[i] = -INFINITY;
+    d_run[i] = 0.f;
   }
-  if (nseg <= 0) bar1(nt);                                 // Mrow/Drow initialised above must be visible
+  for (int k0 = 0; k0 < nseg; k0 += kSegBatch) {
+    float lv[IPT][kSegBatch];
+    float4 ov[IPT][kSegBatch];
+#pragma unroll
+    for (int i = 0; i < IPT; ++i) {
+      const int item = tid + i * nt;                       // item = r * NV + j4
+      const int r = item / NV;
+#pragma unroll
+      for (int k = 0; k < kSegBatch; ++k) {
+        lv[i][k] = -INFINITY;
+        ov[i][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (item < n_items && k0 + k < nseg) {
+          lv[i][k] = __ldcg(partial_lse + (size_t)(slot0 + k0 + k) * kGroupTile + r);
+          ov[i][k] = __ldcg(reinterpret_cast<const float4*>(partial_o + (size_t)(slot0 + k0 + k) * kGroupTile * RV) + item);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < IPT; ++i) {
+      float m = m_run[i];
+#pragma unroll
+      for (int k = 0; k < kSegBatch; ++k) m = fmaxf(m, lv[i][k]);
+      if (m > -INFINITY) {                                 // else: nothing but empty segments so far
+        const float sc = __expf(m_run[i] - m);             // 0 when nothing was accumulated before
+        num[i].x *= sc; num[i].y *= sc; num[i].z *= sc; num[i].w *= sc;
+        float d = d_run[i] * sc;
+#pragma unroll
+        for (int k = 0; k < kSegBatch; ++k) {
+          const float w = __expf(lv[i][k] - m);            // an empty segment (lse = -inf) weighs nothing
+          d += w;
+          num[i].x = fmaf(w, ov[i][k].x, num[i].x);
+          num[i].y = fmaf(w, ov[i][k].y, num[i].y);
+          num[i].z = fmaf(w, ov[i][k].z, num[i].z);
+          num[i].w = fmaf(w, ov[i][k].w, num[i].w);
+        }
+        d_run[i] = d;
+        m_run[i] = m;
+      }
+    }
+  }
 #pragma unroll
   for (int i = 0; i < IPT; ++i) {
     const int item = tid + i * nt;
     if (item < n_items) {
       const int r = item / NV, j4 = item % NV;
-      const float den = Drow[r];
-      const float inv = den > 0.f ? 1.f / den : 0.f;
-      *reinterpret_cast<float4*>(od + r * kD + 4 * j4) = make_float4(num[i].x * inv, num[i].y * inv, num[i].z * inv, num[i].w * inv);
+      const float inv = d_run[i] > 0.f ? 1.f / d_run[i] : 0.f;
+      *reinterpret_cast<float4*>(od + r * S + 4 * j4) = make_float4(num[i].x * inv, num[i].y * inv, num[i].z * inv, num[i].w * inv);
+      // lse_shift: a per-row constant that was left out of every score of the unit (it cancels in the softmax)
+      if (j4 == 0 && out_lse)
+        out_lse[head0 + r] = d_run[i] > 0.f ? m_run[i] + __logf(d_run[i]) + (lse_shift ? lse_shift[r] : 0.f) : -INFINITY;
     }
   }
-  // lse_shift: a per-row constant that was left out of every score of the unit (it cancels in the softmax)
-  if (tid < ng && out_lse)
-    out_lse[head0 + tid] = Drow[tid] > 0.f ? Mrow[tid] + __logf(Drow[tid]) + (lse_shift ? lse_shift[tid] : 0.f) : -INFINITY;
+  for (int idx = tid; idx < (kGroupTile - ng) * RV; idx += nt) od[(ng + idx / RV) * S + idx % RV] = 0.f;   // rows without a query head
   bar1(nt);
-  const int d_out = Uv ? kD : RV;                           // without a value basis the output stays in the compressed space
-  for (int dd = tid; dd < d_out; dd += nt) {
-    float acc[kGroupTile];
+
+  // ---- phase 2: back-projection (Eq. 7 applied to the mixed values), or the compressed rows as they are
+  if (Uv) {
+    if (warp < 4) {
+      float acc[4][4];
 #pragma unroll
-    for (int r = 0; r < kGroupTile; ++r) acc[r] = 0.f;
-    if (Uv) {
-      if (dd != tid) {                                      // second pass of a CTA with fewer than 128 threads
+      for (int t = 0; t < 4; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
+      const float* orow = od + gid * S;
 #pragma unroll
-        for (int c = 0; c < RV / 8; ++c) urow[c] = __ldg(reinterpret_cast<const uint4*>(Uv + (size_t)dd * RV) + c);
-      }
+      for (int q = 0; q < QF; ++q) {
+        const float4 x0 = *reinterpret_cast<const float4*>(orow + 32 * q + 8 * tid4);
+        const float4 x1 = *reinterpret_cast<const float4*>(orow + 32 * q + 8 * tid4 + 4);
+        uint32_t a0[4], a1[4];                             // rows 0-7: value, rows 8-15: remainder
+        split_bf16(x0.x, x0.y, a0[0], a0[1]);
+        split_bf16(x0.z, x0.w, a0[2], a0[3]);
+        split_bf16(x1.x, x1.y, a1[0], a1[1]);
+        split_bf16(x1.z, x1.w, a1[2], a1[3]);
 #pragma unroll
-      for (int c = 0; c < RV / 8; ++c) {
-        const uint32_t w[4] = {urow[c].x, urow[c].y, urow[c].z, urow[c].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float u0 = bf16_lo(w[e]), u1 = bf16_hi(w[e]);
-#pragma unroll
-          for (int r = 0; r < kGroupTile; ++r) {
-            acc[r] = fmaf(od[r * kD + 8 * c + 2 * e], u0, acc[r]);
-            acc[r] = fmaf(od[r * kD + 8 * c + 2 * e + 1], u1, acc[r]);
-          }
+        for (int t = 0; t < 4; ++t) {
+          mma_bf16(acc[t], a0, ub[t][q].x, ub[t][q].y);
+          mma_bf16(acc[t], a1, ub[t][q].z, ub[t][q].w);
         }
       }
-    } else {
+      if constexpr (REM != 0) {
+        const float2 x0 = *reinterpret_cast<const float2*>(orow + 32 * QF + 2 * tid4);
+        const float2 x1 = *reinterpret_cast<const float2*>(orow + 32 * QF + 8 + 2 * tid4);
+        uint32_t a0[4];
+        split_bf16(x0.x, x0.y, a0[0], a0[1]);
+        split_bf16(x1.x, x1.y, a0[2], a0[3]);
 #pragma unroll
-      for (int r = 0; r < kGroupTile; ++r) acc[r] = od[r * kD + dd];
+        for (int t = 0; t < 4; ++t) mma_bf16(acc[t], a0, ur[t][0], ur[t][1]);
+      }
+      if (gid < ng) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int dd = 32 * warp + 8 * t + 2 * tid4;     // accumulator columns 2 tid4, 2 tid4 + 1 of row gid (value) and gid + 8 (remainder)
+          *reinterpret_cast<uint32_t*>(out + (head0 + gid) * kD + dd) = pack_bf16(acc[t][0] + acc[t][2], acc[t][1] + acc[t][3]);
+        }
+      }
     }
-#pragma unroll
-    for (int r = 0; r < kGroupTile; ++r)
-      if (r < ng) out[(head0 + r) * d_out + dd] = __float2bfloat16_rn(acc[r]);
+  } else {
+    for (int idx = tid; idx < ng * RV; idx += nt) out[(head0 + idx / RV) * RV + idx % RV] = __float2bfloat16_rn(od[(idx / RV) * S + idx % RV]);
   }
   bar1(nt);
 }

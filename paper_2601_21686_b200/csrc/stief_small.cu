@@ -149,11 +149,11 @@ combine_kernel(const CombineArgs a) {
   }
   const int slot0 = first + b * upb + j;
   switch (a.L.r_v) {
-    case 32: combine_unit<32>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
-    case 48: combine_unit<48>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
-    case 64: combine_unit<64>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
-    case 96: combine_unit<96>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
-    case 128: combine_unit<128>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, od + kGroupTile * kD, threadIdx.x, kCombThreads); break;
+    case 32: combine_unit<32>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads); break;
+    case 48: combine_unit<48>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads); break;
+    case 64: combine_unit<64>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads); break;
+    case 96: combine_unit<96>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads); break;
+    case 128: combine_unit<128>(a.L, b, h, qt, slot0, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, od, threadIdx.x, kCombThreads); break;
     default: break;
   }
 }
