@@ -435,9 +435,9 @@ def run_trace(args):
 
 
 # ------------------------------------------------------------------------------------------------
-# config 2 on the 8-bit quantised cache (a measurement case, not the headline line)
+# config 2 on the integer-quantised cache, 8-bit or 4-bit codes (a measurement case, not the headline line)
 # ------------------------------------------------------------------------------------------------
-def run_q8(args):
+def run_quant(args, bits):
     import paper_2601_21686_b200 as S
     from paper_2601_21686_b200 import inputs as I
     from paper_2601_21686_b200 import build as Bld
@@ -466,15 +466,16 @@ def run_q8(args):
         # the prompt's own projected keys per head and 64-channel group, widened by 25 %).  A real deployment takes
         # them from calibration data; this einsum only manufactures that input and is no part of the measured path.
         Kd = torch.einsum("bthd,hdr->bthr", K.float(), U_k.to(dev).float())
-        mn = Kd.reshape(B * T, Hkv, r_k // 64, 64).amin(dim=(0, 3))
-        mx = Kd.reshape(B * T, Hkv, r_k // 64, 64).amax(dim=(0, 3))
-        kpar = torch.stack([(mx - mn) * 1.25 / 255.0, mn * 1.25], -1).contiguous()
+        groups = [(lo, min(lo + 64, r_k)) for lo in range(0, r_k, 64)]
+        mn = torch.stack([Kd[..., lo:hi].amin(dim=(0, 1, 3)) for lo, hi in groups], -1)       # [Hkv, groups]
+        mx = torch.stack([Kd[..., lo:hi].amax(dim=(0, 1, 3)) for lo, hi in groups], -1)
+        kpar = torch.stack([(mx - mn) * 1.25 / float(2 ** bits - 1), mn * 1.25], -1).contiguous()
         del Kd
         layers.append(S.QLayer(Hq, Hkv, r_k, r_v, U_k.to(dev), U_v.to(dev), kpar,
-                               torch.zeros(pg.num_pages, Hkv, 64, r_k, dtype=torch.uint8, device=dev),
-                               torch.zeros(pg.num_pages, Hkv, r_v, 64, dtype=torch.uint8, device=dev),
-                               torch.zeros(pg.num_pages, Hkv, 64, r_v // 64, 2, dtype=torch.float32, device=dev)))
-        S.stief_q8_prefill_compress(layers[l], batch, K, V, status=status)
+                               torch.zeros(pg.num_pages, Hkv, 64, S.qkey_row_bytes(r_k, bits), dtype=torch.uint8, device=dev),
+                               torch.zeros(pg.num_pages, Hkv, r_v, 64 if bits == 8 else 32, dtype=torch.uint8, device=dev),
+                               torch.zeros(pg.num_pages, Hkv, 64, S.qgroups(r_v), 2, dtype=torch.float32, device=dev)))
+        S.stief_q_prefill_compress(bits, layers[l], batch, K, V, status=status)
         inputs.append((K, V))
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -482,7 +483,7 @@ def run_q8(args):
     e0.record()
     for r in range(reps):
         for l in range(n_caches):
-            S.stief_q8_prefill_compress(layers[l], batch, inputs[l][0], inputs[l][1], status=status,
+            S.stief_q_prefill_compress(bits, layers[l], batch, inputs[l][0], inputs[l][1], status=status,
                                         flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if (r or l) else 0)
     e1.record()
     torch.cuda.synchronize()
@@ -498,7 +499,7 @@ def run_q8(args):
     overlap = S.STIEF_DECODE_OVERLAP_PREVIOUS if (args.overlap and n_caches >= 2) else 0
 
     def step(i):
-        S.stief_q8_decode_step(layers[i % n_caches], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
+        S.stief_q_decode_step(bits, layers[i % n_caches], batch, qs[i % n_in], kvs[i % n_in][0], kvs[i % n_in][1], ws, out,
                                status=status, flags=overlap)
 
     K_steps, W = min(args.steps, 2000), max(args.warmup, 3)
@@ -512,15 +513,15 @@ def run_q8(args):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     assert int(status.item()) == 0, f"device status {int(status.item())}"
-    per_unit = r_k + r_v + 8 * (r_v // 64)
+    per_unit = S.qkey_row_bytes(r_k, bits) + r_v * bits // 8 + 8 * S.qgroups(r_v)
     sb = B * Hkv * (T + 1) * per_unit
     gbs = sb * K_steps / (ms * 1e-3) / 1e9
     pf_bytes = B * T * Hkv * (2 * 128 * 2 + per_unit)
     print(json.dumps({
-        "metric": "q8_decode_attn_effective_hbm_gbs", "value": gbs, "unit": UNIT, "n_gpus": 1, "steps": K_steps, "warmup": W,
-        "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
-        "dtype_note": "8-bit codes expanded to bf16 tensor-core operands, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": cfg["name"] + f" on the 8-bit quantised cache ({per_unit} bytes per token and KV head instead of {2 * (r_k + r_v)}); "
+        "metric": f"q{bits}_decode_attn_effective_hbm_gbs", "value": gbs, "unit": UNIT, "n_gpus": 1, "steps": K_steps, "warmup": W,
+        "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": f"u{bits}",
+        "dtype_note": f"{bits}-bit codes as integer tensor-core operands (s8 x u8 -> s32), fp32 softmax and accumulation", "data": "synthetic",
+        "config": {"workload": cfg["name"] + f" on the {bits}-bit quantised cache ({per_unit} bytes per token and KV head instead of {2 * (r_k + r_v)}); "
                                "step = append + query projection + split-T attention + combine, one launch"
                                + (", overlapped launches" if overlap else ""), "l2": f"steps rotate over {n_caches} layer caches"},
         "tokens_per_s": B * K_steps / (ms * 1e-3), "frac_of_hbm_peak": gbs / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
@@ -858,6 +859,7 @@ def main():
     ap.add_argument("--num-parts", type=int, default=0, help="CTAs of the persistent decode kernel (0 = one per SM)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--q8", action="store_true", help="config 2 on the 8-bit quantised cache (measurement case)")
+    ap.add_argument("--q4", action="store_true", help="config 2 on the 4-bit quantised cache (measurement case)")
     ap.add_argument("--ranks", default=None, help="r_k,r_v override for the single-layer workloads, e.g. 48,96")
     ap.add_argument("--layers", type=int, default=32, help="layers of the multi-layer workloads (config3, config5)")
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
@@ -879,13 +881,13 @@ def main():
     ap.add_argument("--steady-steps", type=int, default=4000, help="steps of the one long region reported under steady_state")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 128 if args.workload == "config3" else (20 if not (args.q8 or args.mq) else 2000)
+        args.steps = 128 if args.workload == "config3" else (20 if not (args.q8 or args.q4 or args.mq) else 2000)
     if args.impl == "reference":
         run_reference(args)
     elif args.trace:
         run_trace(args)
-    elif args.q8:
-        run_q8(args)
+    elif args.q8 or args.q4:
+        run_quant(args, 8 if args.q8 else 4)
     elif args.mq:
         run_mq(args)
     elif args.workload in SINGLE_LAYER:

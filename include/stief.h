@@ -231,22 +231,34 @@ int stief_decode_attention_static(const stief_layer* layer, const stief_batch* b
                                   int32_t* status, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
- * 8-bit quantised compressed cache (paper Sec. 4.3: asymmetric integer quantisation of the compressed cache
- * tensors, group size 64; keys use group-wise parameters shared across batch and sequence positions within a
- * KV head, values use token-wise group parameters).
- * A group is 64 consecutive channels of the compressed dimension; a code c in 0..255 stands for
- * c * scale + zero.  Key parameters are fixed ahead of time (calibration) per KV head and channel group and
- * given by the caller; a key outside the calibrated range is clamped.  Value parameters are computed from each
- * row when it is written: zero = min, scale = (max - min) / 255 over the group (scale = 1 when max == min).
- * The quantiser sees the projection K U_k / V U_v in fp32 (not rounded to bf16 first) and decides in fp32:
- * code = clamp(rint((x - zero) * (1 / scale))), ties to even.  Ranks must be 64 or 128 and both bases given.
- * Layout: k_codes [num_pages][Hkv][64][r_k] uint8, r fastest, indexed like the bf16 pools; v_codes
- * [num_pages][Hkv][r_v][64] uint8, CHANNEL-major inside a page, and token t of the page sits at position
- * (t & ~15) + 4*((t & 7) >> 1) + (t & 1) + 2*((t >> 3) & 1) of its channel rows (the order in which the
- * tensor-core mix consumes tokens: raw codes are its operands, nothing is expanded in shared memory);
- * k_params [Hkv][r_k / 64][2] fp32 (scale, zero); v_params [num_pages][Hkv][64][r_v / 64][2] fp32 (scale, zero).
- * Alignment: code pools and v_params 128 bytes, k_params 8 bytes.  Bytes per cached (token, KV head):
- * r_k + r_v + 8 * (r_v / 64), against 2 (r_k + r_v) for the bf16 cache. */
+ * Integer-quantised compressed cache, 8-bit (stief_q8_*) and 4-bit (stief_q4_*) codes (paper Sec. 4.3: asymmetric
+ * integer quantisation of the compressed cache tensors, group size 64; keys use group-wise parameters shared across
+ * batch and sequence positions within a KV head, values use token-wise group parameters).
+ * A group is 64 consecutive channels of the compressed dimension; the last group of ranks 32, 48 and 96 is shorter
+ * (32, 48 and 32 channels).  groups(r) = ceil(r / 64).  A b-bit code c in 0 .. 2^b - 1 stands for c * scale + zero.
+ * Key parameters are fixed ahead of time (calibration) per KV head and channel group and given by the caller; a key
+ * outside the calibrated range is clamped.  Value parameters are computed from each row when it is written:
+ * zero = min, scale = (max - min) / (2^b - 1) over the group (scale = 1 when max == min).  The quantiser sees the
+ * projection K U_k / V U_v in fp32 (not rounded to bf16 first) and decides in fp32:
+ * code = clamp(rint((x - zero) * (1 / scale))), ties to even.  All ranks 32, 48, 64, 96, 128; both bases must be given
+ * (a side whose projection is folded into the model's linear layers is not taken: STIEF_ERR_UNSUPPORTED).
+ *
+ * Layout, 8-bit codes:
+ *   k_codes [num_pages][Hkv][64][r_k] uint8, r fastest, indexed like the bf16 pools;
+ *   v_codes [num_pages][Hkv][r_v][64] uint8, CHANNEL-major inside a page, and token t of the page sits at position
+ *           pos(t) = (t & ~15) + 4*((t & 7) >> 1) + (t & 1) + 2*((t >> 3) & 1) of its channel rows (the order in which
+ *           the tensor-core mix consumes tokens: raw codes are its operands, nothing is expanded in shared memory).
+ * Layout, 4-bit codes (two to a byte; within every 32 consecutive indices i of a row, byte i % 16 of that block of 16
+ * bytes holds index i in its low nibble when i % 32 < 16 and in its high nibble otherwise):
+ *   k_codes [num_pages][Hkv][64][krow] bytes, the index being the channel; krow = r_k / 2, except r_k = 48: the row is
+ *           padded to 64 nibbles, krow = 32, unused nibbles zero;
+ *   v_codes [num_pages][Hkv][r_v][32] bytes, channel-major, the index being the position pos(t) above (so tokens whose
+ *           positions differ by 16 inside a block of 32 share a byte).
+ * Parameters, both widths: k_params [Hkv][groups(r_k)][2] fp32 (scale, zero);
+ *   v_params [num_pages][Hkv][64][groups(r_v)][2] fp32 (scale, zero), token-major.
+ * Alignment: code pools and v_params 128 bytes, k_params 8 bytes.  Bytes per cached (token, KV head): 8-bit
+ * r_k + r_v + 8 groups(r_v); 4-bit krow + r_v / 2 + 8 groups(r_v); against 2 (r_k + r_v) for the bf16 cache.
+ * Codes, bytes and nibbles of positions at or beyond a sequence's length are unspecified and never influence a result. */
 typedef struct stief_qlayer {
   int32_t Hq, Hkv, d;
   int32_t r_k, r_v;
@@ -265,23 +277,35 @@ typedef struct stief_qlayer {
 int stief_q8_prefill_compress(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* K,
                               const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
                               uint32_t flags, int32_t* status, void* stream);
+int stief_q4_prefill_compress(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* K,
+                              const uint16_t* V, int64_t stride_b, int64_t stride_t, int32_t T_max,
+                              uint32_t flags, int32_t* status, void* stream);
 
 /* One new token per sequence: projects, quantises and stores k_new, v_new at position seq_lens[b]. */
 int stief_q8_append(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* k_new,
+                    const uint16_t* v_new, int32_t* status, void* stream);
+int stief_q4_append(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* k_new,
                     const uint16_t* v_new, int32_t* status, void* stream);
 
 /* Decode attention on the quantised cache: ordinary attention (Eq. 18) on the reconstructions (Eq. 7) of the
  * DEQUANTISED cache, evaluated in the compressed space (the key scale folds into the projected query, the
  * key zero-point shifts every score of a row by the same amount and so only enters out_lse).  Arguments,
- * workspace (stief_decode_workspace_bytes with the same r_v) and flags as stief_decode_attention. */
+ * workspace (stief_decode_workspace_bytes with the same r_v) and flags as stief_decode_attention; num_parts = 0
+ * means one part per SM. */
 int stief_q8_decode_attention(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q,
+                              int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
+                              uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+int stief_q4_decode_attention(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q,
                               int32_t len_add, void* workspace, size_t workspace_bytes, int32_t num_parts,
                               uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
 
 /* One decode step of one layer on the quantised cache in one launch: project, quantise and store (k_new, v_new)
- * at position seq_lens[b], then attend over seq_lens[b] + 1 tokens.  Same result as stief_q8_append followed by
- * stief_q8_decode_attention with len_add = 1. */
+ * at position seq_lens[b], then attend over seq_lens[b] + 1 tokens.  Same result as the append call followed by the
+ * attention call with len_add = 1. */
 int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
+                         const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts,
+                         uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
+int stief_q4_decode_step(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
                          const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts,
                          uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);
 

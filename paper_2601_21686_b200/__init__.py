@@ -88,6 +88,10 @@ def lib() -> ctypes.CDLL:
             "stief_q8_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
             "stief_q8_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
             "stief_q8_decode_step": (ctypes.c_int, [QP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
+            "stief_q4_prefill_compress": (ctypes.c_int, [QP, BP, P, P, I64, I64, I32, U32, P, P]),
+            "stief_q4_append": (ctypes.c_int, [QP, BP, P, P, P, P]),
+            "stief_q4_decode_attention": (ctypes.c_int, [QP, BP, P, I32, P, SZ, I32, P, P, U32, P, P]),
+            "stief_q4_decode_step": (ctypes.c_int, [QP, BP, P, P, P, P, SZ, I32, P, P, U32, P, P]),
             "stief_mq_attention": (ctypes.c_int, [LP, BP, P, I64, I64, I32, P, P, SZ, I32, P, I64, I64, P, U32, P, P]),
             "stief_mq_num_splits": (I32, [I32, I32, I32, I32, I32]),
             "stief_mq_workspace_bytes": (SZ, [I32, I32, I32, I32, I32]),
@@ -138,9 +142,12 @@ class Layer:
 
 @dataclass
 class QLayer:
-    """One decoder layer's 8-bit quantised compressed cache (device tensors): U_k [Hkv or 1, 128, r_k], U_v
-    [Hkv or 1, 128, r_v] bf16; k_params [Hkv, r_k/64, 2] fp32 (scale, zero; static); k_codes [num_pages, Hkv, 64, r_k] uint8;
-    v_codes [num_pages, Hkv, r_v, 64] uint8 (channel-major pages with permuted token positions, see stief.h); v_params [num_pages, Hkv, 64, r_v/64, 2] fp32 (scale, zero per token and group)."""
+    """One decoder layer's quantised compressed cache (device tensors): U_k [Hkv or 1, 128, r_k], U_v [Hkv or 1, 128, r_v]
+    bf16; k_params [Hkv, groups(r_k), 2] fp32 (scale, zero; static); v_params [num_pages, Hkv, 64, groups(r_v), 2] fp32
+    (scale, zero per token and group), groups(r) = ceil(r / 64).  Code pools as uint8 tensors: 8-bit k_codes
+    [num_pages, Hkv, 64, r_k], v_codes [num_pages, Hkv, r_v, 64]; 4-bit k_codes [num_pages, Hkv, 64, krow] (krow = r_k / 2,
+    32 for r_k = 48), v_codes [num_pages, Hkv, r_v, 32] (channel-major pages, permuted token positions, nibble order: see
+    stief.h).  The same object serves the stief_q8_* and the stief_q4_* calls; the pools must have the matching form."""
     Hq: int
     Hkv: int
     r_k: int
@@ -198,6 +205,15 @@ def stief_prefill_compress(layer: Layer, batch: Batch, K: torch.Tensor, V: torch
                                         V.stride(0), V.stride(1), K.shape[1] if T_max is None else T_max, flags, _ptr(status),
                                         _stream()),
            "stief_prefill_compress")
+
+
+def qkey_row_bytes(r_k: int, bits: int) -> int:
+    """Bytes of one key row of the quantised cache (4-bit rank-48 rows are padded to 32 bytes)."""
+    return r_k if bits == 8 else (32 if r_k == 48 else r_k // 2)
+
+
+def qgroups(r: int) -> int:
+    return (r + 63) // 64
 
 
 def stief_q8_prefill_compress(layer: QLayer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
@@ -418,3 +434,42 @@ def stief_trace_next_decode_kernel(trace: Optional[torch.Tensor]):
         return
     assert trace.dtype == torch.int64 and trace.is_contiguous()
     _check(lib().stief_trace_next_decode_kernel(_ptr(trace), trace.numel() * 8), "stief_trace_next_decode_kernel")
+
+
+def _q(name: str, bits: int):
+    if bits not in (8, 4):
+        raise ValueError("code width must be 8 or 4")
+    return getattr(lib(), f"stief_q{bits}_{name}")
+
+
+def stief_q_prefill_compress(bits: int, layer: QLayer, batch: Batch, K: torch.Tensor, V: torch.Tensor, T_max: Optional[int] = None,
+                             status: Optional[torch.Tensor] = None, flags: int = 0):
+    """stief_q8_prefill_compress / stief_q4_prefill_compress by code width."""
+    assert K.stride(3) == 1 and K.stride(2) == D_HEAD and V.stride() == K.stride()
+    cl, cb = layer.c(), batch.c()
+    _check(_q("prefill_compress", bits)(ctypes.byref(cl), ctypes.byref(cb), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
+                                        K.shape[1] if T_max is None else T_max, flags, _ptr(status), _stream()),
+           f"stief_q{bits}_prefill_compress")
+
+
+def stief_q_append(bits: int, layer: QLayer, batch: Batch, k_new: torch.Tensor, v_new: torch.Tensor, status: Optional[torch.Tensor] = None):
+    cl, cb = layer.c(), batch.c()
+    _check(_q("append", bits)(ctypes.byref(cl), ctypes.byref(cb), _ptr(k_new), _ptr(v_new), _ptr(status), _stream()), f"stief_q{bits}_append")
+
+
+def stief_q_decode_attention(bits: int, layer: QLayer, batch: Batch, q: torch.Tensor, workspace: torch.Tensor, out: torch.Tensor,
+                             num_parts: int = 0, out_lse: Optional[torch.Tensor] = None, len_add: int = 0,
+                             status: Optional[torch.Tensor] = None, flags: int = 0):
+    cl, cb = layer.c(), batch.c()
+    _check(_q("decode_attention", bits)(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), len_add, _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
+                                        flags, _ptr(status), _stream()), f"stief_q{bits}_decode_attention")
+
+
+def stief_q_decode_step(bits: int, layer: QLayer, batch: Batch, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                        workspace: torch.Tensor, out: torch.Tensor, num_parts: int = 0, out_lse: Optional[torch.Tensor] = None,
+                        status: Optional[torch.Tensor] = None, flags: int = 0):
+    cl, cb = layer.c(), batch.c()
+    _check(_q("decode_step", bits)(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
+                                   flags, _ptr(status), _stream()), f"stief_q{bits}_decode_step")

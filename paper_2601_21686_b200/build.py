@@ -31,13 +31,16 @@ def _nvcc() -> str:
 def _units():
     """(source, object, extra flags) for every translation unit."""
     units = [(os.path.join(CSRC, f + ".cu"), os.path.join(OBJ, f + ".o"), [])
-             for f in ("stief_api", "stief_small", "stief_prefill", "stief_prefill_tc", "stief_noalloc", "stief_q8", "stief_rank_select", "stief_mq", "stief_selftest")
+             for f in ("stief_api", "stief_small", "stief_prefill", "stief_prefill_tc", "stief_noalloc", "stief_quant", "stief_rank_select", "stief_mq", "stief_selftest")
              if os.path.exists(os.path.join(CSRC, f + ".cu"))]
     for rk in KEY_RANKS:
         units.append((os.path.join(CSRC, "stief_decode_inst.cu"), os.path.join(OBJ, f"stief_decode_rk{rk}.o"),
                       [f"-DSTIEF_RK={rk}"]))
         units.append((os.path.join(CSRC, "stief_mq_inst.cu"), os.path.join(OBJ, f"stief_mq_rk{rk}.o"),
                       [f"-DSTIEF_RK={rk}"]))
+        for bits in (8, 4):
+            units.append((os.path.join(CSRC, "stief_decode_q_inst.cu"), os.path.join(OBJ, f"stief_decode_q_rk{rk}_b{bits}.o"),
+                          [f"-DSTIEF_RK={rk}", f"-DSTIEF_QBITS={bits}"]))
     return units
 
 

@@ -1,16 +1,24 @@
-// Decode attention over the 8-bit quantised compressed cache (paper Sec. 4.3): the persistent split-T kernel of
-// stief_decode.cuh with the page operands kept as integer codes all the way into the tensor cores.
+// Decode attention over the integer-quantised compressed cache (paper Sec. 4.3; 8-bit and 4-bit codes, every rank):
+// the persistent split-T kernel of stief_decode.cuh with the page operands kept as integer codes all the way into
+// the tensor cores.
 //
-// The cache holds, per (page, head): K codes [64 tokens][RK] uint8 (token-major), V codes [RV channels][64
-// positions] uint8 (channel-major, see below) and the value rows' (scale, zero) pairs.  K and V tiles are fetched by
-// TMA box loads with a hardware swizzle (ldmatrix then reads them without bank conflicts), the parameters by a 1-D
-// bulk copy.  Both contractions run on mma.sync.m16n8k32 (s8 x u8 -> s32) with the raw codes as the B operand:
+// The cache holds, per (page, head): K codes [64 tokens][key row bytes] (token-major), V codes [RV channels][64
+// positions] (channel-major, see below) and the value rows' (scale, zero) pairs, one pair per group of 64 channels
+// (the last group of ranks 32, 48, 96 is shorter).  K and V tiles are fetched by TMA box loads, with a hardware swizzle
+// where ldmatrix would otherwise meet bank conflicts, the parameters by a 1-D bulk copy.  Both contractions run on
+// mma.sync s8 x u8 -> s32 (k = 32; one k = 16 step for the 16-channel remainder of rank 48) with the raw codes as B operand:
 //   scores: A = q' (key scale folded in) as a per-row 16-bit fixed point split into two signed 8-bit digits, which
 //           occupy rows 0-7 and 8-15 of the 16-row operand; the integer sums are recombined as 256 hi + lo and
 //           scaled back per row.  The key zero-point shifts all scores of a row equally: it only enters out_lse.
 //   mix:    A = p_t * scale_t,g per value group g, again as two digits of a per-row, per-page fixed point; the value
 //           zero-points add sum_t p_t zero_t,g to every channel of the group (kept as a running scalar per group).
 // No code is ever expanded to floating point in shared memory.
+//
+// 4-bit codes are stored two to a byte in the order the tensor cores will want them after a shift and a mask: within
+// 32 consecutive contraction indices (channels of a key row, token positions of a value row) byte i holds index i in
+// its low and index i + 16 in its high nibble.  A 32-bit word of ldmatrix output then unpacks with (w & 0x0f0f0f0f) and
+// ((w >> 4) & 0x0f0f0f0f) into exactly the two B registers of one k = 32 step.  Key rows of rank 48 are padded to 64
+// nibbles (32 bytes), the unused ones zero.
 //
 // Why value pages are channel-major and their 64 token positions permuted: the B fragment of the mix needs four
 // consecutive TOKENS of one channel in a register, which is what ldmatrix delivers from channel-major rows; and the
@@ -27,13 +35,13 @@
 
 namespace stief {
 
-struct DecodeQ8Args {
+struct DecodeQArgs {
   LayerDev L;                    // bases and shape (the bf16 pool pointers are unused)
   BatchDev Bt;
-  uint8_t* k_codes;              // [pages][Hkv][64][RK]
-  uint8_t* v_codes;              // [pages][Hkv][RV][64 positions]
-  float* v_params;               // [pages][Hkv][64][RV/64][2] (scale, zero)
-  const float* k_params;         // [Hkv][RK/64][2] (scale, zero)
+  uint8_t* k_codes;              // [pages][Hkv][64][key row bytes]
+  uint8_t* v_codes;              // [pages][Hkv][RV][64 positions, 8 or 4 bits each]
+  float* v_params;               // [pages][Hkv][64][groups of RV][2] (scale, zero)
+  const float* k_params;         // [Hkv][groups of RK][2] (scale, zero)
   const __nv_bfloat16* q;        // [B][Hq][128]
   const __nv_bfloat16* k_new;    // [B][Hkv][128] or NULL: project, quantise and store at position seq_lens[b] first
   const __nv_bfloat16* v_new;
@@ -53,12 +61,78 @@ __host__ __device__ __forceinline__ int v_position(int t) {
   return (t & ~15) + 4 * ((u & 7) >> 1) + (u & 1) + 2 * (u >> 3);
 }
 
-template <int RK, int RV>
-struct DecodeQ8Cfg {
-  using TK = Tile<RK / 2>;               // 64 rows of RK bytes have the geometry of 64 rows of RK/2 bf16
-  using TV = Tile<32>;                   // channel rows of 64 bytes (64-byte swizzle), RV of them
-  static constexpr int NGV = RV / 64;
-  static constexpr int K_BYTES = kPage * RK, V_BYTES = kPage * RV, P_BYTES = kPage * NGV * 8;
+// bytes of one key row: RK codes of BITS bits (rank 48 at 4 bits is padded to 32 bytes)
+__host__ __device__ constexpr int q_key_row_bytes(int rk, int bits) { return bits == 8 ? rk : (rk == 48 ? 32 : rk / 2); }
+__host__ __device__ constexpr int q_groups(int r) { return (r + 63) / 64; }
+
+// Byte offset of 16-byte chunk c of row t in a shared-memory tile of 64 rows of ROWB bytes, as TMA leaves it:
+//   16, 48: dense rows (ldmatrix on 8 consecutive rows is conflict-free as it is)
+//   32:     32-byte swizzle;  64, 96, 128: the forms of Tile<> (64-byte swizzle, linear 32-byte swizzle, 128-byte swizzle)
+// A step of 8 rows leaves the swizzle term unchanged in every form.
+template <int ROWB>
+__device__ __forceinline__ uint32_t qtile_chunk(int t, int c) {
+  if constexpr (ROWB == 16 || ROWB == 48) {
+    return static_cast<uint32_t>(t * ROWB + c * 16);
+  } else if constexpr (ROWB == 32) {
+    uint32_t off = static_cast<uint32_t>(t * 32 + c * 16);
+    off ^= ((off >> 7) & 1u) << 4;
+    return off;
+  } else {
+    return Tile<ROWB / 2>::chunk(t, c);
+  }
+}
+
+// ---- where a code goes ------------------------------------------------------------------------------------------
+// Byte (and, for 4-bit codes, nibble) that holds contraction index i of a row: 8-bit: byte i; 4-bit: within every 32
+// indices, byte i % 16 of the block holds index i (low nibble) and i + 16 (high nibble).
+template <int BITS>
+__host__ __device__ __forceinline__ int q_code_byte(int i) { return BITS == 8 ? i : (i >> 5) * 16 + (i & 15); }
+template <int BITS>
+__host__ __device__ __forceinline__ int q_code_shift(int i) { return BITS == 8 ? 0 : 4 * ((i >> 4) & 1); }
+
+// The quantiser's decision (fp32, round to nearest even, clamp): code = clamp(rint((x - zero) * (1 / scale)))
+template <int BITS>
+__device__ __forceinline__ uint32_t q_encode(float x, float scale, float zero) {
+  const float y = __fmul_rn(__fsub_rn(x, zero), __fdiv_rn(1.f, scale));
+  return (uint32_t)fminf(fmaxf(rintf(y), 0.f), (float)((1 << BITS) - 1));
+}
+
+// Writes one key row from per-channel codes in shared memory (codes[j], j < RK): byte b of the row is assembled by one thread.
+template <int RK, int BITS>
+__device__ __forceinline__ void q_store_key_row(uint8_t* row, const uint8_t* codes, int tid, int nt) {
+  constexpr int KROW = q_key_row_bytes(RK, BITS);
+  for (int bi = tid; bi < KROW; bi += nt) {
+    if constexpr (BITS == 8) {
+      row[bi] = codes[bi];
+    } else {
+      const int lo = (bi >> 4) * 32 + (bi & 15), hi = lo + 16;
+      row[bi] = (uint8_t)((lo < RK ? codes[lo] : 0) | ((hi < RK ? codes[hi] : 0) << 4));
+    }
+  }
+}
+
+// Writes the code of one (channel row, position) of a value page.  4-bit: the byte is shared with the token 16 positions
+// away, which is written at another time: the nibble is replaced with two atomic bit operations on the enclosing word.
+template <int BITS>
+__device__ __forceinline__ void q_store_value_code(uint8_t* channel_row, int pos, uint32_t code) {
+  if constexpr (BITS == 8) {
+    channel_row[pos] = (uint8_t)code;
+  } else {
+    uint8_t* bp = channel_row + q_code_byte<4>(pos);
+    unsigned* w = reinterpret_cast<unsigned*>(reinterpret_cast<uintptr_t>(bp) & ~(uintptr_t)3);
+    const int sh = 8 * (int)(reinterpret_cast<uintptr_t>(bp) & 3) + q_code_shift<4>(pos);
+    atomicAnd(w, ~(0xFu << sh));
+    atomicOr(w, code << sh);
+  }
+}
+
+template <int RK, int RV, int BITS>
+struct DecodeQCfg {
+  static_assert(BITS == 8 || BITS == 4, "8-bit or 4-bit codes");
+  static constexpr int KROW = q_key_row_bytes(RK, BITS); // bytes of a key row
+  static constexpr int VROW = BITS == 8 ? 64 : 32;       // bytes of a value channel row (64 positions)
+  static constexpr int NGK = q_groups(RK), NGV = q_groups(RV);
+  static constexpr int K_BYTES = kPage * KROW, V_BYTES = RV * VROW, P_BYTES = kPage * NGV * 8;
   static constexpr int TX_BYTES = K_BYTES + V_BYTES + P_BYTES;           // bytes one page brings into a stage
   static constexpr int STAGE_BYTES = (TX_BYTES + 1023) / 1024 * 1024;    // stages keep the key tile's swizzle alignment
   static constexpr int HALF = 2;
@@ -78,9 +152,8 @@ struct DecodeQ8Cfg {
   static constexpr int NS = NP * SPW;
   static constexpr int RING_BYTES = NS * STAGE_BYTES;
   static constexpr int SMEM_BYTES = 1024 + RING_BYTES + MISC;
-  static_assert(RK % 64 == 0 && RV % 64 == 0 && RK <= 128 && RV <= 128, "quantisation groups are 64 channels");
-  static_assert(TK::NB == 1 && TK::BYTES == K_BYTES, "key tile is one swizzled box");
-  static_assert(STAGE_BYTES % 1024 == 0 && K_BYTES % 1024 == 0, "tiles keep their swizzle alignment");
+  static_assert(RK % 16 == 0 && RV % 16 == 0 && RK >= 32 && RV >= 32 && RK <= 128 && RV <= 128, "ranks are multiples of 16 in 32..128");
+  static_assert(K_BYTES % 1024 == 0 && V_BYTES % 16 == 0, "the value tile and the parameters keep their alignment behind the key tile");
   static_assert(SPW >= 2 && NS <= 16, "ring shape");
   static_assert((NW * 8 * RV + 2 * NW * 8) * 4 <= UNION_BYTES, "merge scratch must fit");
   static_assert(kCombineScratchFloats * 4 <= UNION_BYTES, "combine scratch must fit");
@@ -93,6 +166,17 @@ __device__ __forceinline__ void mma_s8u8(int (&d)[4], const uint32_t (&a)[4], ui
       "mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// D += A(16x16, row, s8) * B(16x8, col, u8), s32 accumulate
+__device__ __forceinline__ void mma_s8u8_k16(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ void ldsm_x1(uint32_t addr, uint32_t& r0) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x1.shared.b16 {%0}, [%1];" : "=r"(r0) : "r"(addr));
 }
 
 // Two signed 8-bit digits of a 16-bit fixed-point value a in [-32640, 32639]: a = 256 hi + lo, both in [-128, 127]
@@ -115,15 +199,17 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 }
 
 
-template <int RK, int RV>
-__global__ void __launch_bounds__(DecodeQ8Cfg<RK, RV>::THREADS, 1)
-decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeQ8Args a) {
-  using C = DecodeQ8Cfg<RK, RV>;
-  using TK = typename C::TK;
-  using TV = typename C::TV;
+template <int RK, int RV, int BITS>
+__global__ void __launch_bounds__(DecodeQCfg<RK, RV, BITS>::THREADS, 1)
+decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeQArgs a) {
+  using C = DecodeQCfg<RK, RV, BITS>;
   constexpr int NW = C::NW, NS = C::NS, SPW = C::SPW, NT = C::NT, NP = C::NP, HALF = C::HALF;
   constexpr int NJ = 4;                                  // 8-token score tiles per consumer warp and page (32 tokens)
-  constexpr int NGV = C::NGV;
+  constexpr int NGV = C::NGV, NGK = C::NGK, KROW = C::KROW, VROW = C::VROW;
+  constexpr int QMAX = (1 << BITS) - 1;                  // largest code
+  // contraction steps of the scores: blocks of 32 channels, and (8-bit rank 48 only) one step of 16
+  constexpr int KB32 = BITS == 8 ? RK / 32 : KROW / 16;
+  constexpr int KREM = (BITS == 8 && RK % 32 != 0) ? 1 : 0;
 
   extern __shared__ uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -216,8 +302,9 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           const uint32_t st = ring + slot * C::STAGE_BYTES;
           const size_t tile = (size_t)page * Hkv + h;
           mbar_arrive_expect_tx(full_bar(slot), C::TX_BYTES);
-          tma_load_2d(st, &tmK, 0, (int)tile * kPage, full_bar(slot));                  // 64 token rows of RK bytes
-          tma_load_2d(st + C::K_BYTES, &tmV, 0, (int)tile * RV, full_bar(slot));        // RV channel rows of 64 bytes
+          // 64 token rows of KROW bytes (96-byte rows: the tile as 192 lines of 32 bytes); RV channel rows of VROW bytes
+          tma_load_2d(st, &tmK, 0, (int)tile * (KROW == 96 ? 192 : kPage), full_bar(slot));
+          tma_load_2d(st + C::K_BYTES, &tmV, 0, (int)tile * RV, full_bar(slot));
           bulk_load_1d(st + C::K_BYTES + C::V_BYTES, a.v_params + tile * (C::P_BYTES / 4), C::P_BYTES, full_bar(slot));
         }
         __syncwarp();
@@ -236,10 +323,18 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   // covers 8 tokens x 64 channels (four 16-byte chunks); a value ldmatrix.x4 covers two 8-channel tiles x the
   // warp's 32 positions (two chunks each).
   const int pl = warp % NP, hf = warp / NP;               // page lane; which 32 tokens of a page this warp takes
-  uint32_t koff[RK / 64];
+  constexpr int NKC = KROW / 16;                           // 16-byte chunks of a key row
+  uint32_t koff[(NKC + 3) / 4];                            // chunk 4 q + (lane / 8) of row l7 (wrapped inside the row for short tails)
 #pragma unroll
-  for (int ks = 0; ks < RK / 64; ++ks) koff[ks] = TK::chunk(l7, 4 * ks + (lane >> 3));
-  const uint32_t voff = TV::chunk(l7 + 8 * (lane >> 4), 2 * hf + ((lane >> 3) & 1));
+  for (int q4 = 0; q4 < (NKC + 3) / 4; ++q4) {
+    const int rest = NKC - 4 * q4;                         // chunks this ldmatrix really covers: 4, 2 or 1
+    const int m = lane >> 3;
+    koff[q4] = qtile_chunk<KROW>(l7, 4 * q4 + min(m, rest - 1));     // matrices beyond the row's end repeat its last chunk
+  }
+  // value rows: 8-bit: two 8-channel tiles x the warp's two 16-position chunks per ldmatrix.x4;
+  //             4-bit: four 8-channel tiles x the warp's one chunk of 32 positions
+  const uint32_t voff = BITS == 8 ? qtile_chunk<64>(l7 + 8 * (lane >> 4), 2 * hf + ((lane >> 3) & 1))
+                                  : qtile_chunk<32>(l7 + 8 * (lane >> 3), hf);
   int i_base = 0;              // pages of this CTA before the current segment
 
   while (walk.next(seg)) {
@@ -267,6 +362,7 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // q' . zero, which cancels in the softmax and across segments and is added to out_lse at the very end.
     float* rows = un;                    // [9][128] fp32: the queries, row 8 = the new key
     float* vrow = un + 9 * kD;           // [128]: the new value, later its projection
+    uint8_t* kcode_s = reinterpret_cast<uint8_t*>(rows + 8 * kD);    // the new key's codes, once its input row is used up
     float* red = un + 10 * kD;           // [NW][9][128]
     const __nv_bfloat16* Uk = a.L.U_k + (size_t)h * a.L.uk_stride;
     const __nv_bfloat16* Uv = a.L.U_v + (size_t)h * a.L.uv_stride;
@@ -305,16 +401,14 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     BasisSlice<NW, RV> sv;
     if (do_append) sv.load(Uv, warp, lane);                // in flight while the key side is reduced
     bar1(NT);
-    const float* kpar = a.k_params + (size_t)h * (RK / 64) * 2;
+    const float* kpar = a.k_params + (size_t)h * NGK * 2;
     for (int idx = tid; idx < 9 * RK; idx += NT) {
       const int r = idx / RK, j = idx % RK;
       const float x = ((row_mask >> r) & 1u) ? warp_shares<NW>(red, r, j) : 0.f;
       if (r < 8) {
         qp[r * RK + j] = x * qscale * __ldg(kpar + 2 * (j >> 6));
-      } else if (do_append && new_page >= 0) {             // the new key's code under the head's static parameters
-        const float sc = __ldg(kpar + 2 * (j >> 6)), zp = __ldg(kpar + 2 * (j >> 6) + 1);
-        const float y = __fmul_rn(__fsub_rn(x, zp), __fdiv_rn(1.f, sc));
-        a.k_codes[(((size_t)new_page * Hkv + h) * kPage + new_pos) * RK + j] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+      } else if (do_append) {                              // the new key's code under the head's static parameters
+        kcode_s[j] = (uint8_t)q_encode<BITS>(x, __ldg(kpar + 2 * (j >> 6)), __ldg(kpar + 2 * (j >> 6) + 1));
       }
     }
     if (tid < 8) {
@@ -331,6 +425,8 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     bar1(NT);
     if (do_append) {
+      if (new_page >= 0)
+        q_store_key_row<RK, BITS>(a.k_codes + (((size_t)new_page * Hkv + h) * kPage + new_pos) * KROW, kcode_s, tid, NT);
       // the new value row: project (the row sits where row 0 is expected), then token-wise group parameters and codes
       sv.contract(vrow, 1u, red, warp, lane);
       bar1(NT);
@@ -338,16 +434,15 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       bar1(NT);
       if (new_page >= 0) {
         for (int j = tid; j < RV; j += NT) {
-          const int g = j >> 6;
+          const int g = j >> 6, g1 = min(64 * g + 64, RV);
           float mn = vrow[64 * g], mxv = mn;
-          for (int e = 1; e < 64; ++e) {
-            mn = fminf(mn, vrow[64 * g + e]);
-            mxv = fmaxf(mxv, vrow[64 * g + e]);
+          for (int e = 64 * g + 1; e < g1; ++e) {
+            mn = fminf(mn, vrow[e]);
+            mxv = fmaxf(mxv, vrow[e]);
           }
-          const float sc = mxv > mn ? __fdiv_rn(mxv - mn, 255.f) : 1.f;
-          const float y = __fmul_rn(__fsub_rn(vrow[j], mn), __fdiv_rn(1.f, sc));
+          const float sc = mxv > mn ? __fdiv_rn(mxv - mn, (float)QMAX) : 1.f;
           const size_t tile = (size_t)new_page * Hkv + h;
-          a.v_codes[(tile * RV + j) * kPage + v_position(new_pos)] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+          q_store_value_code<BITS>(a.v_codes + (tile * RV + j) * VROW, v_position(new_pos), q_encode<BITS>(vrow[j], sc, mn));
           if ((j & 63) == 0) *reinterpret_cast<float2*>(a.v_params + ((tile * kPage + new_pos) * NGV + g) * 2) = make_float2(sc, mn);
         }
       } else if (tid == 0) {
@@ -361,21 +456,30 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     // A operand of the score MMA: rows 0-7 = high digits of the scaled query rows, rows 8-15 = low digits
     const float dq = q_delta[gid];
-    uint32_t qa[RK / 32][4];
+    uint32_t qa[KB32][4];
+    uint32_t qrem[2] = {0u, 0u};                           // the 16-channel remainder (8-bit codes, rank 48)
     {
       const float inv = 1.f / dq;
+      auto qv = [&](int ch) { return ch < RK ? qp[gid * RK + ch] : 0.f; };   // channels of a padded key row contribute nothing
 #pragma unroll
-      for (int ks = 0; ks < RK / 32; ++ks) {
+      for (int ks = 0; ks < KB32; ++ks) {
         int hi[8], lo[8];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          digits(qp[gid * RK + 32 * ks + 4 * tid4 + e], inv, hi[e], lo[e]);
-          digits(qp[gid * RK + 32 * ks + 16 + 4 * tid4 + e], inv, hi[4 + e], lo[4 + e]);
+          digits(qv(32 * ks + 4 * tid4 + e), inv, hi[e], lo[e]);
+          digits(qv(32 * ks + 16 + 4 * tid4 + e), inv, hi[4 + e], lo[4 + e]);
         }
         qa[ks][0] = pack4(hi[0], hi[1], hi[2], hi[3]);
         qa[ks][1] = pack4(lo[0], lo[1], lo[2], lo[3]);
         qa[ks][2] = pack4(hi[4], hi[5], hi[6], hi[7]);
         qa[ks][3] = pack4(lo[4], lo[5], lo[6], lo[7]);
+      }
+      if constexpr (KREM != 0) {
+        int hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) digits(qv(32 * KB32 + 4 * tid4 + e), inv, hi[e], lo[e]);
+        qrem[0] = pack4(hi[0], hi[1], hi[2], hi[3]);
+        qrem[1] = pack4(lo[0], lo[1], lo[2], lo[3]);
       }
     }
 
@@ -410,11 +514,22 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       for (int j = 0; j < NJ; ++j) {
         int s4[4] = {0, 0, 0, 0};
 #pragma unroll
-        for (int ks = 0; ks < RK / 64; ++ks) {
-          uint32_t r0, r1, r2, r3;
-          ldsm_x4(kt + koff[ks] + (tb + 8 * j) * TK::RB, r0, r1, r2, r3);
-          mma_s8u8(s4, qa[2 * ks], r0, r1);
-          mma_s8u8(s4, qa[2 * ks + 1], r2, r3);
+        for (int q4 = 0; q4 < (NKC + 3) / 4; ++q4) {
+          const int rest = NKC - 4 * q4;                   // chunks left in the row: a compile-time value once unrolled
+          uint32_t r[4] = {0u, 0u, 0u, 0u};
+          const uint32_t addr = kt + koff[q4] + (tb + 8 * j) * KROW;
+          if (rest >= 3) ldsm_x4(addr, r[0], r[1], r[2], r[3]);
+          else if (rest == 2) ldsm_x2(addr, r[0], r[1]);
+          else ldsm_x1(addr, r[0]);
+          if constexpr (BITS == 8) {                       // two chunks of 16 codes per step of 32 channels
+            mma_s8u8(s4, qa[2 * q4], r[0], r[1]);
+            if (rest >= 4) mma_s8u8(s4, qa[2 * q4 + 1], r[2], r[3]);
+            else if (rest == 3) mma_s8u8_k16(s4, qrem[0], qrem[1], r[2]);
+          } else {                                         // one chunk of 32 nibbles per step of 32 channels
+#pragma unroll
+            for (int mm = 0; mm < 4; ++mm)
+              if (mm < rest) mma_s8u8(s4, qa[4 * q4 + mm], r[mm] & 0x0f0f0f0fu, (r[mm] >> 4) & 0x0f0f0f0fu);
+          }
         }
         sc[2 * j] = dq * (float)(256 * s4[0] + s4[2]);
         sc[2 * j + 1] = dq * (float)(256 * s4[1] + s4[3]);
@@ -481,18 +596,43 @@ decode_q8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // k-slots 4 tid4 .. + 3 of the first 16 positions hold tiles 0 and 1, of the second 16 tiles 2 and 3
         const uint32_t pa[4] = {pack4(hi[0], hi[1], hi[2], hi[3]), pack4(lo[0], lo[1], lo[2], lo[3]),
                                 pack4(hi[4], hi[5], hi[6], hi[7]), pack4(lo[4], lo[5], lo[6], lo[7])};
+        const int GT = (min(64 * g + 64, RV) - 64 * g) / 8;       // 8-channel tiles of the group: 8, or 4 / 6 in a short last group
+        if constexpr (BITS == 8) {
 #pragma unroll
-        for (int n2 = 0; n2 < 4; ++n2) {                   // two 8-channel tiles per ldmatrix: 64 channels per group
-          const int n = 8 * g + 2 * n2;
-          uint32_t r0, r1, r2, r3;
-          ldsm_x4(vt + voff + n * 8 * TV::RB, r0, r1, r2, r3);
-          int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
-          mma_s8u8(c0, pa, r0, r1);
-          mma_s8u8(c1, pa, r2, r3);
-          o[n][0] = fmaf(dp, (float)(256 * c0[0] + c0[2]), o[n][0]);
-          o[n][1] = fmaf(dp, (float)(256 * c0[1] + c0[3]), o[n][1]);
-          o[n + 1][0] = fmaf(dp, (float)(256 * c1[0] + c1[2]), o[n + 1][0]);
-          o[n + 1][1] = fmaf(dp, (float)(256 * c1[1] + c1[3]), o[n + 1][1]);
+          for (int n2 = 0; n2 < 4; ++n2) {                 // two 8-channel tiles x two chunks of 16 positions per ldmatrix
+            if (2 * n2 < GT) {
+              const int n = 8 * g + 2 * n2;
+              uint32_t r0, r1, r2, r3;
+              ldsm_x4(vt + voff + n * 8 * VROW, r0, r1, r2, r3);
+              int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
+              mma_s8u8(c0, pa, r0, r1);
+              mma_s8u8(c1, pa, r2, r3);
+              o[n][0] = fmaf(dp, (float)(256 * c0[0] + c0[2]), o[n][0]);
+              o[n][1] = fmaf(dp, (float)(256 * c0[1] + c0[3]), o[n][1]);
+              o[n + 1][0] = fmaf(dp, (float)(256 * c1[0] + c1[2]), o[n + 1][0]);
+              o[n + 1][1] = fmaf(dp, (float)(256 * c1[1] + c1[3]), o[n + 1][1]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int n4 = 0; n4 < 2; ++n4) {                 // four 8-channel tiles x one chunk of 32 positions per ldmatrix
+            const int left = GT - 4 * n4;                  // tiles left in the group: 4 or more, 2, or none
+            if (left > 0) {
+              const int n = 8 * g + 4 * n4;
+              uint32_t r[4] = {0u, 0u, 0u, 0u};
+              if (left >= 4) ldsm_x4(vt + voff + n * 8 * VROW, r[0], r[1], r[2], r[3]);
+              else ldsm_x2(vt + voff + n * 8 * VROW, r[0], r[1]);
+#pragma unroll
+              for (int mm = 0; mm < 4; ++mm) {
+                if (mm < left) {
+                  int c0[4] = {0, 0, 0, 0};
+                  mma_s8u8(c0, pa, r[mm] & 0x0f0f0f0fu, (r[mm] >> 4) & 0x0f0f0f0fu);
+                  o[n + mm][0] = fmaf(dp, (float)(256 * c0[0] + c0[2]), o[n + mm][0]);
+                  o[n + mm][1] = fmaf(dp, (float)(256 * c0[1] + c0[3]), o[n + mm][1]);
+                }
+              }
+            }
+          }
         }
       }
       __syncwarp();

@@ -58,9 +58,9 @@ cudaError_t launch_append_chunk(const AppendChunkArgs& a, cudaStream_t st);
 cudaError_t launch_combine(const CombineArgs& a, cudaStream_t st);
 cudaError_t launch_advance(int32_t* seq_lens, int B, int delta, cudaStream_t st);
 cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st);
-// The same projection with the 8-bit quantising epilogue (both bases required; a.L's bf16 pools are unused).
-cudaError_t launch_prefill_q8(const PrefillArgs& a, uint8_t* k_codes, uint8_t* v_codes, float* v_params, const float* k_params,
-                              cudaStream_t st);
+// The same projection with the quantising epilogue, 8-bit or 4-bit codes (both bases required; a.L's bf16 pools are unused).
+cudaError_t launch_prefill_quant(const PrefillArgs& a, int bits, uint8_t* k_codes, uint8_t* v_codes, float* v_params,
+                                 const float* k_params, cudaStream_t st);
 
 // Returns cudaErrorInvalidValue for a rank pair that is not compiled in.
 cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const CUtensorMap& tmV, cudaStream_t st);

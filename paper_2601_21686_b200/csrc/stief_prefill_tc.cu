@@ -46,16 +46,16 @@ struct Args {
   int n_chunks;              // chunks per unit's tile list (see TileWalker)
   int nst;                   // ring stages
   int rmax;                  // larger of the ranks that are projected
-  // 8-bit quantised cache (Q8 kernel only): code pools [pages][Hkv][64][r] uint8, value parameters
-  // [pages][Hkv][64][r_v/64][2] fp32 (scale, zero), static key parameters [Hkv][r_k/64][2] fp32
+  // quantised cache (QBITS = 8 or 4 only): code pools, value parameters [pages][Hkv][64][groups][2] fp32 (scale, zero),
+  // static key parameters [Hkv][groups][2] fp32; groups of 64 channels, the last one shorter for ranks 32, 48, 96
   uint8_t* k_codes;
   uint8_t* v_codes;
   float* v_params;
   const float* k_params;
 };
 
-// position of token t (0..63) inside a quantised value page's channel rows (see stief_decode_q8.cuh)
-__device__ __forceinline__ int q8_v_position(int t) {
+// position of token t (0..63) inside a quantised value page's channel rows (see stief_decode_q.cuh)
+__device__ __forceinline__ int q_v_position(int t) {
   const int u = t & 15;
   return (t & ~15) + 4 * ((u & 7) >> 1) + (u & 1) + 2 * (u >> 3);
 }
@@ -190,9 +190,9 @@ __device__ __forceinline__ void stage_basis(const __nv_bfloat16* __restrict__ U,
   if (lane == 0) mbar_arrive(ready_bar);
 }
 
-// Q8 = false: bf16 cache.  Q8 = true: the epilogue quantises each 64-channel group of a row to 8-bit codes
-// (asymmetric; static key parameters, token-wise value parameters) instead of rounding it to bf16.
-template <bool Q8>
+// QBITS = 0: bf16 cache.  QBITS = 8 or 4: the epilogue quantises each group of up to 64 channels of a row to integer
+// codes of that width (asymmetric; static key parameters, token-wise value parameters) instead of rounding it to bf16.
+template <int QBITS>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmPK, const __grid_constant__ CUtensorMap tmPV, const Args a) {
@@ -370,7 +370,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
           if (lane == 0) report(p.status, STIEF_ERR_BOUNDS);
           valid = false;
         }
-        const bool full = !Q8 && valid && tok0 + 32 <= t.len;   // else the sequence ends inside these rows (or codes are stored)
+        const bool full = QBITS == 0 && valid && tok0 + 32 <= t.len;   // else the sequence ends inside these rows (or codes are stored)
         const int row0 = (max(page, 0) * Hkv + t.h) * kPage + (tok0 % kPage);  // pool row of the warp's first token
         // full case: rows are rounded to bf16 into swizzled staging boxes and leave by TMA stores.  A box is 32
         // rows x BW elements (BW = 64, 32 or 16: the largest that divides R), swizzle span = box row.
@@ -394,59 +394,103 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int c = 0; c < 4; ++c)
               if ((c0 + c) * 16 < R) tmem_ld16(taddr + (c0 + c) * 16, v[c]);
             tmem_ld_wait();
-            if constexpr (Q8) {
-              // columns 16 c0 .. 16 c0 + 63 are one quantisation group of this thread's row
-              if (row_ok) {
-                const int g = c0 >> 2, ng = R >> 6;
-                float sc, zp;
-                if (t.side == 0) {
-                  const float2 kp = *reinterpret_cast<const float2*>(a.k_params + ((size_t)t.h * ng + g) * 2);
-                  sc = kp.x;
-                  zp = kp.y;
-                } else {
-                  float mn = __uint_as_float(v[0][0]), mx = mn;
+            if constexpr (QBITS != 0) {
+              // columns 16 c0 .. are one quantisation group of this thread's row: 64 of them, or the 32 / 48 that a
+              // short last group has (nc chunks of 16).  Codes are decided in fp32 from the fp32 accumulator.
+              const int g = c0 >> 2, ng = (R + 63) >> 6, nc = min(4, R / 16 - c0);
+              constexpr float kLevels = (float)((1 << QBITS) - 1);
+              float sc = 1.f, zp = 0.f;
+              if (t.side == 0) {
+                const float2 kp = *reinterpret_cast<const float2*>(a.k_params + ((size_t)t.h * ng + g) * 2);
+                sc = kp.x;
+                zp = kp.y;
+              } else {
+                float mn = __uint_as_float(v[0][0]), mx = mn;
 #pragma unroll
-                  for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 4; ++c)
+                  if (c < nc) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                       mn = fminf(mn, __uint_as_float(v[c][e]));
                       mx = fmaxf(mx, __uint_as_float(v[c][e]));
                     }
-                  sc = mx > mn ? __fdiv_rn(mx - mn, 255.f) : 1.f;
-                  zp = mn;
-                  *reinterpret_cast<float2*>(a.v_params + (((size_t)row0 + lane) * ng + g) * 2) = make_float2(sc, zp);
-                }
-                const float inv = __fdiv_rn(1.f, sc);
-                if (t.side) {
-                  // value codes are stored channel-major with the page's 64 positions permuted (v_position): the
-                  // 32 lanes of the warp write 32 bytes of one channel row
-                  const int tp = (row0 % kPage) + lane;                               // token within its page
-                  uint8_t* vrow = a.v_codes + ((size_t)(row0 / kPage) * R + 64 * g) * kPage + q8_v_position(tp);
+                  }
+                sc = mx > mn ? __fdiv_rn(mx - mn, kLevels) : 1.f;
+                zp = mn;
+                if (row_ok) *reinterpret_cast<float2*>(a.v_params + (((size_t)row0 + lane) * ng + g) * 2) = make_float2(sc, zp);
+              }
+              const float inv = __fdiv_rn(1.f, sc);
+              auto code = [&](int c, int e) -> uint32_t {
+                const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][e]), zp), inv);
+                return (uint32_t)fminf(fmaxf(rintf(y), 0.f), kLevels);
+              };
+              const int tp = (row0 % kPage) + lane;                                   // token within its page
+              if (t.side) {
+                // value codes are stored channel-major with the page's 64 positions permuted (q_v_position)
+                if constexpr (QBITS == 8) {
+                  // the 32 lanes of the warp write 32 bytes of one channel row
+                  if (row_ok) {
+                    uint8_t* vrow = a.v_codes + ((size_t)(row0 / kPage) * R + 64 * g) * kPage + q_v_position(tp);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                      if (c < nc) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) vrow[(size_t)(16 * c + e) * kPage] = (uint8_t)code(c, e);
+                      }
+                  }
+                } else {
+                  // 4-bit: a channel row has 32 bytes; the byte of position p also holds position p + 16, which is the
+                  // token 16 rows on (lane + 16).  Lanes exchange their codes eight at a time; the lower lane stores.
+                  const int pos = q_v_position(tp);
+                  uint8_t* vrow = a.v_codes + ((size_t)(row0 / kPage) * R + 64 * g) * 32 + (pos >> 5) * 16 + (pos & 15);
 #pragma unroll
                   for (int c = 0; c < 4; ++c)
+                    if (c < nc) {                                                     // uniform over the warp
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                      const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][e]), zp), inv);
-                      vrow[(size_t)(16 * c + e) * kPage] = (uint8_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
+                      for (int e8 = 0; e8 < 2; ++e8) {
+                        uint32_t mine = 0;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) mine |= (row_ok ? code(c, 8 * e8 + e) : 0u) << (4 * e);
+                        const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 16);
+                        if (lane < 16 && row_ok) {
+#pragma unroll
+                          for (int e = 0; e < 8; ++e)
+                            vrow[(size_t)(16 * c + 8 * e8 + e) * 32] = (uint8_t)(((mine >> (4 * e)) & 0xFu) | (((other >> (4 * e)) & 0xFu) << 4));
+                        }
+                      }
+                    }
+                }
+              } else if (row_ok) {
+                if constexpr (QBITS == 8) {
+                  uint8_t* qdst = a.k_codes + ((size_t)row0 + lane) * R + 64 * g;
+#pragma unroll
+                  for (int c = 0; c < 4; ++c)
+                    if (c < nc) {
+                      uint32_t w[4];
+#pragma unroll
+                      for (int e4 = 0; e4 < 4; ++e4) w[e4] = code(c, 4 * e4) | (code(c, 4 * e4 + 1) << 8) | (code(c, 4 * e4 + 2) << 16) | (code(c, 4 * e4 + 3) << 24);
+                      *reinterpret_cast<uint4*>(qdst + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 } else {
-                uint8_t* qdst = a.k_codes + ((size_t)row0 + lane) * R + 64 * g;
+                  // 4-bit key rows: per 32 channels, byte i holds channel i (low nibble) and i + 16 (high nibble);
+                  // a lone block of 16 channels (rank 48) keeps its high nibbles zero (row padded to 32 bytes)
+                  const int krow = R == 48 ? 32 : R / 2;
+                  uint8_t* qdst = a.k_codes + ((size_t)row0 + lane) * krow + 32 * g;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                  uint32_t w[4];
+                  for (int c = 0; c < 4; c += 2)
+                    if (c < nc) {
+                      const bool has_hi = c + 1 < nc;
+                      uint32_t w[4];
 #pragma unroll
-                  for (int e4 = 0; e4 < 4; ++e4) {
-                    uint32_t word = 0;
+                      for (int e4 = 0; e4 < 4; ++e4) {
+                        uint32_t word = 0;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                      const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][4 * e4 + e]), zp), inv);
-                      const uint32_t code = (uint32_t)fminf(fmaxf(rintf(y), 0.f), 255.f);
-                      word |= code << (8 * e);
+                        for (int e = 0; e < 4; ++e)
+                          word |= (code(c, 4 * e4 + e) | ((has_hi ? code(c + 1, 4 * e4 + e) : 0u) << 4)) << (8 * e);
+                        w[e4] = word;
+                      }
+                      *reinterpret_cast<uint4*>(qdst + 8 * c) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
-                    w[e4] = word;
-                  }
-                  *reinterpret_cast<uint4*>(qdst + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
                 }
               }
             } else {
@@ -550,14 +594,14 @@ int smem_bytes(int nst, int rmax, int B) {
 
 namespace {
 
-template <bool Q8>
+template <int QBITS>
 cudaError_t launch_prefill_tc(const PrefillArgs& a, const Args* q8, cudaStream_t st) {
   const bool proj_k = a.L.U_k != nullptr, proj_v = a.L.U_v != nullptr;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<QBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
@@ -565,7 +609,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, const Args* q8, cudaStream_t
   if (!make_input_map(&tmK, proj_k ? a.K : a.V, a, !proj_k) || !make_input_map(&tmV, proj_v ? a.V : a.K, a, proj_v))
     return cudaErrorInvalidValue;
   CUtensorMap tmPK = tmK, tmPV = tmV;                     // the quantising kernel stores without TMA: placeholders
-  if (!Q8 && (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a)))
+  if (QBITS == 0 && (!make_pool_store_map(&tmPK, a.L.k_pool, a.L.r_k, a) || !make_pool_store_map(&tmPV, a.L.v_pool, a.L.r_v, a)))
     return cudaErrorInvalidValue;
   Args args = {};
   if (q8) args = *q8;
@@ -607,7 +651,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, const Args* q8, cudaStream_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.overlap_previous ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<Q8>, tmK, tmV, tmPK, tmPV, args);
+  return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<QBITS>, tmK, tmV, tmPK, tmPV, args);
 }
 
 }  // namespace
@@ -623,17 +667,17 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
     if (e != cudaSuccess) return e;
   }
   if (!proj_k && !proj_v) return cudaSuccess;
-  return launch_prefill_tc<false>(a, nullptr, st);
+  return launch_prefill_tc<0>(a, nullptr, st);
 }
 
-cudaError_t launch_prefill_q8(const PrefillArgs& a, uint8_t* k_codes, uint8_t* v_codes, float* v_params, const float* k_params,
-                              cudaStream_t st) {
-  Args q8 = {};
-  q8.k_codes = k_codes;
-  q8.v_codes = v_codes;
-  q8.v_params = v_params;
-  q8.k_params = k_params;
-  return launch_prefill_tc<true>(a, &q8, st);
+cudaError_t launch_prefill_quant(const PrefillArgs& a, int bits, uint8_t* k_codes, uint8_t* v_codes, float* v_params,
+                                 const float* k_params, cudaStream_t st) {
+  Args q = {};
+  q.k_codes = k_codes;
+  q.v_codes = v_codes;
+  q.v_params = v_params;
+  q.k_params = k_params;
+  return bits == 8 ? launch_prefill_tc<8>(a, &q, st) : bits == 4 ? launch_prefill_tc<4>(a, &q, st) : cudaErrorInvalidValue;
 }
 
 }  // namespace stief

@@ -12,7 +12,7 @@ from oracle import stief_quant_oracle as Q
 from paper_2601_21686_b200 import inputs as I
 from tests import _util as U
 from tests.test_gpu_fullsize import DEV, DevCase, check_edge_pages, check_pair, decode_full, sync_ok, workspace
-from tests.test_gpu_q8 import vpos
+from tests.test_gpu_quant import unpack_rows, vpos
 
 pytestmark = pytest.mark.gpu
 
@@ -36,8 +36,8 @@ class QDevCase:
     """One layer of the quantised cache at full size: inputs generated on the device, static key parameters calibrated
     on the host (oracle arithmetic) from sequence 0 only, so rows of the other sequences also meet the clamp."""
 
-    def __init__(self, seed, layer, B, Hq, Hkv, r_k, r_v, T, paging):
-        self.B, self.Hq, self.Hkv, self.r_k, self.r_v, self.T = B, Hq, Hkv, r_k, r_v, T
+    def __init__(self, seed, layer, B, Hq, Hkv, r_k, r_v, T, paging, bits=8):
+        self.B, self.Hq, self.Hkv, self.r_k, self.r_v, self.T, self.bits = B, Hq, Hkv, r_k, r_v, T, bits
         self.K = I.lowrank_keys(seed, layer, B, T, Hkv, device=DEV)
         self.V = I.gaussian_kv(seed, I.TAG_V, layer, B, T, Hkv, device=DEV)
         self.U_k, self.U_v = I.stiefel_bases(seed, layer, Hkv, r_k, r_v)
@@ -46,14 +46,15 @@ class QDevCase:
         kp = []
         for h in range(Hkv):
             rows = Q.project_f32(self.K[0, :, h].double().cpu().numpy(), O.basis_of(Uk, h))
-            s, z = Q.key_params_from_calibration(rows, 8)
+            s, z = Q.key_params_from_calibration(rows, bits)
             kp.append(np.stack([s, z], -1))
         self.k_params = np.stack(kp).astype(np.float32)
         P = paging.num_pages
         fill = lambda shape, v, dt: torch.full(shape, v, dtype=dt, device=DEV)
         self.layer = S.QLayer(Hq, Hkv, r_k, r_v, self.U_k.to(DEV), self.U_v.to(DEV), torch.from_numpy(self.k_params).to(DEV),
-                              fill((P, Hkv, 64, r_k), 0xAB, torch.uint8), fill((P, Hkv, r_v, 64), 0xCD, torch.uint8),
-                              fill((P, Hkv, 64, r_v // 64, 2), float("nan"), torch.float32))
+                              fill((P, Hkv, 64, S.qkey_row_bytes(r_k, bits)), 0xAB, torch.uint8),
+                              fill((P, Hkv, r_v, 64 if bits == 8 else 32), 0xCD, torch.uint8),
+                              fill((P, Hkv, 64, S.qgroups(r_v), 2), float("nan"), torch.float32))
         bt = np.where(paging.block_table < 0, 0, paging.block_table).astype(np.int32)
         self.batch = S.Batch(torch.from_numpy(bt).to(DEV), torch.from_numpy(paging.seq_lens.copy()).to(DEV))
         self.status = torch.zeros(1, dtype=torch.int32, device=DEV)
@@ -62,22 +63,22 @@ class QDevCase:
         """GPU codes and parameters of the first n tokens of (b, h): key codes [n, r_k], value codes [n, r_v], params [n, ng, 2]."""
         t = torch.arange(n, device=DEV)
         pages = torch.from_numpy(self.pg.block_table[b].astype(np.int64)).to(DEV)[t // 64]
-        pos = torch.from_numpy(vpos(np.arange(n) % 64)).to(DEV)
-        kc = self.layer.k_codes[pages, h, t % 64, :].cpu().numpy().astype(np.int32)
-        vc = self.layer.v_codes[pages, h, :, pos].cpu().numpy().astype(np.int32)
+        kc = unpack_rows(self.layer.k_codes[pages, h, t % 64, :].cpu().numpy(), self.r_k, self.bits)
+        vrows = unpack_rows(self.layer.v_codes[pages, h].cpu().numpy(), 64, self.bits)          # [n, r_v, 64 positions]
+        vc = vrows[np.arange(n), :, vpos(np.arange(n) % 64)]
         vp = self.layer.v_params[pages, h, t % 64].cpu().numpy()
         return kc, vc, vp
 
 
-@pytest.mark.parametrize("r_k,r_v", [(64, 64), (128, 128)])
-def test_q8_config2_shape_prefill_and_overlapped_steps(r_k, r_v):
+@pytest.mark.parametrize("bits,r_k,r_v", [(8, 64, 64), (8, 128, 128), (4, 64, 64), (4, 96, 48)])
+def test_quantised_config2_shape_prefill_and_overlapped_steps(bits, r_k, r_v):
     # the `bench.py --q8` launch pattern: quantising prefill of two layer caches, then fused steps alternating over
     # them with overlapped launches on one workspace; every CTA's ring wraps many times (512 pages per (b, h))
     B, Hq, Hkv, T = 4, 32, 8, 32768
     pg = I.make_paging(60, [T] * B, reserve_tokens=2, extra_pages=1)
-    cs = [QDevCase(60 + r_k, l, B, Hq, Hkv, r_k, r_v, T, pg) for l in range(2)]
+    cs = [QDevCase(60 + r_k, l, B, Hq, Hkv, r_k, r_v, T, pg, bits=bits) for l in range(2)]
     for i, c in enumerate(cs):
-        S.stief_q8_prefill_compress(c.layer, c.batch, c.K, c.V, status=c.status, flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if i else 0)
+        S.stief_q_prefill_compress(bits, c.layer, c.batch, c.K, c.V, status=c.status, flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if i else 0)
     ws = torch.full((S.stief_decode_workspace_bytes(B, Hq, Hkv, r_v, 0) // 4,), float("nan"), dtype=torch.float32, device=DEV)
     S.stief_decode_workspace_init(ws)
     n_steps = 4
@@ -87,7 +88,7 @@ def test_q8_config2_shape_prefill_and_overlapped_steps(r_k, r_v):
     lses = [torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV) for _ in range(n_steps)]
     for i in range(n_steps):
         c = cs[i % 2]
-        S.stief_q8_decode_step(c.layer, c.batch, qs[i], kvs[i][0], kvs[i][1], ws, outs[i], out_lse=lses[i], status=c.status,
+        S.stief_q_decode_step(bits, c.layer, c.batch, qs[i], kvs[i][0], kvs[i][1], ws, outs[i], out_lse=lses[i], status=c.status,
                                flags=S.STIEF_DECODE_OVERLAP_PREVIOUS if i else 0)
     torch.cuda.synchronize()
     assert all(int(c.status.item()) == 0 for c in cs)
@@ -101,8 +102,8 @@ def test_q8_config2_shape_prefill_and_overlapped_steps(r_k, r_v):
         Vh = np.concatenate([c.V[b, :, h].double().cpu().numpy(), vn[b, h].double().cpu().numpy()[None]], 0)
         Kd, Vd = Q.project_f32(Kh, Uk), Q.project_f32(Vh, Uv)
         ks, kz = c.k_params[h, :, 0], c.k_params[h, :, 1]
-        Kc = Q.quantize_keys(Kd, ks, kz, 8)
-        Vc, vs, vz = Q.quantize_values(Vd, 8)
+        Kc = Q.quantize_keys(Kd, ks, kz, bits)
+        Vc, vs, vz = Q.quantize_values(Vd, bits)
         gk, gv, gp = c.pair(b, h, T + 1)
         assert np.abs(gk - Kc).max() <= 1 and np.abs(gv - Vc).max() <= 1
         frac = (int((gk != Kc).sum()) + int((gv != Vc).sum())) / (Kc.size + Vc.size)
@@ -116,7 +117,7 @@ def test_q8_config2_shape_prefill_and_overlapped_steps(r_k, r_v):
         el = np.abs(lses[step][b, h * G:(h + 1) * G].double().cpu().numpy() - ref_lse).max()
         assert el < 5e-3
         worst = dict(abs=max(worst["abs"], ea), rel=max(worst["rel"], rl), lse=max(worst["lse"], el), codes=max(worst["codes"], frac))
-    print(f"q8 {r_k}/{r_v} full size: worst max-abs {worst['abs']:.2e}, rel-L2 {worst['rel']:.2e}, lse {worst['lse']:.2e}, "
+    print(f"q{bits} {r_k}/{r_v} full size: worst max-abs {worst['abs']:.2e}, rel-L2 {worst['rel']:.2e}, lse {worst['lse']:.2e}, "
           f"share of differing codes {worst['codes']:.2e}")
 
 
