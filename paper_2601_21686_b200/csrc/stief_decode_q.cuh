@@ -191,6 +191,22 @@ __device__ __forceinline__ uint32_t pack4(int b0, int b1, int b2, int b3) {
 }
 constexpr float kFixedMax = 32639.f;
 
+// The same digits for four values at once, already packed as the two A-operand words (high digits, low digits), without
+// a float-to-int conversion: adding 1.5 * 2^23 leaves round(x * inv_delta) in the low mantissa bits; with 128 added the
+// 16-bit pattern's high byte is the high digit and its low byte the low digit + 128 (flip the top bit of each byte).
+// Needs |x * inv_delta| <= 32639, which holds when inv_delta = 32639 / max |x|.
+__device__ __forceinline__ void digits4(float x0, float x1, float x2, float x3, float inv_delta, uint32_t& hi, uint32_t& lo) {
+  constexpr float kMagic = 12582912.f;                     // 0x4B400000
+  constexpr int kBias = 128 - 0x4B400000;
+  const uint32_t u0 = (uint32_t)(__float_as_int(fmaf(x0, inv_delta, kMagic)) + kBias);
+  const uint32_t u1 = (uint32_t)(__float_as_int(fmaf(x1, inv_delta, kMagic)) + kBias);
+  const uint32_t u2 = (uint32_t)(__float_as_int(fmaf(x2, inv_delta, kMagic)) + kBias);
+  const uint32_t u3 = (uint32_t)(__float_as_int(fmaf(x3, inv_delta, kMagic)) + kBias);
+  const uint32_t w01 = __byte_perm(u0, u1, 0x5410), w23 = __byte_perm(u2, u3, 0x5410);
+  hi = __byte_perm(w01, w23, 0x7531);
+  lo = __byte_perm(w01, w23, 0x6420) ^ 0x80808080u;
+}
+
 // 1-D bulk async copy global -> shared (both 16-byte aligned, size a multiple of 16), completion in bytes on an mbarrier
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -553,13 +569,23 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
 
       // ---- online softmax (base 2; the scale is folded into q')
-      float mx = sc[0];
-#pragma unroll
-      for (int e = 1; e < 2 * NJ; ++e) mx = fmaxf(mx, sc[e]);
+      float mx = fmaxf(fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3])), fmaxf(fmaxf(sc[4], sc[5]), fmaxf(sc[6], sc[7])));   // a tree: this sits on the page's critical chain
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
       const float m_new = fmaxf(m, mx);
-      const float alpha = fast_exp2(m - m_new);
+      // the running maximum seldom grows after a sequence's first pages: rescale only when some row's did
+      const bool grew = __any_sync(0xffffffffu, m_new > m);
+      if (grew) {
+        const float alpha = fast_exp2(m - m_new);
+        l *= alpha;
+#pragma unroll
+        for (int n = 0; n < RV / 8; ++n) {
+          o[n][0] *= alpha;
+          o[n][1] *= alpha;
+        }
+#pragma unroll
+        for (int g = 0; g < NGV; ++g) zc[g] *= alpha;
+      }
       m = m_new;
       float pr[2 * NJ];
       float ps = 0.f;
@@ -568,34 +594,33 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         pr[e] = fast_exp2(sc[e] - m);
         ps += pr[e];
       }
-      l = l * alpha + ps;
-#pragma unroll
-      for (int n = 0; n < RV / 8; ++n) {
-        o[n][0] *= alpha;
-        o[n][1] *= alpha;
-      }
+      l += ps;
 
       // ---- mix: per value group, p_t * scale_t,g as two digits of a per-row fixed point against the raw codes
 #pragma unroll
       for (int g = 0; g < NGV; ++g) {
-        float w[2 * NJ], wmax = 0.f, zsum = 0.f;
+        float w[2 * NJ], zsum = 0.f;
 #pragma unroll
         for (int e = 0; e < 2 * NJ; ++e) {
           w[e] = pr[e] * vs[g][e];
-          wmax = fmaxf(wmax, w[e]);
           zsum = fmaf(pr[e], vz[g][e], zsum);
         }
-        zc[g] = zc[g] * alpha + zsum;
+        float wmax = fmaxf(fmaxf(fmaxf(w[0], w[1]), fmaxf(w[2], w[3])), fmaxf(fmaxf(w[4], w[5]), fmaxf(w[6], w[7])));
+        zc[g] += zsum;
         wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, 1));
         wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, 2));
-        const float dp = wmax > 0.f ? wmax / kFixedMax : 1.f;
-        const float inv = 1.f / dp;
-        int hi[8], lo[8];
-#pragma unroll
-        for (int e = 0; e < 2 * NJ; ++e) digits(w[e], inv, hi[e], lo[e]);
+        // fixed-point step of this page's weights and its reciprocal: an approximate reciprocal is enough (the digits
+        // stand for w * inv * dp, and inv * dp = 1 to 2 ulp), and two IEEE divisions would sit on every page's critical chain
+        // (weights all below 1e-30 add nothing that fp32 accumulators holding O(1) sums could register: digits 0)
+        const bool live = wmax > 1e-30f;
+        const float dp = live ? wmax * (1.f / kFixedMax) : 1.f;
+        float inv;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(dp));
+        inv = live ? inv : 0.f;
         // k-slots 4 tid4 .. + 3 of the first 16 positions hold tiles 0 and 1, of the second 16 tiles 2 and 3
-        const uint32_t pa[4] = {pack4(hi[0], hi[1], hi[2], hi[3]), pack4(lo[0], lo[1], lo[2], lo[3]),
-                                pack4(hi[4], hi[5], hi[6], hi[7]), pack4(lo[4], lo[5], lo[6], lo[7])};
+        uint32_t pa[4];
+        digits4(w[0], w[1], w[2], w[3], inv, pa[0], pa[1]);
+        digits4(w[4], w[5], w[6], w[7], inv, pa[2], pa[3]);
         const int GT = (min(64 * g + 64, RV) - 64 * g) / 8;       // 8-channel tiles of the group: 8, or 4 / 6 in a short last group
         if constexpr (BITS == 8) {
 #pragma unroll

@@ -420,9 +420,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 if (row_ok) *reinterpret_cast<float2*>(a.v_params + (((size_t)row0 + lane) * ng + g) * 2) = make_float2(sc, zp);
               }
               const float inv = __fdiv_rn(1.f, sc);
+              // clamp(rint(y), 0, levels) = rint(clamp(y, 0, levels)); adding 1.5 * 2^23 rounds to the nearest integer, ties
+              // to even, and leaves it in the low mantissa bits: no float-to-int conversion on this busy path
               auto code = [&](int c, int e) -> uint32_t {
                 const float y = __fmul_rn(__fsub_rn(__uint_as_float(v[c][e]), zp), inv);
-                return (uint32_t)fminf(fmaxf(rintf(y), 0.f), kLevels);
+                return __float_as_uint(__fadd_rn(fminf(fmaxf(y, 0.f), kLevels), 12582912.f)) & 0xFFu;
               };
               const int tp = (row0 % kPage) + lane;                                   // token within its page
               if (t.side) {
