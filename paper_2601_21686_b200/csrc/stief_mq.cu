@@ -73,8 +73,10 @@ extern "C" int stief_mq_attention(const stief_layer* layer, const stief_batch* b
     return STIEF_ERR_INVALID_ARG;
   if (!host::aligned(q, 16) || !host::aligned(out, 16) || !host::aligned(layer->k_pool, 128) || !host::aligned(layer->v_pool, 128) ||
       (layer->U_k && !host::aligned(layer->U_k, 16)) || (layer->U_v && !host::aligned(layer->U_v, 16)) ||
-      layer->uk_head_stride % 8 || layer->uv_head_stride % 8)
+      layer->uk_head_stride % 8 || layer->uv_head_stride % 8 || layer->uk_head_stride < 0 || layer->uv_head_stride < 0)
     return STIEF_ERR_INVALID_ARG;
+  // the kernels compute pool rows (page * Hkv + head) * 64 in int
+  if ((long long)layer->num_pages * layer->Hkv * kPage >= (1ll << 31)) return STIEF_ERR_INVALID_ARG;
 
   const tc::Blocks bk = tc::blocks_of(RK), bv = tc::blocks_of(RV);
   const int TT = mq::kRows / G;

@@ -36,8 +36,14 @@
 // role walks to the end of its loops and TMEM is released.
 #pragma once
 
+#include <type_traits>
+
 #include "stief_kernels.h"
 #include "stief_tc.cuh"
+
+#ifndef STIEF_MQ_POLY_EVERY
+#define STIEF_MQ_POLY_EVERY 4
+#endif
 
 namespace stief {
 namespace mq {
@@ -51,6 +57,7 @@ constexpr int kCtrlBytes = 1024;
 constexpr int kSmemLimit = 232448;              // 227 KiB per CTA
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 6;
+constexpr int kPolyEvery = STIEF_MQ_POLY_EVERY;   // every kPolyEvery-th pair of exponentials runs as a polynomial on the FMA pipe
 constexpr float kRescaleLog2 = 8.0f;            // rescale the accumulator when a maximum grew by more than 2^8
 
 struct Args {
@@ -592,20 +599,27 @@ mq_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint64_t c2 = pack2(c, c), neg2 = pack2(-m_ref * c, -m_ref * c);
         uint64_t sum2 = pack2(0.f, 0.f);
         uint32_t pk[32];
+        // Part of the pairs go to the FMA pipe as a polynomial, where the exponentials and not the MMAs set the pace
+        // (small ranks).  The polynomial needs x >= -125 and cannot return an exact zero, so a page on which some row of
+        // the warp has masked positions (-inf) takes the special-function unit for all of them: two copies of the loop.
+        auto exponentials = [&](auto poly_tag) {
+          constexpr bool kPoly = decltype(poly_tag)::value;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float x0, x1, e0, e1;
-          unpack2(fma2(pack2(s[2 * i], s[2 * i + 1]), c2, neg2), x0, x1);
-          // every fourth pair on the FMA pipe, where the exponentials and not the MMAs set the pace (small ranks)
-          if ((RK + RV <= 160) && (i & 3) == 0) {
-            exp2_pair_fma(pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f)), e0, e1);
-          } else {
-            e0 = fast_exp2(x0);
-            e1 = fast_exp2(x1);
+          for (int i = 0; i < 32; ++i) {
+            float x0, x1, e0, e1;
+            unpack2(fma2(pack2(s[2 * i], s[2 * i + 1]), c2, neg2), x0, x1);
+            if (kPoly && (i % kPolyEvery) == 0) {
+              exp2_pair_fma(pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f)), e0, e1);
+            } else {
+              e0 = fast_exp2(x0);
+              e1 = fast_exp2(x1);
+            }
+            sum2 = add2(sum2, pack2(e0, e1));
+            pk[i] = pack_bf16(e0, e1);
           }
-          sum2 = add2(sum2, pack2(e0, e1));
-          pk[i] = pack_bf16(e0, e1);
-        }
+        };
+        if ((RK + RV <= 160) && !__any_sync(0xffffffffu, p0 + kPage - 1 > q_pos)) exponentials(std::true_type{});
+        else exponentials(std::false_type{});
         {
           float a0, a1;
           unpack2(sum2, a0, a1);
