@@ -406,6 +406,35 @@ def run_trace(args):
         segs.append(t[:, 10])
         combs.append(t[:, 11])
     assert int(status.item()) == 0
+    chain = None
+    if args.trace_chain:
+        # a chain of overlapped launches with the time stamps of two consecutive kernels: when does the next kernel's CTA
+        # enter an SM relative to the previous kernel's CTA leaving it, and how long is the SM without page traffic
+        ov = S.STIEF_DECODE_OVERLAP_PREVIOUS
+        gaps, idle, period = [], [], []
+        for rep_ in range(10):
+            trs = [torch.zeros(ns, S.TRACE_SLOTS, dtype=torch.int64, device=dev) for _ in range(2)]
+            torch.cuda.synchronize()
+            for i in range(8):
+                if i in (5, 6):
+                    S.stief_trace_next_decode_kernel(trs[i - 5])
+                S.stief_decode_step(layers[i % n_caches], batch, q, k_new, v_new, ws, out, num_parts=ns, status=status,
+                                    flags=ov if i else 0)
+            torch.cuda.synchronize()
+            a_, b_ = (t_.cpu().numpy().astype(np.float64) for t_ in trs)
+            a_, b_ = a_[a_[:, 0] > 0], b_[b_[:, 0] > 0]
+            exit_by_sm = {int(r[13]): r[9] for r in a_}
+            last_page_by_sm = {int(r[13]): r[6] for r in a_}
+            for r in b_:
+                sm = int(r[13])
+                if sm in exit_by_sm:
+                    gaps.append((r[0] - exit_by_sm[sm]) * 1e-3)          # previous CTA's exit -> this CTA's entry on the SM
+                    idle.append((r[4] - last_page_by_sm[sm]) * 1e-3)     # previous CTA's last page consumed -> first page landed
+            period.append((np.median(b_[:, 0]) - np.median(a_[:, 0])) * 1e-3)
+        chain = {"what": "overlapped chain, two consecutive kernels traced, matched by SM",
+                 "exit_to_next_entry_us": {"median": float(np.median(gaps)), "p90": float(np.percentile(gaps, 90))},
+                 "sm_without_page_traffic_us": {"median": float(np.median(idle)), "p90": float(np.percentile(idle, 90))},
+                 "entry_to_entry_us": float(np.median(period))}
     rel = np.stack(rel)                                                  # [launch, cta, slot]
     if args.trace_dump:                                                  # per-CTA table of the last launch, one line per CTA
         with open(args.trace_dump, "w") as f:
@@ -430,6 +459,7 @@ def run_trace(args):
         "stream_phase_us": {"median_cta": float(np.nanmedian(rel[:, :, 6] - rel[:, :, 4])),
                             "effective_gbs_over_first_landed_to_last_consumed":
                                 sb / (float(np.nanmedian(np.nanmax(rel[:, :, 6], axis=1) - np.nanmin(rel[:, :, 4], axis=1))) * 1e-6) / 1e9},
+        "chain": chain,
         "segments_per_cta": {"mean": float(np.mean(segs)), "max": float(np.max(segs))},
         "combines_per_cta": {"mean": float(np.mean(combs)), "max": float(np.max(combs))}}))
 
@@ -875,6 +905,7 @@ def main():
     ap.add_argument("--traffic-source", default=None, help="where --traffic comes from (profile file and commit of the capture)")
     ap.add_argument("--trace", action="store_true",
                     help="single-layer workloads: per-CTA time stamps of lone decode launches (where the time of a launch goes)")
+    ap.add_argument("--trace-chain", action="store_true", help="--trace: also trace two consecutive kernels of an overlapped chain")
     ap.add_argument("--trace-dump", default=None, help="--trace: also write the last launch's per-CTA table to this file")
     ap.add_argument("--seconds", type=float, default=0.6,
                     help="device time to collect by repeating the K-step timed region (the median region is reported)")

@@ -324,7 +324,7 @@ int stief_time_next_decode_kernel(void* start_event, void* stop_event);
  * never reached: 0 entry, 1 partition known, 2 first page request issued, 3 first segment's projections done,
  * 4 first page landed, 5 last page request issued, 6 last page consumed, 7 last partial stored, 8 last combine done,
  * 9 exit; words 10, 11 count the CTA's segments and the unit merges it performed; word 12 is the time at which the
- * last segment's arrival at its unit's counter was known.  One-shot; NULL cancels. */
+ * last segment's arrival at its unit's counter was known, word 13 the SM the CTA ran on.  One-shot; NULL cancels. */
 #define STIEF_TRACE_SLOTS 16
 int stief_trace_next_decode_kernel(uint64_t* trace, size_t trace_bytes);
 

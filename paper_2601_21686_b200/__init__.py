@@ -134,10 +134,17 @@ class Layer:
         return self.k_pool.shape[0]
 
     def c(self) -> _CLayer:
+        # the descriptor is rebuilt only when a tensor was replaced (marshalling is on the path of every step)
+        key = (_ptr(self.U_k), _ptr(self.U_v), _ptr(self.k_pool), _ptr(self.v_pool), self.Hq, self.Hkv, self.r_k, self.r_v)
+        cached = self.__dict__.get("_c")
+        if cached is not None and cached[0] == key:
+            return cached[1]
         uk_stride = 0 if self.U_k is None or self.U_k.shape[0] == 1 else self.U_k.stride(0)
         uv_stride = 0 if self.U_v is None or self.U_v.shape[0] == 1 else self.U_v.stride(0)
-        return _CLayer(self.Hq, self.Hkv, D_HEAD, self.r_k, self.r_v, self.num_pages, _ptr(self.U_k), uk_stride,
-                       _ptr(self.U_v), uv_stride, _ptr(self.k_pool), _ptr(self.v_pool))
+        st = _CLayer(self.Hq, self.Hkv, D_HEAD, self.r_k, self.r_v, self.num_pages, _ptr(self.U_k), uk_stride,
+                     _ptr(self.U_v), uv_stride, _ptr(self.k_pool), _ptr(self.v_pool))
+        self.__dict__["_c"] = (key, st)
+        return st
 
 
 @dataclass
@@ -178,7 +185,13 @@ class Batch:
     seq_lens: torch.Tensor
 
     def c(self) -> _CBatch:
-        return _CBatch(self.block_table.shape[0], self.block_table.shape[1], _ptr(self.block_table), _ptr(self.seq_lens))
+        key = (_ptr(self.block_table), _ptr(self.seq_lens), self.block_table.shape[0], self.block_table.shape[1])
+        cached = self.__dict__.get("_c")
+        if cached is not None and cached[0] == key:
+            return cached[1]
+        st = _CBatch(self.block_table.shape[0], self.block_table.shape[1], _ptr(self.block_table), _ptr(self.seq_lens))
+        self.__dict__["_c"] = (key, st)
+        return st
 
 
 def _check(rc: int, where: str):

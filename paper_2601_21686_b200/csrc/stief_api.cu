@@ -112,8 +112,37 @@ bool encode_u8_map(CUtensorMap* tm, const void* base, int rank, const unsigned l
 
 namespace {
 
-// pool viewed as a 2-D bf16 tensor [rows = num_pages*Hkv*64][r]; box = 64 rows x box-width, swizzle span = box row
+// pool viewed as a 2-D bf16 tensor [rows = num_pages*Hkv*64][r]; box = 64 rows x box-width, swizzle span = box row.
+// A descriptor is a pure function of (pool, r, rows); a decoder calls with the same few pools step after step, so the
+// last ones encoded by this thread are kept (encoding is a driver call on the path of every step).
+struct PoolMapEntry {
+  const void* pool;
+  int r;
+  long long rows;
+  CUtensorMap tm;
+};
+constexpr int kPoolMapCache = 128;
+thread_local PoolMapEntry g_pool_maps[kPoolMapCache];
+thread_local int g_pool_map_next = 0;
+
+bool encode_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows);
+
 bool make_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
+  for (int i = 0; i < kPoolMapCache; ++i) {
+    const PoolMapEntry& e = g_pool_maps[i];
+    if (e.pool == pool && e.r == r && e.rows == rows) {
+      *tm = e.tm;
+      return true;
+    }
+  }
+  if (!encode_pool_map(tm, pool, r, rows)) return false;
+  PoolMapEntry& e = g_pool_maps[g_pool_map_next];
+  g_pool_map_next = (g_pool_map_next + 1) % kPoolMapCache;
+  e.pool = pool; e.r = r; e.rows = rows; e.tm = *tm;
+  return true;
+}
+
+bool encode_pool_map(CUtensorMap* tm, const void* pool, int r, long long rows) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   const int span = decode_swizzle_span(r), bw = span / 2;

@@ -606,6 +606,9 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     stamp(trc, kTrExit);
     trc[kTrSegments] = (unsigned long long)n_seg;
     trc[kTrCombines] = (unsigned long long)n_comb;
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    trc[kTrSm] = smid;
   }
 }
 

@@ -37,6 +37,7 @@ enum TraceSlot {
   kTrSegments = 10,    // number of segments this CTA worked on (a count, not a time)
   kTrCombines = 11,    // number of unit combines this CTA performed (a count)
   kTrArrived = 12,     // last segment: arrival at the unit's counter known (a time)
+  kTrSm = 13,          // the SM the CTA ran on
   kTraceSlots = 16
 };
 
