@@ -281,6 +281,23 @@ def run_ours(args):
         sampler.stop()
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
+    # ---- context for the fraction: what a kernel that only reads gets from HBM (the peak in the denominator is a copy)
+    read_gbs = None
+    if rank == 0:
+        scratch = torch.empty(2 << 30, dtype=torch.uint8, device=dev)      # one launch reads 2 GiB: launch cost is out of the picture
+        for _ in range(2):
+            S.stief_measure_read_stream(scratch, status)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        r0.record()
+        for _ in range(5):
+            S.stief_measure_read_stream(scratch, status)
+        r1.record()
+        torch.cuda.synchronize()
+        read_gbs = 5 * scratch.numel() / (r0.elapsed_time(r1) * 1e-3) / 1e9
+        del scratch
+        assert int(status.item()) == 0
+
     # ---- max over ranks, region by region; then the median region
     def med(v):
         v = R.max_over_ranks(me, v, device=dev)
@@ -321,6 +338,10 @@ def run_ours(args):
             "tokens_per_s": world * B * K_steps / (ms * 1e-3), "seq_lens": seq_lengths(cfg) if cfg.get("ragged") else None,
             "frac_of_hbm_peak": value / world / hbm_peak, "hbm_peak_gbs": hbm_peak, "peak_kind": peak_kind,
             "frac_of_hbm_spec_8000": value / world / 8000.0,
+            "read_only_stream": {"gbs": read_gbs, "frac_of_it": value / world / read_gbs if read_gbs else None,
+                                 "what": "the decode kernel's streaming skeleton without its arithmetic over a 2 GiB buffer "
+                                         "(stief_measure_read_stream, CUDA events): what a read-only kernel gets from HBM, as context "
+                                         "for a fraction whose denominator is a copy"},
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": (B * Hq + 2 * B * Hkv) * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2, "ms_per_step": ms_host / K_steps,
                     "regions": {"count": n_reg_host, "median_ms": ms_host, "min_ms": ms_host_min, "max_ms": ms_host_max},

@@ -408,6 +408,14 @@ int stief_select_ranks(int32_t L, int32_t d_h, const int32_t* cand_k, int32_t n_
  * Asynchronous on `stream`. */
 int stief_selftest_wait_limit(int32_t* status, int32_t* report, int32_t poll_limit, void* stream);
 
+/* Measurement aid (no counterpart in the paper): one read-only pass over `bytes` (>= 16 KiB, rounded down to a multiple
+ * of 16 KiB) of the 16-byte aligned device buffer `buffer`, by the decode kernels' streaming skeleton without their
+ * arithmetic (one persistent CTA per SM, bulk async copies into a shared-memory ring); nothing is written.  Timed by the
+ * caller with events on `stream`, it gives the bandwidth a kernel that only reads can get from the memory system, as
+ * context for roofline fractions whose denominator is a copy (which reads and writes).  `status`: optional device word
+ * for STIEF_ERR_TIMEOUT. */
+int stief_measure_read_stream(const void* buffer, size_t bytes, int32_t* status, void* stream);
+
 const char* stief_status_string(int status);
 int stief_version(void);
 

@@ -98,6 +98,7 @@ def lib() -> ctypes.CDLL:
             "stief_select_ranks": (ctypes.c_int, [I32, I32, P, I32, P, I32, ctypes.c_double, P, _SURFACE_FN, P, P, P, P, P]),
             "stief_selftest_wait_limit": (ctypes.c_int, [P, P, I32, P]),
             "stief_trace_next_decode_kernel": (ctypes.c_int, [P, SZ]),
+            "stief_measure_read_stream": (ctypes.c_int, [P, SZ, P, P]),
             "stief_status_string": (ctypes.c_char_p, [ctypes.c_int]),
             "stief_version": (ctypes.c_int, []),
         }
@@ -486,3 +487,9 @@ def stief_q_decode_step(bits: int, layer: QLayer, batch: Batch, q: torch.Tensor,
     _check(_q("decode_step", bits)(ctypes.byref(cl), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), num_parts, _ptr(out), _ptr(out_lse),
                                    flags, _ptr(status), _stream()), f"stief_q{bits}_decode_step")
+
+
+def stief_measure_read_stream(buffer: torch.Tensor, status: Optional[torch.Tensor] = None):
+    """One read-only pass over a device tensor (time it with events): the bandwidth a kernel that only reads can get."""
+    _check(lib().stief_measure_read_stream(_ptr(buffer), buffer.numel() * buffer.element_size(), _ptr(status), _stream()),
+           "stief_measure_read_stream")

@@ -56,3 +56,76 @@ extern "C" int stief_selftest_wait_limit(int32_t* status, int32_t* report, int32
   stief::selftest_wait_kernel<<<1, 96, 0, static_cast<cudaStream_t>(stream)>>>(status, report, (uint32_t)poll_limit);
   return cudaGetLastError() == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------------------------------
+// stief_measure_read_stream: a read-only pass over a device buffer, for the roofline's context.  The usual denominator
+// is a copy (which reads AND writes); the decode kernels only read.  This is their streaming skeleton with the
+// arithmetic taken out: one persistent CTA per SM, four lanes of three 16 KiB stages each, every lane fed by its own
+// producer warp with 1-D bulk async copies that complete on an mbarrier, a consumer warp per lane that only waits for a
+// stage and hands it back.  Chunk i of the buffer goes to CTA i mod grid.  Nothing is written to global memory; every
+// wait is bounded.
+// ---------------------------------------------------------------------------------------------------------------------
+namespace stief {
+
+constexpr int kRsLanes = 4, kRsStages = 3, kRsChunk = 16384;
+
+__global__ void __launch_bounds__(2 * kRsLanes * 32, 1) read_stream_kernel(const uint8_t* __restrict__ p, long long n_chunks, int32_t* status) {
+  extern __shared__ uint8_t rs_smem[];
+  __shared__ __align__(8) unsigned long long bars[2 * kRsLanes * kRsStages];
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t ring = (smem_u32(rs_smem) + 127u) & ~127u;
+  auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
+  auto empty_bar = [&](int s) { return smem_u32(&bars[kRsLanes * kRsStages + s]); };
+  if (tid == 0) {
+    for (int s = 0; s < kRsLanes * kRsStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  volatile int* af = &abort_flag;
+  const int pl = warp % kRsLanes;
+  const bool producer = warp >= kRsLanes;
+  if (lane != 0) return;
+  // the CTA's chunks are c, c + grid, ...; its k-th chunk belongs to lane k % kRsLanes
+  long long k = 0;
+  for (long long i = blockIdx.x; i < n_chunks; i += gridDim.x, ++k) {
+    if ((int)(k % kRsLanes) != pl) continue;
+    const long long kw = k / kRsLanes;
+    const int slot = pl * kRsStages + (int)(kw % kRsStages);
+    const uint32_t phase = (uint32_t)((kw / kRsStages) & 1);
+    if (producer) {
+      if (kw >= kRsStages) mbar_wait(empty_bar(slot), phase ^ 1u, af, status);
+      mbar_arrive_expect_tx(full_bar(slot), kRsChunk);
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(ring + slot * kRsChunk), "l"(reinterpret_cast<uint64_t>(p + i * kRsChunk)), "r"(kRsChunk), "r"(full_bar(slot))
+                   : "memory");
+    } else {
+      mbar_wait(full_bar(slot), phase, af, status);
+      mbar_arrive(empty_bar(slot));
+    }
+  }
+}
+
+}  // namespace stief
+
+extern "C" int stief_measure_read_stream(const void* buffer, size_t bytes, int32_t* status, void* stream) {
+  if (!buffer || bytes < (size_t)stief::kRsChunk || (reinterpret_cast<uintptr_t>(buffer) & 15u)) return STIEF_ERR_INVALID_ARG;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    sms = 148;
+  }
+  const int smem = stief::kRsLanes * stief::kRsStages * stief::kRsChunk + 128;
+  static bool configured[64] = {};
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(stief::read_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return STIEF_ERR_CUDA;
+    configured[dev] = true;
+  }
+  stief::read_stream_kernel<<<sms, 2 * stief::kRsLanes * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint8_t*>(buffer), (long long)(bytes / stief::kRsChunk), status);
+  return cudaGetLastError() == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
+}
