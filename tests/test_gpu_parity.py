@@ -168,6 +168,39 @@ def test_rank_128_with_orthogonal_basis_is_exact_attention():
     U.check_out(out, ref, max_abs=3e-2, rel_l2=2e-2)
 
 
+@pytest.mark.parametrize("num_parts", [0, 5])
+def test_maximum_batch_of_tiny_sequences_fused_step(num_parts):
+    # B = 1024 (the limit of one call) with lengths 0 .. 130, many of them 0, 63, 64, 65: every CTA walks dozens of
+    # segments (its list of noted arrivals fills and is settled several times), empty sequences get their zero rows, and
+    # the appended row lands on and beside page boundaries.  One KV head, two query heads.
+    B, Hq, Hkv = 1024, 2, 1
+    special = [0, 1, 63, 64, 65, 127, 128, 129]
+    lens = [special[b % 8] if b % 3 else int(I.randint(I.stream_key(41, I.TAG_LENS), B, 0, 130)[b]) for b in range(B)]
+    c = U.make_case(41, B, Hq, Hkv, 32, 48, lens, reserve=2)
+    Kd, Vd = U.oracle_cache(c)
+    S.stief_prefill_compress(c.layer, c.batch, c.K.cuda(), c.V.cuda(), status=c.status)
+    k_new, v_new = I.new_token_kv(41, 0, B, Hkv)
+    ws = U.workspace_for(c, num_parts)
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+    S.stief_decode_step(c.layer, c.batch, c.q.cuda(), k_new.cuda(), v_new.cuda(), ws, out, num_parts=num_parts, out_lse=lse,
+                        status=c.status)
+    assert _sync_status(c) == 0
+    Uk, Uv = U.f64(c.U_k), U.f64(c.U_v)
+    kn, vn = U.f64(k_new), U.f64(v_new)
+    for b in range(B):
+        Kd[b] = np.concatenate([Kd[b], O.compress(kn[b, 0][None], O.basis_of(Uk, 0))[None]], 0)
+        Vd[b] = np.concatenate([Vd[b], O.compress(vn[b, 0][None], O.basis_of(Uv, 0))[None]], 0)
+    ref, ref_lse = O.decode_layer(U.f64(c.q), Kd, Vd, Uk, Uv, "b")
+    U.check_out(out, ref)
+    assert np.abs(lse.double().cpu().numpy() - ref_lse).max() < 2e-3
+    # B = 1025 is refused on the host
+    big = S.Batch(torch.zeros(1025, 4, dtype=torch.int32, device="cuda"), torch.zeros(1025, dtype=torch.int32, device="cuda"))
+    with pytest.raises(S.StiefError) as e:
+        S.stief_decode_attention(c.layer, big, c.q.cuda(), ws, num_parts, out)
+    assert e.value.code == S.STIEF_ERR_INVALID_ARG
+
+
 def test_append_and_decode_step_across_a_page_boundary():
     B, Hq, Hkv = 2, 8, 2
     c = U.make_case(40, B, Hq, Hkv, 48, 96, [62, 127], reserve=8)
