@@ -433,6 +433,8 @@ def run_trace(args):
         # enter an SM relative to the previous kernel's CTA leaving it, and how long is the SM without page traffic
         ov = S.STIEF_DECODE_OVERLAP_PREVIOUS
         gaps, idle, period = [], [], []
+        phases = {k_: [] for k_ in ("last_page_to_partial", "partial_to_arrived", "arrived_to_exit", "entry_to_partition",
+                                    "partition_to_first_request", "first_request_to_landed")}
         for rep_ in range(10):
             trs = [torch.zeros(ns, S.TRACE_SLOTS, dtype=torch.int64, device=dev) for _ in range(2)]
             torch.cuda.synchronize()
@@ -452,10 +454,18 @@ def run_trace(args):
                     gaps.append((r[0] - exit_by_sm[sm]) * 1e-3)          # previous CTA's exit -> this CTA's entry on the SM
                     idle.append((r[4] - last_page_by_sm[sm]) * 1e-3)     # previous CTA's last page consumed -> first page landed
             period.append((np.median(b_[:, 0]) - np.median(a_[:, 0])) * 1e-3)
+            for x_ in (a_, b_):                                           # slots: see stief.h
+                phases["last_page_to_partial"] += list((x_[:, 7] - x_[:, 6]) * 1e-3)
+                phases["partial_to_arrived"] += list((x_[:, 12] - x_[:, 7]) * 1e-3)
+                phases["arrived_to_exit"] += list((x_[:, 9] - x_[:, 12]) * 1e-3)
+                phases["entry_to_partition"] += list((x_[:, 1] - x_[:, 0]) * 1e-3)
+                phases["partition_to_first_request"] += list((x_[:, 2] - x_[:, 1]) * 1e-3)
+                phases["first_request_to_landed"] += list((x_[:, 4] - x_[:, 2]) * 1e-3)
         chain = {"what": "overlapped chain, two consecutive kernels traced, matched by SM",
                  "exit_to_next_entry_us": {"median": float(np.median(gaps)), "p90": float(np.percentile(gaps, 90))},
                  "sm_without_page_traffic_us": {"median": float(np.median(idle)), "p90": float(np.percentile(idle, 90))},
-                 "entry_to_entry_us": float(np.median(period))}
+                 "entry_to_entry_us": float(np.median(period)),
+                 "phases_us_median_p90": {k_: [float(np.median(v_)), float(np.percentile(v_, 90))] for k_, v_ in phases.items()}}
     rel = np.stack(rel)                                                  # [launch, cta, slot]
     if args.trace_dump:                                                  # per-CTA table of the last launch, one line per CTA
         with open(args.trace_dump, "w") as f:
