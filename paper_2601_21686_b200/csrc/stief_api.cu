@@ -25,8 +25,8 @@ cudaError_t launch_decode(const DecodeLaunch& a, const CUtensorMap& tmK, const C
 
 // Swizzle span (bytes) of the page-tile boxes of rank r, and whether the tile is fetched in its linear view
 // (must agree with Tile<R> in stief_common.cuh)
-int decode_swizzle_span(int r) { return r == 48 ? 32 : r == 96 ? 64 : (r % 64 == 0) ? 128 : 64; }
-bool decode_tile_linear(int r) { return r == 48 || r == 96; }
+int decode_swizzle_span(int r) { return r == 48 ? 32 : r == 96 ? 64 : 128; }
+bool decode_tile_linear(int r) { return r == 32 || r == 48 || r == 96; }
 
 namespace {
 

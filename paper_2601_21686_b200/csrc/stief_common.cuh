@@ -142,6 +142,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// one contiguous piece of global memory (16-byte aligned, a multiple of 16 bytes) into shared memory
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -195,21 +201,28 @@ __device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& hi, uin
 // ---------------------------------------------------------------------------------------------
 // swizzled page tiles in shared memory
 // ---------------------------------------------------------------------------------------------
-// A page tile holds 64 cache rows of R bf16 and is one contiguous block of 128 R bytes in the pool.  It is
-// fetched by TMA with a hardware swizzle chosen so that the eight 16-byte row pieces of an 8x8 ldmatrix tile
-// fall in distinct banks:
-//   R = 32, 64, 128 ("boxed"): boxes of 64 rows x min(R, 64) elements, swizzle span = box row (64 or 128 bytes);
-//                             R = 128 takes two boxes.
-//   R = 48, 96 ("linear"):    the block is viewed as lines of 32 (R = 48) or 64 (R = 96) bytes and fetched as ONE
-//                             box of 192 lines with that swizzle span; shared memory then holds the rows back to
-//                             back (row stride 2 R bytes) with the swizzle applied to the linear offset.  One
-//                             wide request instead of three narrow ones, and still conflict-free.
-// In both forms a step of 8 (or 16) rows leaves the swizzle term of an address unchanged, so the kernels add
-// plain multiples of 8 * RB to a per-lane base.
+// A page tile holds 64 cache rows of R bf16 and is one contiguous block of 128 R bytes in the pool.  The TMA unit
+// works through a box line by line, and at about one line per 1.3 cycles the line count, not the byte count,
+// bounds what an SM can request: narrow lines waste it.  So every tile is fetched with the widest lines its
+// ldmatrix access pattern allows:
+//   R = 64, 128 ("boxed"):  boxes of 64 rows x 64 elements with the 128-byte swizzle (R = 128 takes two boxes);
+//                           the eight 16-byte row pieces of an 8x8 ldmatrix tile fall in distinct banks.
+//   R = 32 ("linear"):      the block is viewed as 32 lines of 128 bytes (two cache rows per line) with the 128-byte
+//                           swizzle applied to the linear offset: conflict-free, half the lines of a 64-byte box.
+//   R = 96 ("linear"):      192 lines of 64 bytes with the 64-byte swizzle (conflict-free; wider lines would cost a
+//                           two-way conflict).
+//   R = 48 ("bulk"):        one 1-D bulk copy of the 6144 contiguous bytes, no swizzle: rows back to back at 96 bytes,
+//                           a two-way bank conflict on every ldmatrix, which is cheap beside the 192 lines of 32 bytes
+//                           that a conflict-free swizzled fetch needs (rank 48/48 decode: 37.1 -> 32.0 us).
+// A step of 16 rows leaves the swizzle term of an address unchanged in every form; a step of 8 rows does too except
+// for R = 32, where it flips the term's bit 6 for odd 8-row groups: K8X is that bit, to be XORed into a lane's base
+// offset (which addresses rows 0-7) before the plain multiple of 8 * RB is added.
 template <int R>
 struct Tile {
-  static constexpr bool LINEAR = (R == 48 || R == 96);
-  static constexpr int SW = (R == 48) ? 32 : (R == 96) ? 64 : (R % 64 == 0) ? 128 : 64;   // swizzle span, bytes
+  static constexpr bool LINEAR = (R == 32 || R == 48 || R == 96);
+  static constexpr bool BULK = (R == 48);                                  // fetched as one contiguous piece, unswizzled
+  static constexpr int SW = (R == 48) ? 32 : (R == 96) ? 64 : 128;          // swizzle span = line width, bytes (unused for BULK)
+  static constexpr uint32_t K8X = (R == 32) ? 64u : 0u;                     // see above
   static constexpr int BW = SW / 2;                                         // box width, elements
   static constexpr int NB = LINEAR ? 1 : (2 * R) / SW;                      // boxes per tile
   static constexpr int RB = LINEAR ? 2 * R : SW;                            // bytes from one token row to the next
@@ -219,7 +232,9 @@ struct Tile {
   static constexpr int BYTES = kPage * R * 2;
   // byte offset inside the tile of 16-byte chunk c (0 .. R/8-1) of row t
   __device__ static __forceinline__ uint32_t chunk(int t, int c) {
-    if constexpr (LINEAR) {
+    if constexpr (BULK) {
+      return static_cast<uint32_t>(t * RB + c * 16);
+    } else if constexpr (LINEAR) {
       uint32_t off = static_cast<uint32_t>(t * RB + c * 16);
       off ^= ((off >> 7) & (CPB - 1)) << 4;
       return off;

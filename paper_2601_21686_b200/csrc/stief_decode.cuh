@@ -219,12 +219,20 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
           const uint32_t st = ring + slot * C::STAGE_BYTES;
           const int tile = page * Hkv + h;
           mbar_arrive_expect_tx(full_bar(slot), C::STAGE_BYTES);
+          if constexpr (TK::BULK) {
+            bulk_load_1d(st, a.L.k_pool + (size_t)tile * kPage * RK, TK::BYTES, full_bar(slot));
+          } else {
 #pragma unroll
-          for (int nb = 0; nb < TK::NB; ++nb)
-            tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, TK::tma_x(nb), TK::tma_y(tile), full_bar(slot));
+            for (int nb = 0; nb < TK::NB; ++nb)
+              tma_load_2d(st + nb * TK::BOX_BYTES, &tmK, TK::tma_x(nb), TK::tma_y(tile), full_bar(slot));
+          }
+          if constexpr (TV::BULK) {
+            bulk_load_1d(st + TK::BYTES, a.L.v_pool + (size_t)tile * kPage * RV, TV::BYTES, full_bar(slot));
+          } else {
 #pragma unroll
-          for (int nb = 0; nb < TV::NB; ++nb)
-            tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, TV::tma_x(nb), TV::tma_y(tile), full_bar(slot));
+            for (int nb = 0; nb < TV::NB; ++nb)
+              tma_load_2d(st + TK::BYTES + nb * TV::BOX_BYTES, &tmV, TV::tma_x(nb), TV::tma_y(tile), full_bar(slot));
+          }
           if (pw == 0) {
             if (!issued) stamp(trc, kTrFirstIssue);
             issued = true;
@@ -455,13 +463,13 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 #pragma unroll
         for (int q4 = 0; 4 * q4 + 4 <= NCH; ++q4) {
           uint32_t r0, r1, r2, r3;
-          ldsm_x4(kt + koff[q4] + (hf * NJ + j) * 8 * TK::RB, r0, r1, r2, r3);
+          ldsm_x4(kt + (koff[q4] ^ ((j & 1) * TK::K8X)) + (hf * NJ + j) * 8 * TK::RB, r0, r1, r2, r3);
           mma_bf16(s, qa[2 * q4], r0, r1);
           mma_bf16(s, qa[2 * q4 + 1], r2, r3);
         }
         if constexpr (NCH % 4 == 2) {
           uint32_t r0, r1;
-          ldsm_x2(kt + koff[NCH / 4] + (hf * NJ + j) * 8 * TK::RB, r0, r1);
+          ldsm_x2(kt + (koff[NCH / 4] ^ ((j & 1) * TK::K8X)) + (hf * NJ + j) * 8 * TK::RB, r0, r1);
           mma_bf16(s, qa[NCH / 2 - 1], r0, r1);
         }
         sc[2 * j] = s[0] + s[2];

@@ -207,13 +207,6 @@ __device__ __forceinline__ void digits4(float x0, float x1, float x2, float x3, 
   lo = __byte_perm(w01, w23, 0x6420) ^ 0x80808080u;
 }
 
-// 1-D bulk async copy global -> shared (both 16-byte aligned, size a multiple of 16), completion in bytes on an mbarrier
-__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
 
 template <int RK, int RV, int BITS>
 __global__ void __launch_bounds__(DecodeQCfg<RK, RV, BITS>::THREADS, 1)
