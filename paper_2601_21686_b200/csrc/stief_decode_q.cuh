@@ -67,19 +67,16 @@ __host__ __device__ constexpr int q_groups(int r) { return (r + 63) / 64; }
 
 // Byte offset of 16-byte chunk c of row t in a shared-memory tile of 64 rows of ROWB bytes, as TMA leaves it:
 //   16, 48: dense rows (ldmatrix on 8 consecutive rows is conflict-free as it is)
-//   32:     32-byte swizzle;  64, 96, 128: the forms of Tile<> (64-byte swizzle, linear 32-byte swizzle, 128-byte swizzle)
+//   32, 64, 128: boxes of 64 rows with the swizzle span of the row (32-, 64-, 128-byte swizzle)
+//   96:     the tile viewed as 192 lines of 32 bytes, 32-byte swizzle on the linear offset
 // A step of 8 rows leaves the swizzle term unchanged in every form.
 template <int ROWB>
 __device__ __forceinline__ uint32_t qtile_chunk(int t, int c) {
-  if constexpr (ROWB == 16 || ROWB == 48) {
-    return static_cast<uint32_t>(t * ROWB + c * 16);
-  } else if constexpr (ROWB == 32) {
-    uint32_t off = static_cast<uint32_t>(t * 32 + c * 16);
-    off ^= ((off >> 7) & 1u) << 4;
-    return off;
-  } else {
-    return Tile<ROWB / 2>::chunk(t, c);
-  }
+  uint32_t off = static_cast<uint32_t>(t * ROWB + c * 16);
+  if constexpr (ROWB == 32 || ROWB == 96) off ^= ((off >> 7) & 1u) << 4;
+  if constexpr (ROWB == 64) off ^= ((off >> 7) & 3u) << 4;
+  if constexpr (ROWB == 128) off ^= ((off >> 7) & 7u) << 4;
+  return off;
 }
 
 // ---- where a code goes ------------------------------------------------------------------------------------------
