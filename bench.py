@@ -696,6 +696,10 @@ def run_multilayer(args):
     if args.rho is not None:
         # ranks from the library's own selector (Algorithm 2) on synthetic error surfaces of the shape the paper reports
         prof, _ = S.stief_select_ranks(L, I.RANK_SET, I.RANK_SET, args.rho, surfaces=I.error_surfaces(SEED, L))
+    elif args.ranks:
+        # every layer at the same ranks (not the named workload): separates what the mix of kernel variants costs
+        pairs = [tuple(int(x) for x in pr.split(",")) for pr in args.ranks.split(";")]
+        prof = [pairs[l % len(pairs)] for l in range(L)]
     else:
         prof = I.rank_profile(SEED)[:L]
     pg = I.make_paging(SEED, [T] * B, reserve_tokens=max(n_steps, 1) + 1)
@@ -719,7 +723,7 @@ def run_multilayer(args):
     torch.cuda.synchronize()
     ws = torch.empty(S.stief_decode_workspace_bytes(B, Hq, Hkv, 128, 0) // 4, dtype=torch.float32, device=dev)
     S.stief_decode_workspace_init(ws)
-    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    outs = [torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev) for _ in range(L)]   # overlapped kernels never share an output
     n_in = 4
     qs = [[I.queries(SEED, l, B, Hq, scale=1.0 / np.sqrt(128.0), device=dev, step=i) for l in range(L)] for i in range(n_in)]
     kvs = [[I.new_token_kv(SEED, l, B, Hkv, device=dev, step=i) for l in range(L)] for i in range(n_in)]
@@ -729,7 +733,7 @@ def run_multilayer(args):
         """One token for every sequence: append + attention in every layer, then advance the lengths."""
         for l in range(L):
             k_new, v_new = kvs[i % n_in][l]
-            S.stief_decode_step(layers[l], batch, qs[i % n_in][l], k_new, v_new, ws, out, status=status, flags=ov if l else 0)
+            S.stief_decode_step(layers[l], batch, qs[i % n_in][l], k_new, v_new, ws, outs[l], status=status, flags=ov if l else 0)
         S.stief_advance_seq_lens(lens, 1)
 
     cache_bytes_per_token = sum(Hkv * 2 * (rk + rv) for rk, rv in prof)      # per cached token, all layers
@@ -921,7 +925,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--q8", action="store_true", help="config 2 on the 8-bit quantised cache (measurement case)")
     ap.add_argument("--q4", action="store_true", help="config 2 on the 4-bit quantised cache (measurement case)")
-    ap.add_argument("--ranks", default=None, help="r_k,r_v override for the single-layer workloads, e.g. 48,96")
+    ap.add_argument("--ranks", default=None, help="r_k,r_v override for the single-layer workloads, e.g. 48,96; with config3/config5: every layer at these ranks, or several pairs separated by ; taken in turn")
     ap.add_argument("--layers", type=int, default=32, help="layers of the multi-layer workloads (config3, config5)")
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="launch every step's kernel fully serialised (no programmatic dependent launch)")

@@ -1,10 +1,20 @@
 // C-ABI entry points: argument checks, workspace carving, tensor-map encoding and kernel launches.
 // No allocation, no synchronisation; everything is enqueued on the caller's stream.
+#include <atomic>
 #include <cstring>
 
 #include "stief_host_util.h"
 
 namespace stief {
+
+namespace host {
+unsigned next_workspace_epoch() {
+  static std::atomic<unsigned> counter{0u};
+  unsigned e = counter.fetch_add(1u) + 1u;
+  if (e == 0u) e = counter.fetch_add(1u) + 1u;             // 0 means "not known"
+  return e;
+}
+}  // namespace host
 
 cudaError_t launch_decode_rk32(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
 cudaError_t launch_decode_rk48(const DecodeLaunch&, const CUtensorMap&, const CUtensorMap&, cudaStream_t);
@@ -193,7 +203,7 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   const int QT = query_tiles(layer->Hq, layer->Hkv);
   if ((long long)batch->B * (batch->max_pages_per_seq + seg_pad_pages(layer->r_k, layer->r_v)) * layer->Hkv * QT >= (1ll << 31))
     return STIEF_ERR_INVALID_ARG;
-  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
+  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta, workspace_bytes);
   if (w.bytes > workspace_bytes) return STIEF_ERR_WORKSPACE;
 
   const long long rows = (long long)layer->num_pages * layer->Hkv * kPage;
@@ -214,9 +224,16 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  a.partial_o = w.partial_o;
-  a.partial_lse = w.partial_lse;
-  a.counters = w.counters;
+  // fused launches alternate the workspace halves and publish their epoch; a partials-only launch keeps to half 0,
+  // where stief_split_combine looks for its results
+  const WorkspaceTurn turn = out ? take_workspace_turn(workspace) : take_workspace_half0(workspace);
+  a.partial_o = w.partial_o[turn.half];
+  a.partial_lse = w.partial_lse[turn.half];
+  a.counters = w.counters[turn.half];
+  a.control = w.control;
+  a.half = turn.half;
+  a.epoch = turn.epoch;
+  a.prev_epoch = dl.overlap_previous ? turn.prev_epoch : 0u;
   a.out = reinterpret_cast<__nv_bfloat16*>(out);
   a.out_lse = out ? out_lse : nullptr;
   a.len_add = len_add;
@@ -316,6 +333,7 @@ size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t 
 
 int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   if (!workspace || workspace_bytes == 0) return STIEF_ERR_INVALID_ARG;
+  forget_workspace(workspace);
   return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 
@@ -340,7 +358,7 @@ int stief_split_combine(const stief_layer* layer, const stief_batch* batch, int3
   const Workspace w = carve(const_cast<void*>(workspace), batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
   CombineArgs ca;
   ca.L = to_dev(layer); ca.Bt = host::to_dev(batch);
-  ca.partial_o = w.partial_o; ca.partial_lse = w.partial_lse;
+  ca.partial_o = w.partial_o[0]; ca.partial_lse = w.partial_lse[0];
   ca.n_cta = n_cta; ca.QT = query_tiles(layer->Hq, layer->Hkv); ca.len_add = len_add;
   ca.out = reinterpret_cast<__nv_bfloat16*>(out); ca.out_lse = out_lse;
   if ((long long)layer->Hkv * ca.QT > 2147483647ll || batch->B > 65535) return STIEF_ERR_INVALID_ARG;

@@ -153,6 +153,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   volatile int* n_pending = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);   // segments whose arrival is not yet counted
   constexpr int kMaxPending = 4;
   int* pending = reinterpret_cast<int*>(ctrl_ptr + 34 * 8);                           // [kMaxPending][4]: b, j, first CTA or -1, segments
+  volatile int* half_free = reinterpret_cast<volatile int*>(ctrl_ptr + 34 * 8 + kMaxPending * 16);   // see the producer
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -168,6 +169,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
     *abort_flag = 0;
     *n_pending = 0;
+    *half_free = 0;
     mbar_fence_init();
   }
   const int pad = seg_pad_pages(RK, RV);
@@ -194,6 +196,19 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
     }
+    // This kernel may overlap its predecessor, which works in the other half of the workspace.  What must be over
+    // before the consumers write into this half is the half's previous user, two launches back; it normally is by
+    // the time this CTA starts.  Producer 0 looks (here, and again after each segment while the answer is no) and
+    // leaves the answer in shared memory; consumers that find none there fall back to waiting for the predecessor
+    // grid to complete, which implies it.
+    auto look_at_half = [&]() {
+      if (pw == 0 && lane == 0 && a.prev_epoch != 0u && *half_free == 0) {
+        int seen;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.control + a.half) : "memory");
+        if ((unsigned)seen == a.prev_epoch) *half_free = 1;
+      }
+    };
+    look_at_half();
     int i_base = 0;            // pages of this CTA before the current segment
     bool issued = false;
     while (walk.next(seg)) {
@@ -241,6 +256,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         __syncwarp();
       }
       i_base += npg;
+      look_at_half();
     }
     if (pw == 0 && lane == 0) stamp(trc, kTrLastIssue);
     return;
@@ -553,9 +569,10 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     bar1(NT);
     const int u = b * upb + seg.j;
     const int slot_id = c + u;
-    // Everything up to here only read inputs (and appended this step's rows); the workspace and the
-    // outputs may still be in use by the kernel before this one when the launch overlaps it.
-    grid_dependency_wait();
+    // Everything up to here only read inputs (and appended this step's rows).  This half of the workspace may still
+    // be in use by its previous user when the launch overlaps earlier kernels: go on if producer 0 saw that user's
+    // epoch in the control word, else wait for the predecessor grid (which completes only after all before it).
+    if (*half_free == 0) grid_dependency_wait();
     for (int idx = tid; idx < ng * RV; idx += NT) {
       const int gg = idx / RV, j = idx % RV;
       float M = wm[gg];
@@ -596,8 +613,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   }
 
   // units of empty sequences get their zero rows from CTA (u mod n_cta)
+  int n_zero = 0;
   if (a.out != nullptr) {
-    grid_dependency_wait();
     for (int u = c; u < B * upb; u += n_cta) {
       const int b = u / upb, j = u % upb;
       if (pref[b + 1] != pref[b]) continue;
@@ -607,9 +624,28 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       const int d_out = a.L.U_v ? kD : RV;
       for (int idx = tid; idx < ng * d_out; idx += NT) a.out[head0 * d_out + idx] = __float2bfloat16_rn(0.f);
       if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
+      ++n_zero;
     }
   }
-  grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
+  // Every unit is finalised by exactly one CTA (merged, or zero-filled).  The CTA that finalises the kernel's last unit
+  // publishes the kernel's epoch: from then on this half of the workspace is free for its next user.  That CTA also
+  // waits for the predecessor grid before it leaves, so that this grid never completes before an earlier one (stream
+  // order stays transitive); the others leave at once and hand their SMs to the next kernel.
+  if (a.out == nullptr) {
+    grid_dependency_wait();
+  } else if (n_comb + n_zero > 0) {
+    bar1(NT);                                              // all of the CTA's reads of partials and writes of outputs are issued
+    if (tid == 0) {
+      __threadfence();
+      const int before = atomicAdd(a.control + 2 + a.half, n_comb + n_zero);
+      if (before + n_comb + n_zero == B * upb) {
+        a.control[2 + a.half] = 0;
+        __threadfence();
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.control + a.half), "r"((int)a.epoch) : "memory");
+        grid_dependency_wait();
+      }
+    }
+  }
   if (tid == 0 && trc) {
     stamp(trc, kTrExit);
     trc[kTrSegments] = (unsigned long long)n_seg;

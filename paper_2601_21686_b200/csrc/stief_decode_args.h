@@ -14,6 +14,13 @@ struct DecodeArgs {
   float* partial_o;              // [n_cta + n_units][8][RV]
   float* partial_lse;            // [n_cta + n_units][8]
   int* counters;                 // [n_units], zero on entry, zero again on exit (fused combine only)
+  // The three arrays above are one of the workspace's two halves.  control[half] holds the epoch of the last kernel
+  // that finished with this half, control[2 + half] counts the units this kernel has finalised.  A kernel whose
+  // launch overlaps its predecessor may write its half as soon as control[half] == prev_epoch (the half's previous
+  // user is done); prev_epoch == 0: not known, wait for the predecessor grid instead.
+  int* control;
+  int half;
+  unsigned epoch, prev_epoch;
   __nv_bfloat16* out;            // [B][Hq][128] or NULL (partials only)
   float* out_lse;                // [B][Hq] or NULL
   int len_add;                   // tokens attended beyond seq_lens (1 when appending)

@@ -19,6 +19,11 @@ static cudaError_t launch_one_q(const DecodeQArgs& a, int n_cta, bool overlap_pr
   if (dev >= 0 && dev < 64 && !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
+    // Every rank pair asks for the same (largest) shared-memory carve-out, whatever its ring needs: a kernel whose
+    // carve-out differs from its predecessor's cannot enter an SM before that SM has drained and been reconfigured,
+    // which undoes the overlap of consecutive layers when their ranks differ.
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   cudaLaunchConfig_t cfg = {};

@@ -39,14 +39,15 @@ def test_status_strings_and_version(lib):
 
 
 def test_workspace_planning(lib):
-    # counters [n_units] int32 | partial_o [parts + n_units][8][r_v] fp32 | partial_lse [parts + n_units][8] fp32
+    # 128 bytes of control words | counters [n_units] int32, twice | then twice (one per half of the workspace):
+    # partial_o [parts + n_units][8][r_v] fp32 | partial_lse [parts + n_units][8] fp32
     up = lambda x: (x + 127) // 128 * 128
-    n_units = 4 * 8 * 1
-    n = S.stief_decode_workspace_bytes(4, 32, 8, 64, 148)
-    assert n == up(n_units * 4) + up((148 + n_units) * 8 * 64 * 4) + up((148 + n_units) * 8 * 4)
+    size = lambda n_units, parts, r_v: 128 + 2 * up(n_units * 4) + 2 * (up((parts + n_units) * 8 * r_v * 4) + up((parts + n_units) * 8 * 4))
+    assert S.stief_decode_workspace_bytes(4, 32, 8, 64, 148) == size(4 * 8 * 1, 148, 64)
     # a group of 16 query heads per KV head is two units per (sequence, KV head)
-    n_units = 2 * 2 * 2
-    assert S.stief_decode_workspace_bytes(2, 32, 2, 96, 10) == up(n_units * 4) + up((10 + n_units) * 8 * 96 * 4) + up((10 + n_units) * 8 * 4)
+    assert S.stief_decode_workspace_bytes(2, 32, 2, 96, 10) == size(2 * 2 * 2, 10, 96)
+    # the built-in scratch of the workspace-free entry point holds 359 units at one part per SM of a B200 and r_v = 128
+    assert size(359, 148, 128) <= S.STATIC_WORKSPACE_BYTES < size(360, 148, 128)
     assert S.stief_decode_workspace_bytes(0, 32, 8, 64, 1) == 0
     assert S.stief_decode_workspace_bytes(4, 30, 8, 64, 1) == 0          # Hq not a multiple of Hkv
     assert S.stief_decode_num_parts() >= 1                                  # 148 when no device is present

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 
 
 # 128/128, 128/96, 96/128: two page lanes x two warps (tiles above 24 KiB); 96/96, 32/32, 48/48, 32/128: four lanes x one warp;
-# 48 and 96 use the linear tile form, 32/64/128 the boxed one
+# 64 and 128 use boxed tiles, 32 and 96 the linear forms, 48 the unswizzled bulk copy
 @pytest.mark.parametrize("r_k,r_v", [(128, 128), (128, 96), (96, 128), (96, 96), (32, 32), (48, 48), (32, 128), (64, 48)])
 def test_config2_shape_with_named_rank_pairs(r_k, r_v):
     c = DevCase(40 + r_k + 3 * r_v, 0, 4, 32, 8, r_k, r_v, [32768] * 4)
@@ -30,6 +30,46 @@ def test_config2_shape_with_named_rank_pairs(r_k, r_v):
     check_edge_pages(c)
     for b, h in ((0, 7), (2, 3)):
         check_pair(c, b, h, q, out, new_kv=[(kn, vn)], lens=c.seq_lens + 1)
+
+
+def test_overlapped_chain_of_long_and_short_kernels_matches_serial_launches():
+    # Layers of very different ranks chained with the overlap flag on ONE workspace, as a 32-layer step does: a short
+    # kernel (32/32) that follows a long one (128/128) has CTAs that are done long before the long kernel is, and they
+    # leave without waiting for it, so three and more kernels are in flight and the workspace halves, the epochs in its
+    # control words and the "last CTA waits" rule all get used.  Every step must equal the serial run bit for bit, and
+    # sampled pairs the oracle.
+    ranks = [(128, 128), (32, 32), (96, 128), (48, 32)]
+    pg = I.make_paging(7, [32768] * 4, reserve_tokens=2, extra_pages=1)
+    cs = [DevCase(70 + l, l, 4, 32, 8, rk, rv, [32768] * 4, paging=pg) for l, (rk, rv) in enumerate(ranks)]
+    for i, c in enumerate(cs):
+        S.stief_prefill_compress(c.layer, c.batch, c.K, c.V, status=c.status, flags=S.STIEF_PREFILL_OVERLAP_PREVIOUS if i else 0)
+    sync_ok(*cs)
+    ws = workspace(cs[0], r_v=128)
+    n_steps = 14
+    order = [0, 1, 2, 3, 1, 0, 3, 2, 0, 1, 1, 2, 0, 3]          # long -> short, short -> long, and a layer twice in a row
+    qs = [I.queries(7, order[i], 4, 32, scale=1.0 / np.sqrt(128.0), device=DEV, step=i) for i in range(n_steps)]
+    kvs = [I.new_token_kv(7, order[i], 4, 8, device=DEV, step=i) for i in range(n_steps)]
+    res = {}
+    for flags in (0, S.STIEF_DECODE_OVERLAP_PREVIOUS):
+        outs = [torch.full((4, 32, 128), float("nan"), dtype=torch.bfloat16, device=DEV) for _ in range(n_steps)]
+        lses = [torch.full((4, 32), float("nan"), dtype=torch.float32, device=DEV) for _ in range(n_steps)]
+        for i in range(n_steps):
+            c = cs[order[i]]
+            S.stief_decode_step(c.layer, c.batch, qs[i], kvs[i][0], kvs[i][1], ws, outs[i], out_lse=lses[i], status=c.status,
+                                flags=flags if i else 0)
+        sync_ok(*cs)
+        res[flags] = (outs, lses)
+    for i in range(n_steps):
+        assert torch.equal(res[0][0][i], res[1][0][i]), f"step {i}: outputs differ from the serial run"
+        assert torch.equal(res[0][1][i], res[1][1][i]), f"step {i}: log-sum-exps differ from the serial run"
+    # the workspace is clean for whoever comes next: counters and unit counts zero in both halves
+    n_ctrl = (128 + 2 * 128) // 4
+    ctrl = ws[:n_ctrl].view(torch.int32).cpu().numpy()
+    assert not ctrl[2:4].any() and not ctrl[32:].any()
+    last_of = {l: max(i for i in range(n_steps) if order[i] == l) for l in range(len(cs))}
+    for l, (b, h) in zip(range(len(cs)), ((0, 1), (1, 6), (2, 3), (3, 4))):
+        i = last_of[l]                                            # every step of a layer rewrites the same appended row
+        check_pair(cs[l], b, h, qs[i], res[1][0][i], new_kv=[kvs[i]], lens=cs[l].seq_lens + 1)
 
 
 class QDevCase:
