@@ -225,7 +225,7 @@ int stief_advance_seq_lens(int32_t* seq_lens, int32_t B, int32_t delta, void* st
  *    clears the counters it relies on (a cudaMemsetAsync on `stream`) before its kernel.  Two calls
  *    that overlap on the GPU -- different streams, or different host threads -- race on the array
  *    and give wrong results: serialise them. */
-#define STIEF_STATIC_WORKSPACE_BYTES (4u << 20)
+#define STIEF_STATIC_WORKSPACE_BYTES (8u << 20)
 int stief_decode_attention_static(const stief_layer* layer, const stief_batch* batch, const uint16_t* q,
                                   int32_t len_add, int32_t num_parts, uint16_t* out, float* out_lse,
                                   int32_t* status, void* stream);

@@ -292,7 +292,7 @@ def stief_decode_attention(layer: Layer, batch: Batch, q: torch.Tensor, workspac
                                         flags, _ptr(status), _stream()), "stief_decode_attention")
 
 
-STATIC_WORKSPACE_BYTES = 4 << 20
+STATIC_WORKSPACE_BYTES = 8 << 20
 
 
 def stief_decode_attention_static(layer: Layer, batch: Batch, q: torch.Tensor, out: torch.Tensor, num_parts: int = 0,

@@ -224,14 +224,14 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  // fused launches alternate the workspace halves and publish their epoch; a partials-only launch keeps to half 0,
-  // where stief_split_combine looks for its results
-  const WorkspaceTurn turn = out ? take_workspace_turn(workspace) : take_workspace_half0(workspace);
-  a.partial_o = w.partial_o[turn.half];
-  a.partial_lse = w.partial_lse[turn.half];
-  a.counters = w.counters[turn.half];
-  a.control = w.control;
-  a.half = turn.half;
+  // fused launches take the workspace sections in turn and publish their epoch; a partials-only launch keeps to
+  // section 0, where stief_split_combine looks for its results
+  const WorkspaceTurn turn = out ? take_workspace_turn(workspace) : take_workspace_section0(workspace);
+  a.partial_o = w.partial_o[turn.section];
+  a.partial_lse = w.partial_lse[turn.section];
+  a.counters = w.counters[turn.section];
+  a.finished = w.control + turn.section;
+  a.units_done = w.control + kWorkspaceSections + turn.section;
   a.epoch = turn.epoch;
   a.prev_epoch = dl.overlap_previous ? turn.prev_epoch : 0u;
   a.out = reinterpret_cast<__nv_bfloat16*>(out);

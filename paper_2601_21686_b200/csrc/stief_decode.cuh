@@ -153,7 +153,8 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   volatile int* n_pending = reinterpret_cast<volatile int*>(ctrl_ptr + 33 * 8 + 4);   // segments whose arrival is not yet counted
   constexpr int kMaxPending = 4;
   int* pending = reinterpret_cast<int*>(ctrl_ptr + 34 * 8);                           // [kMaxPending][4]: b, j, first CTA or -1, segments
-  volatile int* half_free = reinterpret_cast<volatile int*>(ctrl_ptr + 34 * 8 + kMaxPending * 16);   // see the producer
+  volatile int* section_free = reinterpret_cast<volatile int*>(ctrl_ptr + 34 * 8 + kMaxPending * 16);   // see the producer
+  volatile int* gate = section_free + 1;                   // thread 0's verdict for the segment at hand (see the merge)
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -169,7 +170,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
     *abort_flag = 0;
     *n_pending = 0;
-    *half_free = 0;
+    *section_free = 0;
     mbar_fence_init();
   }
   const int pad = seg_pad_pages(RK, RV);
@@ -196,19 +197,18 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
     }
-    // This kernel may overlap its predecessor, which works in the other half of the workspace.  What must be over
-    // before the consumers write into this half is the half's previous user, two launches back; it normally is by
-    // the time this CTA starts.  Producer 0 looks (here, and again after each segment while the answer is no) and
-    // leaves the answer in shared memory; consumers that find none there fall back to waiting for the predecessor
-    // grid to complete, which implies it.
-    auto look_at_half = [&]() {
-      if (pw == 0 && lane == 0 && a.prev_epoch != 0u && *half_free == 0) {
+    // This kernel may overlap its predecessors, which work in other sections of the workspace.  What must be over
+    // before the consumers write into this section is the section's previous user, a few launches back; it normally
+    // is by the time this CTA starts.  Producer 0 looks (here, and again after each segment while the answer is no)
+    // and leaves the answer in shared memory.
+    auto look_at_section = [&]() {
+      if (pw == 0 && lane == 0 && a.prev_epoch != 0u && *section_free == 0) {
         int seen;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.control + a.half) : "memory");
-        if ((unsigned)seen == a.prev_epoch) *half_free = 1;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.finished) : "memory");
+        if ((unsigned)seen == a.prev_epoch) *section_free = 1;
       }
     };
-    look_at_half();
+    look_at_section();
     int i_base = 0;            // pages of this CTA before the current segment
     bool issued = false;
     while (walk.next(seg)) {
@@ -256,7 +256,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         __syncwarp();
       }
       i_base += npg;
-      look_at_half();
+      look_at_section();
     }
     if (pw == 0 && lane == 0) stamp(trc, kTrLastIssue);
     return;
@@ -566,13 +566,24 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       wm[warp * 8 + gid] = m;
       wl[warp * 8 + gid] = l;
     }
+    // Everything up to here only read inputs (and appended this step's rows).  This section of the workspace may
+    // still be in use by its previous user when the launch overlaps earlier kernels.  Thread 0 settles the question
+    // for the CTA before the barrier: yes if producer 0 saw that user's epoch in the control word, else it looks once
+    // more itself; without a yes everyone waits for the predecessor grid (which completes only after all before it).
+    if (tid == 0) {
+      int go = *section_free;
+      if (go == 0 && a.prev_epoch != 0u) {
+        int seen;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.finished) : "memory");
+        go = (unsigned)seen == a.prev_epoch;
+        if (go) *section_free = 1;
+      }
+      *gate = go;
+    }
     bar1(NT);
     const int u = b * upb + seg.j;
     const int slot_id = c + u;
-    // Everything up to here only read inputs (and appended this step's rows).  This half of the workspace may still
-    // be in use by its previous user when the launch overlaps earlier kernels: go on if producer 0 saw that user's
-    // epoch in the control word, else wait for the predecessor grid (which completes only after all before it).
-    if (*half_free == 0) grid_dependency_wait();
+    if (*gate == 0) grid_dependency_wait();
     for (int idx = tid; idx < ng * RV; idx += NT) {
       const int gg = idx / RV, j = idx % RV;
       float M = wm[gg];
@@ -637,11 +648,11 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     bar1(NT);                                              // all of the CTA's reads of partials and writes of outputs are issued
     if (tid == 0) {
       __threadfence();
-      const int before = atomicAdd(a.control + 2 + a.half, n_comb + n_zero);
+      const int before = atomicAdd(a.units_done, n_comb + n_zero);
       if (before + n_comb + n_zero == B * upb) {
-        a.control[2 + a.half] = 0;
+        *a.units_done = 0;
         __threadfence();
-        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.control + a.half), "r"((int)a.epoch) : "memory");
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.finished), "r"((int)a.epoch) : "memory");
         grid_dependency_wait();
       }
     }

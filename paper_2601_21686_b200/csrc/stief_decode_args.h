@@ -14,12 +14,12 @@ struct DecodeArgs {
   float* partial_o;              // [n_cta + n_units][8][RV]
   float* partial_lse;            // [n_cta + n_units][8]
   int* counters;                 // [n_units], zero on entry, zero again on exit (fused combine only)
-  // The three arrays above are one of the workspace's two halves.  control[half] holds the epoch of the last kernel
-  // that finished with this half, control[2 + half] counts the units this kernel has finalised.  A kernel whose
-  // launch overlaps its predecessor may write its half as soon as control[half] == prev_epoch (the half's previous
-  // user is done); prev_epoch == 0: not known, wait for the predecessor grid instead.
-  int* control;
-  int half;
+  // The three arrays above are one section of the workspace.  *finished holds the epoch of the last kernel that
+  // finished with this section, *units_done counts the units this kernel has finalised.  A kernel whose launch
+  // overlaps its predecessors may write its section as soon as *finished == prev_epoch (the section's previous user
+  // is done); prev_epoch == 0: not known, wait for the predecessor grid instead.
+  int* finished;
+  int* units_done;
   unsigned epoch, prev_epoch;
   __nv_bfloat16* out;            // [B][Hq][128] or NULL (partials only)
   float* out_lse;                // [B][Hq] or NULL

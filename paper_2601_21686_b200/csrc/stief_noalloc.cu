@@ -51,11 +51,11 @@ extern "C" int stief_decode_attention_static(const stief_layer* layer, const sti
   void* ws = nullptr;
   const int rc = static_workspace(&ws);
   if (rc != STIEF_OK) return rc;
-  // The array keeps whatever the previous call left.  Only the control words and the arrival counters of the two
-  // halves, which sit at its start, must be zero on entry (a call that ended with a device-side error may have left
-  // them non-zero): 128 bytes, then twice the counters rounded up to 128 bytes.
+  // The array keeps whatever the previous call left.  Only the control words and the arrival counters of its four
+  // sections, which sit at its start, must be zero on entry (a call that ended with a device-side error may have left
+  // them non-zero): 128 bytes, then four times the counters rounded up to 128 bytes.
   const size_t groups = (size_t)(layer->Hq / layer->Hkv + 7) / 8;
-  const size_t counter_bytes = 128 + 2 * (((size_t)batch->B * layer->Hkv * groups * 4 + 127) / 128 * 128);
+  const size_t counter_bytes = 128 + 4 * (((size_t)batch->B * layer->Hkv * groups * 4 + 127) / 128 * 128);
   if (cudaMemsetAsync(ws, 0, counter_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return STIEF_ERR_CUDA;
   return stief_decode_attention(layer, batch, q, len_add, ws, (size_t)STIEF_STATIC_WORKSPACE_BYTES, num_parts, out, out_lse,
                                 0u, status, stream);

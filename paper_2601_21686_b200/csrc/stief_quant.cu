@@ -218,8 +218,8 @@ int run_q_decode(int bits, const stief_qlayer* layer, const stief_batch* batch, 
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  // this kernel keeps to the plain dependency wait before it touches the workspace: half 0, no epoch published
-  take_workspace_half0(workspace);
+  // this kernel keeps to the plain dependency wait before it touches the workspace: section 0, no epoch published
+  take_workspace_section0(workspace);
   a.partial_o = w.partial_o[0]; a.partial_lse = w.partial_lse[0]; a.counters = w.counters[0];
   a.out = reinterpret_cast<__nv_bfloat16*>(out);
   a.out_lse = out_lse;

@@ -39,10 +39,10 @@ def test_status_strings_and_version(lib):
 
 
 def test_workspace_planning(lib):
-    # 128 bytes of control words | counters [n_units] int32, twice | then twice (one per half of the workspace):
-    # partial_o [parts + n_units][8][r_v] fp32 | partial_lse [parts + n_units][8] fp32
+    # 128 bytes of control words | counters [n_units] int32, once per section | then per section:
+    # partial_o [parts + n_units][8][r_v] fp32 | partial_lse [parts + n_units][8] fp32; four sections
     up = lambda x: (x + 127) // 128 * 128
-    size = lambda n_units, parts, r_v: 128 + 2 * up(n_units * 4) + 2 * (up((parts + n_units) * 8 * r_v * 4) + up((parts + n_units) * 8 * 4))
+    size = lambda n_units, parts, r_v: 128 + 4 * up(n_units * 4) + 4 * (up((parts + n_units) * 8 * r_v * 4) + up((parts + n_units) * 8 * 4))
     assert S.stief_decode_workspace_bytes(4, 32, 8, 64, 148) == size(4 * 8 * 1, 148, 64)
     # a group of 16 query heads per KV head is two units per (sequence, KV head)
     assert S.stief_decode_workspace_bytes(2, 32, 2, 96, 10) == size(2 * 2 * 2, 10, 96)

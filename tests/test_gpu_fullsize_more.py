@@ -35,7 +35,7 @@ def test_config2_shape_with_named_rank_pairs(r_k, r_v):
 def test_overlapped_chain_of_long_and_short_kernels_matches_serial_launches():
     # Layers of very different ranks chained with the overlap flag on ONE workspace, as a 32-layer step does: a short
     # kernel (32/32) that follows a long one (128/128) has CTAs that are done long before the long kernel is, and they
-    # leave without waiting for it, so three and more kernels are in flight and the workspace halves, the epochs in its
+    # leave without waiting for it, so three and more kernels are in flight and the workspace sections, the epochs in its
     # control words and the "last CTA waits" rule all get used.  Every step must equal the serial run bit for bit, and
     # sampled pairs the oracle.
     ranks = [(128, 128), (32, 32), (96, 128), (48, 32)]
@@ -62,10 +62,10 @@ def test_overlapped_chain_of_long_and_short_kernels_matches_serial_launches():
     for i in range(n_steps):
         assert torch.equal(res[0][0][i], res[1][0][i]), f"step {i}: outputs differ from the serial run"
         assert torch.equal(res[0][1][i], res[1][1][i]), f"step {i}: log-sum-exps differ from the serial run"
-    # the workspace is clean for whoever comes next: counters and unit counts zero in both halves
-    n_ctrl = (128 + 2 * 128) // 4
-    ctrl = ws[:n_ctrl].view(torch.int32).cpu().numpy()
-    assert not ctrl[2:4].any() and not ctrl[32:].any()
+    # the workspace is clean for whoever comes next: 32 control words (four epochs, four unit counts that must be zero
+    # again), then the arrival counters of the four sections (32 units each here), all zero
+    ctrl = ws[:32 + 4 * 32].view(torch.int32).cpu().numpy()
+    assert ctrl[:4].all() and not ctrl[4:].any()
     last_of = {l: max(i for i in range(n_steps) if order[i] == l) for l in range(len(cs))}
     for l, (b, h) in zip(range(len(cs)), ((0, 1), (1, 6), (2, 3), (3, 4))):
         i = last_of[l]                                            # every step of a layer rewrites the same appended row
