@@ -132,33 +132,50 @@ int stief_append_chunk(const stief_layer* layer, const stief_batch* batch, const
  * chunk-normalised partial result.  num_parts = 0 lets the library choose (one CTA per SM of the current device, which is also
  * what stief_decode_num_parts returns); it must not exceed 65535.  The same num_parts must be given
  * to stief_decode_workspace_bytes and to every call that shares the workspace.
- * Workspace layout, n_units = B * Hkv * ceil((Hq/Hkv) / 8):
- *   counters    int32 [n_units]                    arrivals per unit; zero between calls
+ * Workspace layout, n_units = B * Hkv * ceil((Hq/Hkv) / 8).  Kernels of an overlapped chain (see the flag below) may be
+ * at work on one workspace at the same time, so what a kernel writes exists in four sections that consecutive fused
+ * launches take in turn:
+ *   control     int32 [32]                       words 0-3: per section, the epoch (a number the library gives every
+ *                                                launch) of the last kernel that finished with it; words 4-7: per
+ *                                                section, units finalised by the kernel now using it; zero between calls
+ *   counters    int32 [4][n_units]               arrivals per unit (each section's array padded to 128 bytes); zero between calls
+ *   then per section, sections at equal distances that depend on the buffer's size only (layers of different r_v share
+ *   a workspace, so give every call on a buffer the same workspace_bytes):
  *   partial_o   fp32  [num_parts + n_units][8][r_v]  chunk-normalised mixes p V_down (compressed space)
  *   partial_lse fp32  [num_parts + n_units][8]       natural-log sum-exp of each segment's scores
+ * A call with out == NULL (partials for stief_split_combine) always uses section 0.
  * The buffer must be 128-byte aligned and must be cleared once with stief_decode_workspace_init
  * (a cudaMemsetAsync of the whole buffer) before its first use; calls that end normally leave the
- * counters zero again.  Calls that share a workspace must not overlap on the GPU.  B <= 1024. */
+ * counters zero again.  Which section comes next is remembered per host thread and buffer address; a thread that meets
+ * a buffer for the first time merely waits more than it must for a few launches.  Apart from the flagged chains below,
+ * calls that share a workspace must not overlap on the GPU.  B <= 1024. */
 int32_t stief_decode_num_parts(void);
 size_t stief_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t r_v, int32_t num_parts);
 int stief_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Flags of the decode calls.
- * STIEF_DECODE_OVERLAP_PREVIOUS: the kernel may start before the kernel that precedes it on the stream
- * has finished (programmatic dependent launch): it takes over each SM as the earlier kernel's work there
- * ends, reads its inputs, appends this step's rows and streams the cache, and only then waits for the
- * earlier kernel to complete before it first touches `workspace`, `out` and `out_lse`.  Back-to-back
- * decode kernels (the layers of one step) then run without an idle gap between them.  By setting the
- * flag the caller promises that the preceding kernel on the stream writes none of this call's inputs
- * (q, k_new, v_new, seq_lens, block_table, the bases, this layer's pools) and does not read the cache
- * rows this call appends.  Two consecutive decode calls of this library on different layers satisfy
- * that; a call that follows stief_advance_seq_lens, or whose q is produced by the preceding kernel,
- * does not.  If the preceding stream operation is not a kernel the flag has no effect.
- * Chains: the promise is about the ONE kernel directly before.  In an unbroken run of flagged calls at most two
- * kernels are ever on the GPU together: a kernel's CTAs stay resident until the kernel before it has completed
- * and each fills more than half of an SM, so the kernel after next cannot begin until the one before has gone.
- * That argument needs a grid of at least one CTA per SM, so the flag is honoured only when num_parts is 0 or at
- * least the SM count; with fewer parts the launch is silently serialised (same results, no overlap). */
+ * STIEF_DECODE_OVERLAP_PREVIOUS: the kernel may start before the kernels that precede it on the stream have finished
+ * (programmatic dependent launch): it takes over each SM as earlier work there ends, reads its inputs, appends this
+ * step's rows and streams the cache.  Before a CTA first writes the workspace it makes sure that the previous user of
+ * its workspace section (four launches back) has finished, which it reads from the section's control word; it does
+ * NOT wait for the kernel directly before it, so the CTAs of a short kernel that follows a long one finish, leave and
+ * hand their SMs on while the long one still runs: the layers of one step, whatever their ranks, run without idle SMs
+ * between them.  One CTA of every kernel (the one that finalises its last unit) waits for the preceding kernel to
+ * complete before it leaves, so kernels still COMPLETE in stream order and whatever follows the chain on the stream
+ * sees all of its results.
+ * By setting the flag the caller promises, for every kernel of the unbroken run of flagged calls that ends directly
+ * before this one (and the unflagged call that heads the run): it writes none of this call's inputs (q, k_new, v_new,
+ * seq_lens, block_table, the bases, this layer's pools), does not read the cache rows this call appends, and neither
+ * reads nor writes this call's out and out_lse.  Consecutive decode calls of this library on different layers, each
+ * with its own output buffer, satisfy that; a call that follows stief_advance_seq_lens, or whose q is produced by the
+ * preceding kernel, does not.  If the preceding stream operation is not a kernel the flag has no effect.
+ * A layer may come up again within one run (a benchmark that repeats a step without advancing seq_lens): every call
+ * attends to its own new token, whatever the other calls store, but which call's rows the pool keeps at that position
+ * is then not defined unless all of them append the same rows.
+ * The flag is honoured only when num_parts is 0 or at least the SM count; with fewer parts the launch is silently
+ * serialised (same results, no overlap).  When the library cannot tell who used the section last (first launches on a
+ * buffer, another host thread, a replayed graph's first nodes) the kernel falls back to waiting for the kernel
+ * directly before it, which is always sufficient because of the completion order above. */
 #define STIEF_DECODE_OVERLAP_PREVIOUS 1u
 
 /* Decode attention (Eq. 18 on the reconstructions of Eq. 7, one query row per head): q [B][Hq][128]

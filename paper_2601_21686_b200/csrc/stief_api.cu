@@ -213,10 +213,9 @@ int run_decode(const stief_layer* layer, const stief_batch* batch, const uint16_
 
   DecodeLaunch dl;
   dl.n_cta = n_cta;
-  // The early start is only honoured for a grid that covers every SM.  A CTA of these kernels takes more than half of
-  // an SM's shared memory and stays resident until its predecessor grid has completed, so with >= one CTA per SM the
-  // grid after next cannot start before the grid before has left the GPU: at most two kernels of a chain overlap.  A
-  // smaller grid would let a third kernel in, which could append a row its pre-predecessor is still streaming.
+  // The early start is only honoured for a grid that covers every SM: a smaller grid leaves SMs free, its successor
+  // would start on them at once and the two would share the memory system for their whole length instead of handing
+  // SMs over.
   dl.overlap_previous = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0 && n_cta >= sm_count();
   DecodeArgs& a = dl.args;
   a.L = to_dev(layer);

@@ -48,7 +48,8 @@ def test_overlapped_chain_of_long_and_short_kernels_matches_serial_launches():
     n_steps = 14
     order = [0, 1, 2, 3, 1, 0, 3, 2, 0, 1, 1, 2, 0, 3]          # long -> short, short -> long, and a layer twice in a row
     qs = [I.queries(7, order[i], 4, 32, scale=1.0 / np.sqrt(128.0), device=DEV, step=i) for i in range(n_steps)]
-    kvs = [I.new_token_kv(7, order[i], 4, 8, device=DEV, step=i) for i in range(n_steps)]
+    # a layer that comes up again within the run appends the same rows (else which rows the pool keeps is not defined)
+    kvs = [I.new_token_kv(7, order[i], 4, 8, device=DEV, step=0) for i in range(n_steps)]
     res = {}
     for flags in (0, S.STIEF_DECODE_OVERLAP_PREVIOUS):
         outs = [torch.full((4, 32, 128), float("nan"), dtype=torch.bfloat16, device=DEV) for _ in range(n_steps)]
