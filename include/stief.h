@@ -92,13 +92,14 @@ typedef struct stief_batch {
  * contiguous blocks of 128 elements (r elements on a side without basis); rows must be 16-byte aligned.  T_max bounds seq_lens (it sizes the launch; tokens
  * beyond seq_lens[b] are never stored; the input rows of a sequence's last 128-token tile are read up
  * to T_max).
- * flags: 0, or STIEF_PREFILL_OVERLAP_PREVIOUS: the kernel may start (and write its pools) before the kernel
- * that precedes it on the stream has finished, so that the per-layer launches of one prompt run without
- * idle gaps.  By setting it the caller promises that the preceding kernel neither writes this call's
- * inputs (K, V, seq_lens, block_table, the bases) nor touches this layer's pools; consecutive calls for
- * different layers satisfy that.  The kernel still completes only after its predecessor has.  The grid always has
- * one CTA per SM and every CTA stays resident until the preceding kernel has completed, so in a run of flagged
- * calls no more than two kernels overlap: the promise concerns the directly preceding kernel only. */
+ * flags: 0, or STIEF_PREFILL_OVERLAP_PREVIOUS: the kernel may start (and write its pools) before the kernels that
+ * precede it on the stream have finished, so that the per-layer launches of one prompt run without idle gaps.  The grid
+ * has one CTA per SM; a CTA takes over an SM as earlier work there ends and leaves it as soon as its own tiles are
+ * stored, whether or not the kernel before it is still at work, so several kernels of a run of flagged calls can be in
+ * flight.  By setting the flag the caller promises that no kernel of the unbroken run of flagged calls before this one
+ * (nor the unflagged call that heads it) writes this call's inputs (K, V, seq_lens, block_table, the bases) or touches
+ * this layer's pools; consecutive calls for different layers satisfy that.  One CTA of the kernel waits for the
+ * preceding kernel to complete before it leaves, so kernels still complete in stream order. */
 #define STIEF_PREFILL_OVERLAP_PREVIOUS 1u
 int stief_prefill_compress(const stief_layer* layer, const stief_batch* batch, const uint16_t* K,
                            const uint16_t* V, int64_t stride_b, int64_t stride_t, int64_t v_stride_b,

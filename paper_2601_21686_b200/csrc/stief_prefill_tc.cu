@@ -547,7 +547,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   }
 
   if (warp >= 2 && lane == 0) bulk_wait_all();            // this lane's TMA stores are complete
-  grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
+  // Never complete before the kernel this one was allowed to overlap (stream order stays transitive).  One CTA that
+  // waits is enough for that; the others leave and hand their SMs to the next kernel, also when the kernel before
+  // this one is a longer one that is still at work.
+  if (blockIdx.x == 0) grid_dependency_wait();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
