@@ -319,7 +319,9 @@ int stief_q4_decode_attention(const stief_qlayer* layer, const stief_batch* batc
 
 /* One decode step of one layer on the quantised cache in one launch: project, quantise and store (k_new, v_new)
  * at position seq_lens[b], then attend over seq_lens[b] + 1 tokens.  Same result as the append call followed by the
- * attention call with len_add = 1. */
+ * attention call with len_add = 1.  With STIEF_DECODE_OVERLAP_PREVIOUS: this kernel reads its new token's codes back
+ * from the pools, so a layer must not come up again within one run of flagged calls unless every such call appends
+ * the same rows. */
 int stief_q8_decode_step(const stief_qlayer* layer, const stief_batch* batch, const uint16_t* q, const uint16_t* k_new,
                          const uint16_t* v_new, void* workspace, size_t workspace_bytes, int32_t num_parts,
                          uint16_t* out, float* out_lse, uint32_t flags, int32_t* status, void* stream);

@@ -48,6 +48,10 @@ struct DecodeQArgs {
   float* partial_o;
   float* partial_lse;
   int* counters;
+  // one section of the workspace, its control words and the epochs: as in DecodeArgs
+  int* finished;
+  int* units_done;
+  unsigned epoch, prev_epoch;
   __nv_bfloat16* out;
   float* out_lse;
   int len_add;
@@ -232,6 +236,8 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   float* lse_shift = reinterpret_cast<float*>(ctrl_ptr + 34 * 8);      // [8]: q' . key zero-point / sqrt(128) of the unit's rows
   float* q_delta = reinterpret_cast<float*>(ctrl_ptr + 38 * 8);        // [8]: fixed-point step of the unit's scaled query rows
   volatile int* append_done = reinterpret_cast<volatile int*>(ctrl_ptr + 32 * 8);   // appending segments whose rows are stored
+  volatile int* section_free = reinterpret_cast<volatile int*>(ctrl_ptr + 42 * 8);  // the workspace section's previous user is done
+  volatile int* gate = section_free + 1;                                            // thread 0's verdict for the segment at hand
   int* pref = reinterpret_cast<int*>(ctrl_ptr + C::CTRL_BYTES);
   float* qp = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES);
   float* un = reinterpret_cast<float*>(ctrl_ptr + C::CTRL_BYTES + C::PREF_BYTES + C::QP_BYTES);
@@ -244,6 +250,7 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mbar_init(empty_bar(s), HALF);
     }
     *abort_flag = 0;
+    *section_free = 0;
     *last_flag = 0;
     *append_done = 0;
     mbar_fence_init();
@@ -272,6 +279,16 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmV);
     }
+    // Consecutive launches take the workspace sections in turn; before the consumers write into this one its previous
+    // user must be done, which the section's control word tells (decode_persistent_kernel does the same).
+    auto look_at_section = [&]() {
+      if (pw == 0 && lane == 0 && a.prev_epoch != 0u && *section_free == 0) {
+        int seen;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.finished) : "memory");
+        if ((unsigned)seen == a.prev_epoch) *section_free = 1;
+      }
+    };
+    look_at_section();
     int i_base = 0;            // pages of this CTA before the current segment
     int n_append = 0;          // appending segments of this CTA so far
     while (walk.next(seg)) {
@@ -317,6 +334,7 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       }
       i_base += npg;
       if (wait_append) ++n_append;
+      look_at_section();
     }
     return;
   }
@@ -342,6 +360,7 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t voff = BITS == 8 ? qtile_chunk<64>(l7 + 8 * (lane >> 4), 2 * hf + ((lane >> 3) & 1))
                                   : qtile_chunk<32>(l7 + 8 * (lane >> 3), hf);
   int i_base = 0;              // pages of this CTA before the current segment
+  int n_final = 0;             // units this CTA finalised (merged or zero-filled)
 
   while (walk.next(seg)) {
     const int b = seg.b, h = seg.j / QT, qt = seg.j % QT;
@@ -674,12 +693,24 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       wm[warp * 8 + gid] = m;
       wl[warp * 8 + gid] = l;
     }
+    // Everything up to here only read inputs (and appended this step's rows).  This section of the workspace may
+    // still be in use by its previous user when the launch overlaps earlier kernels.  Thread 0 settles the question
+    // for the CTA before the barrier: yes if producer 0 saw that user's epoch in the control word, else it looks once
+    // more itself; without a yes everyone waits for the predecessor grid (which completes only after all before it).
+    if (tid == 0) {
+      int go = *section_free;
+      if (go == 0 && a.prev_epoch != 0u) {
+        int seen;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.finished) : "memory");
+        go = (unsigned)seen == a.prev_epoch;
+        if (go) *section_free = 1;
+      }
+      *gate = go;
+    }
     bar1(NT);
     const int u = b * upb + seg.j;
     const int slot_id = c + u;
-    // Everything up to here only read inputs (and appended this step's rows); the workspace and the
-    // outputs may still be in use by the kernel before this one when the launch overlaps it.
-    grid_dependency_wait();
+    if (*gate == 0) grid_dependency_wait();
     for (int idx = tid; idx < ng * RV; idx += NT) {
       const int gg = idx / RV, j = idx % RV;
       float M = wm[gg];
@@ -716,6 +747,7 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       if (*last_flag) {
         __threadfence();
         combine_unit<RV>(a.L, b, h, qt, first + u, nseg, a.partial_o, a.partial_lse, a.out, a.out_lse, un, tid, NT, lse_shift);
+        ++n_final;
       }
     }
     bar1(NT);
@@ -723,7 +755,6 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
   // units of empty sequences get their zero rows from CTA (u mod n_cta)
   if (a.out != nullptr) {
-    grid_dependency_wait();
     for (int u = c; u < B * upb; u += n_cta) {
       const int b = u / upb, j = u % upb;
       if (pref[b + 1] != pref[b]) continue;
@@ -732,9 +763,28 @@ decode_q_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const size_t head0 = (size_t)b * a.L.Hq + (size_t)h * G + (size_t)qt * kGroupTile;
       for (int idx = tid; idx < ng * kD; idx += NT) a.out[head0 * kD + idx] = __float2bfloat16_rn(0.f);
       if (a.out_lse && tid < ng) a.out_lse[head0 + tid] = -INFINITY;
+      ++n_final;
     }
   }
-  grid_dependency_wait();    // never finish before the kernel this one was allowed to overlap (keeps stream order transitive)
+  // Every unit is finalised by exactly one CTA (merged, or zero-filled).  The CTA that finalises the kernel's last unit
+  // publishes the kernel's epoch: from then on this section of the workspace is free for its next user.  That CTA also
+  // waits for the predecessor grid before it leaves, so that this grid never completes before an earlier one (stream
+  // order stays transitive); the others leave at once and hand their SMs to the next kernel.
+  if (a.out == nullptr) {
+    grid_dependency_wait();
+  } else if (n_final > 0) {
+    bar1(NT);                                              // all of the CTA's reads of partials and writes of outputs are issued
+    if (tid == 0) {
+      __threadfence();
+      const int before = atomicAdd(a.units_done, n_final);
+      if (before + n_final == B * upb) {
+        *a.units_done = 0;
+        __threadfence();
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.finished), "r"((int)a.epoch) : "memory");
+        grid_dependency_wait();
+      }
+    }
+  }
 }
 
 }  // namespace stief

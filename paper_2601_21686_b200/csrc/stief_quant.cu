@@ -209,7 +209,7 @@ int run_q_decode(int bits, const stief_qlayer* layer, const stief_batch* batch, 
   const int QT = query_tiles(layer->Hq, layer->Hkv);
   if ((long long)batch->B * (batch->max_pages_per_seq + seg_pad_pages(layer->r_k, layer->r_v)) * layer->Hkv * QT >= (1ll << 31))
     return STIEF_ERR_INVALID_ARG;
-  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta);
+  const Workspace w = carve(workspace, batch->B, layer->Hq, layer->Hkv, layer->r_v, n_cta, workspace_bytes);
   if (w.bytes > workspace_bytes) return STIEF_ERR_WORKSPACE;
   DecodeQArgs a;
   a.L = qlayer_to_dev(layer);
@@ -218,15 +218,18 @@ int run_q_decode(int bits, const stief_qlayer* layer, const stief_batch* batch, 
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
   a.k_new = reinterpret_cast<const __nv_bfloat16*>(k_new);
   a.v_new = reinterpret_cast<const __nv_bfloat16*>(v_new);
-  // this kernel keeps to the plain dependency wait before it touches the workspace: section 0, no epoch published
-  take_workspace_section0(workspace);
-  a.partial_o = w.partial_o[0]; a.partial_lse = w.partial_lse[0]; a.counters = w.counters[0];
+  const bool ov = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0 && n_cta >= sm_count();   // full grids only (see run_decode)
+  const WorkspaceTurn turn = take_workspace_turn(workspace);
+  a.partial_o = w.partial_o[turn.section]; a.partial_lse = w.partial_lse[turn.section]; a.counters = w.counters[turn.section];
+  a.finished = w.control + turn.section;
+  a.units_done = w.control + kWorkspaceSections + turn.section;
+  a.epoch = turn.epoch;
+  a.prev_epoch = ov ? turn.prev_epoch : 0u;
   a.out = reinterpret_cast<__nv_bfloat16*>(out);
   a.out_lse = out_lse;
   a.len_add = len_add;
   a.QT = QT;
   a.status = status;
-  const bool ov = (flags & STIEF_DECODE_OVERLAP_PREVIOUS) != 0 && n_cta >= sm_count();   // full grids only (see run_decode)
   return launch_decode_q(a, bits, n_cta, ov, static_cast<cudaStream_t>(stream)) == cudaSuccess ? STIEF_OK : STIEF_ERR_CUDA;
 }
 

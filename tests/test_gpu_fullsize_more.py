@@ -124,7 +124,8 @@ def test_quantised_config2_shape_prefill_and_overlapped_steps(bits, r_k, r_v):
     S.stief_decode_workspace_init(ws)
     n_steps = 4
     qs = [I.queries(60, 0, B, Hq, scale=1.0 / np.sqrt(128.0), device=DEV, step=i) for i in range(n_steps)]
-    kvs = [I.new_token_kv(60, 0, B, Hkv, device=DEV, step=i) for i in range(n_steps)]
+    # a layer cache that comes up again within the flagged run appends the same rows (the contract of the flag)
+    kvs = [I.new_token_kv(60, 0, B, Hkv, device=DEV, step=i % 2) for i in range(n_steps)]
     outs = [torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device=DEV) for _ in range(n_steps)]
     lses = [torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV) for _ in range(n_steps)]
     for i in range(n_steps):
