@@ -342,6 +342,59 @@ def test_flagged_chain_with_few_parts_over_two_caches_matches_serial(num_parts):
         assert torch.equal(a, b), f"step {i}"
 
 
+def test_flagged_chains_when_the_library_cannot_know_the_workspace_history():
+    # The overlap flag lets a kernel skip the wait for its predecessor when the library knows who used its workspace
+    # section last; where it cannot know, it must fall back to waiting.  Here: a captured graph of an ODD number of
+    # launches, all flagged (the first too), replayed several times, eager flagged launches in between (so the epochs
+    # baked into the graph are stale), and launches made from another host thread (whose record of the workspace is
+    # empty).  Every output must equal that of plain serial launches bit for bit.
+    import threading
+    B, Hq, Hkv = 3, 8, 2
+    ranks = [(128, 128), (32, 32), (64, 96)]
+    cs = [U.make_case(120 + l, B, Hq, Hkv, rk, rv, [2100, 700, 1300], reserve=8) for l, (rk, rv) in enumerate(ranks)]
+    for c in cs:
+        _prefill_and_check(c)
+    ws = U.workspace_for(cs[0], 0)                       # sized for r_v = 128, the largest of the three
+    ov = S.STIEF_DECODE_OVERLAP_PREVIOUS
+    qs = [I.queries(120, l, B, Hq).cuda() for l in range(3)]
+    kvs = [tuple(t.cuda() for t in I.new_token_kv(120, l, B, Hkv)) for l in range(3)]
+    mk = lambda: [torch.full((B, Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+
+    def step(outs, flags):
+        for l, c in enumerate(cs):
+            S.stief_decode_step(c.layer, c.batch, qs[l], kvs[l][0], kvs[l][1], ws, outs[l], status=c.status, flags=flags)
+
+    ref = mk()
+    step(ref, 0)
+    torch.cuda.synchronize()
+    g_out = mk()
+    graph = torch.cuda.CUDAGraph()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        with torch.cuda.graph(graph, stream=cap):
+            step(g_out, ov)
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for o in g_out:
+            o.fill_(float("nan"))
+        graph.replay()
+        graph.replay()
+        e_out = mk()
+        step(e_out, ov)                                   # eager, flagged, right behind a replay
+        t_out = mk()
+        th = threading.Thread(target=step, args=(t_out, ov))   # same stream, another host thread
+        th.start()
+        th.join()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert all(int(c.status.item()) == 0 for c in cs)
+        for l in range(3):
+            assert torch.equal(g_out[l], ref[l]), f"replayed graph, round {rep}, layer {l}"
+            assert torch.equal(e_out[l], ref[l]), f"eager launch after a replay, round {rep}, layer {l}"
+            assert torch.equal(t_out[l], ref[l]), f"launch from another thread, round {rep}, layer {l}"
+
+
 def test_overlapped_prefill_launches_match_serial_ones():
     # the per-layer prefill launches of one prompt, enqueued back to back with STIEF_PREFILL_OVERLAP_PREVIOUS
     B, Hq, Hkv = 2, 8, 2
