@@ -395,6 +395,37 @@ def test_flagged_chains_when_the_library_cannot_know_the_workspace_history():
             assert torch.equal(t_out[l], ref[l]), f"launch from another thread, round {rep}, layer {l}"
 
 
+def test_flagged_chain_with_empty_sequences_and_wide_groups_matches_serial():
+    # attention only (no append) over layers whose batches hold empty sequences (their units are zero-filled, which
+    # also counts towards a kernel's finalised units), groups of 16 query heads per KV head (two units per pair) and a
+    # batch that is empty altogether: the section bookkeeping must come out right for all of them, chained with the flag
+    ov = S.STIEF_DECODE_OVERLAP_PREVIOUS
+    specs = [(8, 2, 64, 64, [700, 0, 1300]), (32, 2, 128, 32, [0, 2500, 0]), (8, 2, 48, 96, [0, 0, 0]), (32, 2, 32, 128, [64, 1, 0])]
+    cs = [U.make_case(130 + i, 3, Hq, Hkv, rk, rv, lens) for i, (Hq, Hkv, rk, rv, lens) in enumerate(specs)]
+    for c in cs:
+        _prefill_and_check(c)
+    n_ws = max(S.stief_decode_workspace_bytes(3, c.Hq, c.Hkv, c.r_v, 0) for c in cs)
+    ws = torch.full((n_ws // 4,), float("nan"), dtype=torch.float32, device="cuda")
+    S.stief_decode_workspace_init(ws)
+    order = [0, 1, 2, 3, 2, 1, 0, 3, 3, 2]
+    res = {}
+    for flags in (0, ov):
+        outs = [torch.full((3, cs[l].Hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for l in order]
+        lses = [torch.full((3, cs[l].Hq), float("nan"), dtype=torch.float32, device="cuda") for l in order]
+        for i, l in enumerate(order):
+            c = cs[l]
+            S.stief_decode_attention(c.layer, c.batch, c.q.cuda(), ws, 0, outs[i], out_lse=lses[i], status=c.status, flags=flags if i else 0)
+        torch.cuda.synchronize()
+        assert all(int(c.status.item()) == 0 for c in cs)
+        res[flags] = (outs, lses)
+    for i, l in enumerate(order):
+        assert torch.equal(res[0][0][i], res[ov][0][i]) and torch.equal(res[0][1][i], res[ov][1][i]), f"launch {i} (layer {l})"
+        empty = np.asarray(specs[l][4]) == 0
+        o = res[ov][0][i].float().cpu().numpy()
+        assert not np.isnan(o).any() and not o[empty].any()                   # zero rows for empty sequences
+        assert np.isneginf(res[ov][1][i].cpu().numpy()[empty]).all()
+
+
 def test_overlapped_prefill_launches_match_serial_ones():
     # the per-layer prefill launches of one prompt, enqueued back to back with STIEF_PREFILL_OVERLAP_PREVIOUS
     B, Hq, Hkv = 2, 8, 2
