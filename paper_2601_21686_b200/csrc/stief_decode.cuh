@@ -639,7 +639,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
   }
   // Every unit is finalised by exactly one CTA (merged, or zero-filled).  The CTA that finalises the kernel's last unit
-  // publishes the kernel's epoch: from then on this half of the workspace is free for its next user.  That CTA also
+  // publishes the kernel's epoch: from then on this section of the workspace is free for its next user.  That CTA also
   // waits for the predecessor grid before it leaves, so that this grid never completes before an earlier one (stream
   // order stays transitive); the others leave at once and hand their SMs to the next kernel.
   if (a.out == nullptr) {
